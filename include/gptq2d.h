@@ -1,0 +1,125 @@
+/* gptq2d.h -- C ABI of the B200 (sm_100a) two-sided adaptive rounding library.
+ *
+ * Problem (paper Section 3.2, Eq. 6-9): given X (m x n, real) and nonsingular bases
+ * A (m x m), B (n x n), produce the integer matrix Z (m x n) that one-dimensional
+ * adaptive rounding (Algorithm 1: Babai nearest plane / GPTQ) yields on vec(X) under
+ * the Kronecker Gram (B B^T) (x) (A^T A).  GPTQ-2D (Algorithm 3, Theorem 2) reaches
+ * exactly that Z with O(m n max(m,n)) sweep work after an O(max(m,n)^3) set-up.
+ *
+ * Conventions for every call
+ *   - Matrix pointers are DEVICE pointers owned by the caller, row-major, with a
+ *     leading dimension given in elements (ld >= number of columns).  Pointers must
+ *     be 8-byte aligned; 16-byte alignment with even leading dimensions is faster.
+ *   - Nothing is allocated: scratch comes from a caller-provided device workspace
+ *     whose size the matching *_workspace_bytes query returns (256-byte aligned).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
+ *     enqueue work and return; they do not synchronise.
+ *   - The return value reports argument / launch errors found on the host
+ *     (gptq2d_status_t).  Data-dependent errors are written by the device into
+ *     `info` (device int[4]: {status, index, aux0, aux1}; may be NULL), valid once the
+ *     stream has been synchronised.  `info` is reset to zeros by each call.
+ *   - A and B are general nonsingular matrices.  No damping, permutation, clamping,
+ *     scale or zero point is applied: the paper rounds to all of Z^{m x n} in the
+ *     natural order.
+ *   - Requires an sm_100 device; anything else returns GPTQ2D_ERR_UNSUPPORTED_DEVICE.
+ *     There is no CPU fallback.
+ */
+#ifndef GPTQ2D_H
+#define GPTQ2D_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GPTQ2D_OK = 0,
+    GPTQ2D_ERR_INVALID_ARG = 1,        /* null pointer, m or n < 1, ld too small, misaligned pointer   */
+    GPTQ2D_ERR_WORKSPACE = 2,          /* workspace missing, misaligned or smaller than the query says  */
+    GPTQ2D_ERR_UNSUPPORTED_DEVICE = 3, /* current device is not compute capability 10.x                 */
+    GPTQ2D_ERR_CUDA = 4,               /* a CUDA runtime call failed (launch, attribute query, copy)    */
+    GPTQ2D_ERR_NOT_SPD = 5,            /* device: Gram pivot <= 0 or non-finite; info[1] = pivot index,
+                                          info[2] = 0 for A^T A, 1 for B B^T                            */
+    GPTQ2D_ERR_NONFINITE = 6,          /* device: NaN/Inf met while rounding; info[1] = row, info[2] = col */
+    GPTQ2D_ERR_INT_OVERFLOW = 7,       /* device: |corrected value| >= 2^31; info[1] = row, info[2] = col  */
+    GPTQ2D_ERR_DEVICE_TIMEOUT = 8      /* device: a bounded wait gave up; info[1] = where it waited     */
+} gptq2d_status_t;
+
+typedef enum {
+    GPTQ2D_FP64 = 0,   /* all sweep arithmetic in fp64 (tiled wavefront kernel)                       */
+    GPTQ2D_FP32 = 1,   /* X, L, U rounded to fp32 and all sweep arithmetic in fp32 (Algorithm 3 as
+                          written, one grid-wide barrier per anti-diagonal); Z may differ from FP64  */
+    GPTQ2D_FP64_UNTILED = 2 /* fp64 with the untiled Algorithm-3 kernel; a cross-check, not fast      */
+} gptq2d_precision_t;
+
+/* Human-readable name of a status code (static storage). */
+const char *gptq2d_status_string(int status);
+
+/* ---- set-up: feedback factors (Section 3.1; Section 4.1 below Eq. 9; Algorithm 3 lines 1-2) ----
+ * L (m x m): unit lower triangular, (A^T A)^{-1} = L Lambda_L L^T.
+ * U (n x n): unit upper triangular, (B B^T)^{-1} = U^T Lambda_U U.
+ * Computed without forming an inverse Gram: G = P^T P with P lower triangular (a Cholesky
+ * factorisation run from the last index to the first), L = P^{-1} diag(P), Lambda^{-1} = diag(P)^2.
+ * Outputs have exact ones on the diagonal and exact zeros in the opposite triangle.
+ * dL (m) / dU (n), optional (NULL ok): 1/Lambda_L and 1/Lambda_U, so that
+ * ||A (Z-X) B||_F^2 = sum_ij E_ij^2 dL_i dU_j for the local errors E.
+ * A or B may be NULL, meaning the identity (L or U is then the identity).
+ * Device error: GPTQ2D_ERR_NOT_SPD when a Gram is numerically not positive definite
+ * (A or B singular); L and U are then undefined.
+ */
+size_t gptq2d_factor_workspace_bytes(int m, int n);
+int gptq2d_factor(int m, int n,
+                  const double *A, long lda, const double *B, long ldb,
+                  double *L, long ldl, double *U, long ldu,
+                  double *dL, double *dU,
+                  void *workspace, size_t workspace_bytes, int *info, void *stream);
+
+/* ---- the sweep (Algorithm 3; tiled restatement via Eq. 11 and Eq. 15-17) ----
+ * Z (m x n, int32): Z_ij = round-half-even(Y_ij) with Y the corrected matrix.
+ * E (m x n), optional: local errors E_ij = Z_ij - Y_ij (Algorithm 3 line 5), each in [-1/2, 1/2].
+ * min_margin, optional device scalar: min_ij (1/2 - |E_ij|), the distance of the closest
+ *   pre-rounding value from a tie.
+ * L, U: as produced by gptq2d_factor (only the strict triangles are read; the unit diagonal
+ *   is implied).  They must stay fixed during the call (Section 6, first caveat).
+ * Initialisation (Y <- X, C <- 0; Algorithm 3 lines 4-5) is part of this call.
+ * Device errors: NONFINITE, INT_OVERFLOW (Z is int32), DEVICE_TIMEOUT.
+ * Calls on different streams must use different workspaces.
+ */
+size_t gptq2d_round_workspace_bytes(int m, int n, int precision);
+int gptq2d_round(int m, int n,
+                 const double *X, long ldx,
+                 const double *L, long ldl, const double *U, long ldu,
+                 int32_t *Z, long ldz,
+                 double *E, long lde, double *min_margin,
+                 int precision,
+                 void *workspace, size_t workspace_bytes, int *info, void *stream);
+
+/* Same sweep with HOST buffers: X, L, U are copied to the device workspace, the sweep runs, and
+ * Z (and E, min_margin if non-NULL) are copied back; all on `stream`, which is synchronised
+ * before returning.  hX, hL, hU, hZ, hE are host pointers (pinned memory makes the copies
+ * asynchronous and fast), dense row-major (leading dimension = number of columns).
+ * hinfo: host int[4], receives the device info words.  The workspace is still a device buffer.
+ */
+size_t gptq2d_round_host_workspace_bytes(int m, int n, int precision);
+int gptq2d_round_host(int m, int n,
+                      const double *hX, const double *hL, const double *hU,
+                      int32_t *hZ, double *hE, double *hmin_margin,
+                      int precision,
+                      void *workspace, size_t workspace_bytes, int *hinfo, void *stream);
+
+/* ---- the objective (Eq. 7): obj = || A (Z - X) B ||_F^2 ----
+ * obj: device scalar.  A or B may be NULL (identity).
+ */
+size_t gptq2d_objective_workspace_bytes(int m, int n);
+int gptq2d_objective(int m, int n,
+                     const double *X, long ldx, const int32_t *Z, long ldz,
+                     const double *A, long lda, const double *B, long ldb,
+                     double *obj,
+                     void *workspace, size_t workspace_bytes, int *info, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GPTQ2D_H */

@@ -1,0 +1,217 @@
+// Set-up of the feedback factors (Section 3.1 and Section 4.1; Algorithm 3 lines 1-2).
+//
+// For a Gram S (= A^T A, or B B^T) the paper wants the unit lower factor F of the LDL
+// decomposition of S^{-1}.  Writing S = P^T P with P LOWER triangular (a Cholesky
+// factorisation that eliminates from the last index to the first) gives
+//     S^{-1} = P^{-1} P^{-T} = F Lambda F^T,   F = P^{-1} diag(P),   Lambda^{-1} = diag(P)^2,
+// so no Gram inverse is ever formed.  L = F(A^T A); U = F(B B^T)^T.
+//
+// Blocked, right-looking, block size 128, from the last diagonal block to the first:
+//   diag kernel  : P_KK from the 128 x 128 Schur complement, and W_KK = P_KK^{-1}
+//   panel GEMM   : P_K,0:K = W_KK^T G_K,0:K
+//   trailing GEMM: G_0:K,0:K -= P_K,0:K^T P_K,0:K           (lower tiles only)
+// then the triangular inverse X = P^{-1} by recursive doubling over diagonal blocks
+//   X21 = -X22 (P21 X11)      (strided-batched GEMMs, one batch entry per block pair)
+// and a final column scaling (transposed on the way out for U).
+#include "common.cuh"
+#include "gemm.cuh"
+
+namespace gptq2d {
+
+constexpr int FB = 128;
+
+// One CTA.  S: bs x bs Schur complement (lower triangle read).  Writes P (lower, in place),
+// W = P^{-1} (full block, zeros above the diagonal) and diag(P).
+__global__ void __launch_bounds__(256) factor_diag_kernel(double *S, long lds, int bs, double *W, long ldw,
+                                                          double *pdiag, int *info, int side, int k0) {
+    extern __shared__ double sm[];
+    double *a = sm;               // [128][129]
+    double *w = sm + 128 * 129;   // [128][129]
+    const int tid = threadIdx.x;
+    for (int idx = tid; idx < bs * bs; idx += blockDim.x) {
+        int i = idx / bs, j = idx % bs;
+        if (j <= i) a[i * 129 + j] = S[(long)i * lds + j];
+        w[i * 129 + j] = 0.0;
+    }
+    __syncthreads();
+    for (int k = bs - 1; k >= 0; --k) {
+        double d = a[k * 129 + k];
+        __syncthreads();
+        if (!(d > 0.0) || !isfinite(d)) {
+            if (tid == 0) report(info, GPTQ2D_ERR_NOT_SPD, k0 + k, side, 0);
+            d = 1.0;
+        }
+        double pk = sqrt(d);
+        if (tid == 0) a[k * 129 + k] = pk;
+        for (int i = tid; i < k; i += blockDim.x) a[k * 129 + i] /= pk;     // P[k][i], i < k
+        __syncthreads();
+        // Schur complement of the leading k x k part (lower triangle)
+        for (int idx = tid; idx < k * k; idx += blockDim.x) {
+            int i = idx / k, j = idx % k;
+            if (j <= i) a[i * 129 + j] -= a[k * 129 + i] * a[k * 129 + j];
+        }
+        __syncthreads();
+    }
+    // W = P^{-1}: thread j owns column j (forward substitution down the column)
+    for (int j = tid; j < bs; j += blockDim.x) {
+        w[j * 129 + j] = 1.0 / a[j * 129 + j];
+        for (int i = j + 1; i < bs; ++i) {
+            double s = 0.0;
+            for (int k = j; k < i; ++k) s = fma(a[i * 129 + k], w[k * 129 + j], s);
+            w[i * 129 + j] = -s / a[i * 129 + i];
+        }
+    }
+    __syncthreads();
+    for (int idx = tid; idx < bs * bs; idx += blockDim.x) {
+        int i = idx / bs, j = idx % bs;
+        if (j <= i) S[(long)i * lds + j] = a[i * 129 + j];
+        W[(long)i * ldw + j] = w[i * 129 + j];
+    }
+    for (int i = tid; i < bs; i += blockDim.x) pdiag[i] = a[i * 129 + i];
+}
+
+// out[i][j] (transpose == 0) or out[j][i] (transpose == 1) = X[i][j] * p[j] below the
+// diagonal, 1 on it, 0 above; dinv[j] = p[j]^2.
+__global__ void __launch_bounds__(256) factor_finish_kernel(const double *X, long ldx, const double *p, int k,
+                                                            double *out, long ldo, int transpose, double *dinv) {
+    __shared__ double tile[32][33];
+    const int bi = blockIdx.y * 32, bj = blockIdx.x * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8
+    for (int r = ty; r < 32; r += 8) {
+        int i = bi + r, j = bj + tx;
+        double v = 0.0;
+        if (i < k && j < k) v = (i > j) ? X[(long)i * ldx + j] * p[j] : (i == j ? 1.0 : 0.0);
+        tile[r][tx] = v;
+    }
+    __syncthreads();
+    if (!transpose) {
+        for (int r = ty; r < 32; r += 8) {
+            int i = bi + r, j = bj + tx;
+            if (i < k && j < k) out[(long)i * ldo + j] = tile[r][tx];
+        }
+    } else {
+        for (int r = ty; r < 32; r += 8) {
+            int j = bj + r, i = bi + tx;      // out row = j, out col = i
+            if (i < k && j < k) out[(long)j * ldo + i] = tile[tx][r];
+        }
+    }
+    if (dinv && blockIdx.y == 0 && ty == 0) {
+        int j = bj + tx;
+        if (j < k) dinv[j] = p[j] * p[j];
+    }
+}
+
+__global__ void identity_kernel(double *out, long ldo, int k, double *dinv) {
+    long idx = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx < (long)k * k) {
+        int i = (int)(idx / k), j = (int)(idx % k);
+        out[(long)i * ldo + j] = (i == j) ? 1.0 : 0.0;
+    }
+    if (dinv && idx < k) dinv[idx] = 1.0;
+}
+
+static inline long round_up(long x, long a) { return (x + a - 1) / a * a; }
+
+size_t factor_workspace_bytes(int m, int n) {
+    long k = m > n ? m : n;
+    long ld = round_up(k, 16);
+    size_t mat = (size_t)ld * (size_t)round_up(k, 16) * sizeof(double);
+    return 3 * mat + (size_t)round_up(k, 32) * sizeof(double) + 256;
+}
+
+#define CK(x)                                          \
+    do {                                               \
+        if ((x) != cudaSuccess) return GPTQ2D_ERR_CUDA; \
+    } while (0)
+
+// side 0: S = M^T M -> out = F (unit lower).  side 1: S = M M^T -> out = F^T (unit upper).
+int factor_one_side(int k, const double *M, long ldm, int side, double *out, long ldo, double *dinv, void *ws,
+                    int *info, cudaStream_t stream) {
+    if (!M) {
+        long tot = (long)k * k;
+        identity_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, stream>>>(out, ldo, k, dinv);
+        CK(cudaGetLastError());
+        return GPTQ2D_OK;
+    }
+    const long ld = round_up(k, 16);
+    const size_t mat = (size_t)ld * (size_t)round_up(k, 16);
+    double *G = static_cast<double *>(ws);
+    double *X = G + mat;
+    double *T = X + mat;
+    double *p = T + mat;
+    const int nblk = (k + FB - 1) / FB;
+
+    CK(cudaMemsetAsync(X, 0, mat * sizeof(double), stream));
+    {   // Gram, lower tiles: S = M^T M or M M^T
+        GemmArgs g{};
+        g.opA = side == 0 ? OP_T : OP_N;
+        g.opB = side == 0 ? OP_N : OP_T;
+        g.M = g.N = g.K = k;
+        g.alpha = 1.0; g.beta = 0.0;
+        g.A = M; g.lda = ldm; g.B = M; g.ldb = ldm;
+        g.C = G; g.ldc = ld; g.batch = 1; g.lower_tiles_only = 1;
+        CK(launch_gemm(g, stream));
+    }
+    const size_t diag_smem = 2 * 128 * 129 * sizeof(double);
+    CK(cudaFuncSetAttribute(factor_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)diag_smem));
+    for (int K = nblk - 1; K >= 0; --K) {
+        const long k0 = (long)K * FB;
+        const int bs = (int)((k - k0) < FB ? (k - k0) : FB);
+        double *Gkk = G + k0 * ld + k0;
+        double *Wkk = X + k0 * ld + k0;
+        factor_diag_kernel<<<1, 256, diag_smem, stream>>>(Gkk, ld, bs, Wkk, ld, p + k0, info, side, (int)k0);
+        CK(cudaGetLastError());
+        if (K == 0) break;
+        GemmArgs g{};   // panel, in place: P_K,0:k0 = W^T G_K,0:k0
+        g.opA = OP_T; g.opB = OP_N;
+        g.M = bs; g.N = (int)k0; g.K = bs;
+        g.alpha = 1.0; g.beta = 0.0;
+        g.A = Wkk; g.lda = ld; g.B = G + k0 * ld; g.ldb = ld;
+        g.C = G + k0 * ld; g.ldc = ld; g.batch = 1;
+        CK(launch_gemm(g, stream));
+        GemmArgs t{};   // trailing: G_0:k0,0:k0 -= panel^T panel
+        t.opA = OP_T; t.opB = OP_N;
+        t.M = t.N = (int)k0; t.K = bs;
+        t.alpha = -1.0; t.beta = 1.0;
+        t.A = G + k0 * ld; t.lda = ld; t.B = G + k0 * ld; t.ldb = ld;
+        t.C = G; t.ldc = ld; t.batch = 1; t.lower_tiles_only = 1;
+        CK(launch_gemm(t, stream));
+    }
+    // X = P^{-1}: diagonal blocks are in place; double the block size level by level
+    for (long b = FB; b < k; b *= 2) {
+        const long npair_full = k / (2 * b);            // pairs with two full halves
+        const long rem = k - npair_full * 2 * b;        // what is left after them
+        for (int pass = 0; pass < 2; ++pass) {
+            long s0, b2, cnt;
+            if (pass == 0) { s0 = 0; b2 = b; cnt = npair_full; }
+            else { s0 = npair_full * 2 * b; b2 = rem - b; cnt = 1; }
+            if (cnt <= 0 || b2 <= 0) continue;
+            const long off11 = s0 * ld + s0, off21 = (s0 + b) * ld + s0, off22 = (s0 + b) * ld + (s0 + b);
+            const long stride = 2 * b * (ld + 1);
+            GemmArgs g1{};   // T21 = P21 X11
+            g1.opA = OP_N; g1.opB = OP_N;
+            g1.M = (int)b2; g1.N = (int)b; g1.K = (int)b;
+            g1.alpha = 1.0; g1.beta = 0.0;
+            g1.A = G + off21; g1.lda = ld; g1.strideA = stride;
+            g1.B = X + off11; g1.ldb = ld; g1.strideB = stride;
+            g1.C = T + off21; g1.ldc = ld; g1.strideC = stride;
+            g1.batch = (int)cnt;
+            CK(launch_gemm(g1, stream));
+            GemmArgs g2{};   // X21 = -X22 T21
+            g2.opA = OP_N; g2.opB = OP_N;
+            g2.M = (int)b2; g2.N = (int)b; g2.K = (int)b2;
+            g2.alpha = -1.0; g2.beta = 0.0;
+            g2.A = X + off22; g2.lda = ld; g2.strideA = stride;
+            g2.B = T + off21; g2.ldb = ld; g2.strideB = stride;
+            g2.C = X + off21; g2.ldc = ld; g2.strideC = stride;
+            g2.batch = (int)cnt;
+            CK(launch_gemm(g2, stream));
+        }
+    }
+    dim3 grid((k + 31) / 32, (k + 31) / 32);
+    factor_finish_kernel<<<grid, 256, 0, stream>>>(X, ld, p, k, out, ldo, side, dinv);
+    CK(cudaGetLastError());
+    return GPTQ2D_OK;
+}
+
+}  // namespace gptq2d

@@ -1,0 +1,28 @@
+// Host-side interface of the library's own fp64 GEMM (DMMA tiles, see dmma_gemm.cuh).
+// Used by the set-up (Gram, blocked Cholesky, triangular inverse) and by the objective.
+#pragma once
+#include <cuda_runtime.h>
+
+namespace gptq2d {
+
+enum GemmOp { OP_N = 0, OP_T = 1 };
+
+struct GemmArgs {
+    // C[b] = alpha * op(A[b]) * op(B[b]) + beta * C[b]   for b in [0, batch)
+    // op(A) is M x K, op(B) is K x N, all row-major with leading dimensions in elements.
+    GemmOp opA, opB;
+    int M, N, K;
+    double alpha, beta;
+    const double *A; long lda; long strideA;
+    const double *B; long ldb; long strideB;
+    double *C; long ldc; long strideC;
+    int batch;
+    int lower_tiles_only;   // skip 128 x 128 output tiles strictly above the block diagonal
+    double *sumsq_partials; // if non-null: do not store C; write sum(C^2) of each CTA tile
+                            // to sumsq_partials[tile index] (tiles_m * tiles_n * batch entries)
+};
+
+// Enqueues the GEMM on `stream`.  Returns cudaSuccess or the launch error.
+cudaError_t launch_gemm(const GemmArgs &g, cudaStream_t stream);
+
+}  // namespace gptq2d

@@ -1,0 +1,38 @@
+// Internal launch interfaces of the sweep kernels (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include "common.cuh"
+
+namespace gptq2d {
+
+struct UntiledParams {
+    int m, n;
+    const double *X; long ldx;
+    const double *L; long ldl;
+    const double *U; long ldu;
+    int *Z; long ldz;
+    double *E; long lde;      // optional
+    double *max_abs_e;        // workspace scalar, max |E| over the matrix
+    int *info;
+    void *Ybuf, *Cbuf;        // m x n working copies (fp64 or fp32), dense
+    GridSync sync;
+};
+size_t round_untiled_workspace_bytes(int m, int n, bool fp32);
+int launch_round_untiled(const UntiledParams &p, bool fp32, void *ws, cudaStream_t stream);
+
+struct TiledParams {
+    int m, n;
+    const double *X; long ldx;
+    const double *L; long ldl;
+    const double *U; long ldu;
+    int *Z; long ldz;
+    double *E; long lde;      // optional user copy of the local errors
+    double *max_abs_e;
+    int *info;
+};
+size_t round_tiled_workspace_bytes(int m, int n);
+int launch_round_tiled(const TiledParams &p, void *ws, size_t ws_bytes, cudaStream_t stream);
+// where the max |E| scalar lives inside either workspace
+inline double *workspace_max_abs_e(void *ws) { return reinterpret_cast<double *>(static_cast<char *>(ws) + 64); }
+
+}  // namespace gptq2d

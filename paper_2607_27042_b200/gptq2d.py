@@ -1,0 +1,215 @@
+"""Thin ctypes binding over libgptq2d.so (the C ABI of include/gptq2d.h).
+
+Argument marshalling only: every step of the method runs in the CUDA library.
+PyTorch supplies device memory and streams.  There is no CPU fallback: importing
+this module raises if the library has not been built.
+
+Function names mirror the C entry points.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libgptq2d.so")
+
+FP64, FP32, FP64_UNTILED = 0, 1, 2
+
+OK = 0
+STATUS_NAMES = {
+    0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_WORKSPACE", 3: "ERR_UNSUPPORTED_DEVICE", 4: "ERR_CUDA",
+    5: "ERR_NOT_SPD", 6: "ERR_NONFINITE", 7: "ERR_INT_OVERFLOW", 8: "ERR_DEVICE_TIMEOUT",
+}
+
+EXPORTS = (
+    "gptq2d_status_string", "gptq2d_factor_workspace_bytes", "gptq2d_factor",
+    "gptq2d_round_workspace_bytes", "gptq2d_round", "gptq2d_round_host_workspace_bytes",
+    "gptq2d_round_host", "gptq2d_objective_workspace_bytes", "gptq2d_objective",
+)
+
+
+class Gptq2dError(RuntimeError):
+    def __init__(self, status, info=None):
+        self.status = int(status)
+        self.info = info
+        name = STATUS_NAMES.get(self.status, str(status))
+        super().__init__("gptq2d: %s%s" % (name, "" if info is None else " info=%s" % (list(info),)))
+
+
+def _load():
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(
+            "libgptq2d.so is not built (%s). Run `python -m paper_2607_27042_b200.build` "
+            "or __graft_entry__.build(); there is no CPU fallback." % _LIB_PATH)
+    lib = ctypes.CDLL(_LIB_PATH)
+    c = ctypes
+    vp, sz, i32, lng = c.c_void_p, c.c_size_t, c.c_int, c.c_long
+    lib.gptq2d_status_string.restype = c.c_char_p
+    lib.gptq2d_status_string.argtypes = [i32]
+    for name in ("gptq2d_factor_workspace_bytes", "gptq2d_objective_workspace_bytes"):
+        getattr(lib, name).restype = sz
+        getattr(lib, name).argtypes = [i32, i32]
+    for name in ("gptq2d_round_workspace_bytes", "gptq2d_round_host_workspace_bytes"):
+        getattr(lib, name).restype = sz
+        getattr(lib, name).argtypes = [i32, i32, i32]
+    lib.gptq2d_factor.restype = i32
+    lib.gptq2d_factor.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, vp, sz, vp, vp]
+    lib.gptq2d_round.restype = i32
+    lib.gptq2d_round.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, lng, vp, i32, vp, sz, vp, vp]
+    lib.gptq2d_round_host.restype = i32
+    lib.gptq2d_round_host.argtypes = [i32, i32, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp, vp]
+    lib.gptq2d_objective.restype = i32
+    lib.gptq2d_objective.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, sz, vp, vp]
+    return lib
+
+
+_lib = _load()
+
+
+def library_path():
+    return _LIB_PATH
+
+
+def status_string(status):
+    return _lib.gptq2d_status_string(int(status)).decode()
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _mat(t, dtype, name):
+    if t is None:
+        return None, 0
+    if not (t.is_cuda and t.dtype == dtype and t.dim() == 2 and t.stride(1) == 1):
+        raise ValueError("%s must be a 2-D CUDA tensor of %s with unit column stride" % (name, dtype))
+    return ctypes.c_void_p(t.data_ptr()), int(t.stride(0))
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _workspace(nbytes, device):
+    # torch's caching allocator returns 512-byte aligned blocks
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def check_info(info):
+    """Synchronises and raises if the device reported a data-dependent error."""
+    vals = info.cpu().tolist()
+    if vals[0] != 0:
+        raise Gptq2dError(vals[0], vals)
+
+
+def gptq2d_factor_workspace_bytes(m, n):
+    return int(_lib.gptq2d_factor_workspace_bytes(m, n))
+
+
+def gptq2d_round_workspace_bytes(m, n, precision=FP64):
+    return int(_lib.gptq2d_round_workspace_bytes(m, n, precision))
+
+
+def gptq2d_round_host_workspace_bytes(m, n, precision=FP64):
+    return int(_lib.gptq2d_round_host_workspace_bytes(m, n, precision))
+
+
+def gptq2d_objective_workspace_bytes(m, n):
+    return int(_lib.gptq2d_objective_workspace_bytes(m, n))
+
+
+def gptq2d_factor(A, B, L=None, U=None, dL=None, dU=None, workspace=None, info=None, stream=None, m=None, n=None):
+    """L, U (and 1/Lambda_L, 1/Lambda_U) from the bases A (m x m) and B (n x n).
+
+    A or B may be None (identity) if m / n is given.  Returns (L, U, dL, dU, info)."""
+    m = A.shape[0] if A is not None else m
+    n = B.shape[0] if B is not None else n
+    dev = (A if A is not None else B).device if (A is not None or B is not None) else torch.device("cuda")
+    L = torch.empty((m, m), dtype=torch.float64, device=dev) if L is None else L
+    U = torch.empty((n, n), dtype=torch.float64, device=dev) if U is None else U
+    dL = torch.empty(m, dtype=torch.float64, device=dev) if dL is None else dL
+    dU = torch.empty(n, dtype=torch.float64, device=dev) if dU is None else dU
+    info = torch.zeros(4, dtype=torch.int32, device=dev) if info is None else info
+    nbytes = gptq2d_factor_workspace_bytes(m, n)
+    workspace = _workspace(nbytes, dev) if workspace is None else workspace
+    pA, lda = _mat(A, torch.float64, "A")
+    pB, ldb = _mat(B, torch.float64, "B")
+    pL, ldl = _mat(L, torch.float64, "L")
+    pU, ldu = _mat(U, torch.float64, "U")
+    st = _lib.gptq2d_factor(m, n, pA, lda, pB, ldb, pL, ldl, pU, ldu, _ptr(dL), _ptr(dU),
+                            _ptr(workspace), workspace.numel(), _ptr(info), _stream_ptr(stream))
+    if st != OK:
+        raise Gptq2dError(st)
+    return L, U, dL, dU, info
+
+
+def gptq2d_round(X, L, U, Z=None, E=None, min_margin=None, precision=FP64, workspace=None, info=None,
+                 stream=None, want_E=False, want_margin=False):
+    """The sweep.  Returns (Z, E, min_margin, info); E / min_margin are None unless asked for."""
+    m, n = X.shape
+    dev = X.device
+    Z = torch.empty((m, n), dtype=torch.int32, device=dev) if Z is None else Z
+    if E is None and want_E:
+        E = torch.empty((m, n), dtype=torch.float64, device=dev)
+    if min_margin is None and want_margin:
+        min_margin = torch.empty(1, dtype=torch.float64, device=dev)
+    info = torch.zeros(4, dtype=torch.int32, device=dev) if info is None else info
+    nbytes = gptq2d_round_workspace_bytes(m, n, precision)
+    workspace = _workspace(nbytes, dev) if workspace is None else workspace
+    pX, ldx = _mat(X, torch.float64, "X")
+    pL, ldl = _mat(L, torch.float64, "L")
+    pU, ldu = _mat(U, torch.float64, "U")
+    pZ, ldz = _mat(Z, torch.int32, "Z")
+    pE, lde = _mat(E, torch.float64, "E")
+    st = _lib.gptq2d_round(m, n, pX, ldx, pL, ldl, pU, ldu, pZ, ldz, pE, lde, _ptr(min_margin), int(precision),
+                           _ptr(workspace), workspace.numel(), _ptr(info), _stream_ptr(stream))
+    if st != OK:
+        raise Gptq2dError(st)
+    return Z, E, min_margin, info
+
+
+def gptq2d_round_host(hX, hL, hU, hZ=None, hE=None, hmargin=None, precision=FP64, workspace=None, hinfo=None,
+                      stream=None, device=None):
+    """Host-buffer variant: hX, hL, hU are CPU tensors (pinned for speed); copies in, sweeps, copies Z back,
+    synchronises.  Returns (hZ, hinfo)."""
+    m, n = hX.shape
+    for t, name in ((hX, "hX"), (hL, "hL"), (hU, "hU")):
+        if t.is_cuda or t.dtype != torch.float64 or not t.is_contiguous():
+            raise ValueError("%s must be a contiguous CPU float64 tensor" % name)
+    device = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    hZ = torch.empty((m, n), dtype=torch.int32).pin_memory() if hZ is None else hZ
+    hinfo = torch.zeros(4, dtype=torch.int32).pin_memory() if hinfo is None else hinfo
+    nbytes = gptq2d_round_host_workspace_bytes(m, n, precision)
+    workspace = _workspace(nbytes, device) if workspace is None else workspace
+    st = _lib.gptq2d_round_host(m, n, _ptr(hX), _ptr(hL), _ptr(hU), _ptr(hZ), _ptr(hE), _ptr(hmargin),
+                                int(precision), _ptr(workspace), workspace.numel(), _ptr(hinfo),
+                                _stream_ptr(stream))
+    if st != OK:
+        raise Gptq2dError(st)
+    if int(hinfo[0]) != 0:
+        raise Gptq2dError(int(hinfo[0]), hinfo.tolist())
+    return hZ, hinfo
+
+
+def gptq2d_objective(X, Z, A, B, obj=None, workspace=None, info=None, stream=None):
+    """|| A (Z - X) B ||_F^2 as a 1-element CUDA tensor.  A or B may be None (identity)."""
+    m, n = X.shape
+    dev = X.device
+    obj = torch.empty(1, dtype=torch.float64, device=dev) if obj is None else obj
+    info = torch.zeros(4, dtype=torch.int32, device=dev) if info is None else info
+    nbytes = gptq2d_objective_workspace_bytes(m, n)
+    workspace = _workspace(nbytes, dev) if workspace is None else workspace
+    pX, ldx = _mat(X, torch.float64, "X")
+    pZ, ldz = _mat(Z, torch.int32, "Z")
+    pA, lda = _mat(A, torch.float64, "A")
+    pB, ldb = _mat(B, torch.float64, "B")
+    st = _lib.gptq2d_objective(m, n, pX, ldx, pZ, ldz, pA, lda, pB, ldb, _ptr(obj), _ptr(workspace),
+                               workspace.numel(), _ptr(info), _stream_ptr(stream))
+    if st != OK:
+        raise Gptq2dError(st)
+    return obj
