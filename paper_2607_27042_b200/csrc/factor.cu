@@ -26,12 +26,11 @@ __global__ void __launch_bounds__(256) factor_diag_kernel(double *S, long lds, i
                                                           double *pdiag, int *info, int side, int k0) {
     extern __shared__ double sm[];
     double *a = sm;               // [128][129]
-    double *w = sm + 128 * 129;   // [128][129]
+    double *w = sm + 128 * 129;   // packed lower triangle: (i, j <= i) at i(i+1)/2 + j
     const int tid = threadIdx.x;
     for (int idx = tid; idx < bs * bs; idx += blockDim.x) {
         int i = idx / bs, j = idx % bs;
         if (j <= i) a[i * 129 + j] = S[(long)i * lds + j];
-        w[i * 129 + j] = 0.0;
     }
     __syncthreads();
     for (int k = bs - 1; k >= 0; --k) {
@@ -54,18 +53,18 @@ __global__ void __launch_bounds__(256) factor_diag_kernel(double *S, long lds, i
     }
     // W = P^{-1}: thread j owns column j (forward substitution down the column)
     for (int j = tid; j < bs; j += blockDim.x) {
-        w[j * 129 + j] = 1.0 / a[j * 129 + j];
+        w[j * (j + 1) / 2 + j] = 1.0 / a[j * 129 + j];
         for (int i = j + 1; i < bs; ++i) {
             double s = 0.0;
-            for (int k = j; k < i; ++k) s = fma(a[i * 129 + k], w[k * 129 + j], s);
-            w[i * 129 + j] = -s / a[i * 129 + i];
+            for (int k = j; k < i; ++k) s = fma(a[i * 129 + k], w[k * (k + 1) / 2 + j], s);
+            w[i * (i + 1) / 2 + j] = -s / a[i * 129 + i];
         }
     }
     __syncthreads();
     for (int idx = tid; idx < bs * bs; idx += blockDim.x) {
         int i = idx / bs, j = idx % bs;
         if (j <= i) S[(long)i * lds + j] = a[i * 129 + j];
-        W[(long)i * ldw + j] = w[i * 129 + j];
+        W[(long)i * ldw + j] = (j <= i) ? w[i * (i + 1) / 2 + j] : 0.0;
     }
     for (int i = tid; i < bs; i += blockDim.x) pdiag[i] = a[i * 129 + i];
 }
@@ -152,7 +151,7 @@ int factor_one_side(int k, const double *M, long ldm, int side, double *out, lon
         g.C = G; g.ldc = ld; g.batch = 1; g.lower_tiles_only = 1;
         CK(launch_gemm(g, stream));
     }
-    const size_t diag_smem = 2 * 128 * 129 * sizeof(double);
+    const size_t diag_smem = (128 * 129 + 128 * 129 / 2) * sizeof(double);
     CK(cudaFuncSetAttribute(factor_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)diag_smem));
     for (int K = nblk - 1; K >= 0; --K) {
         const long k0 = (long)K * FB;
