@@ -20,11 +20,10 @@
 //
 // In-tile sweep.  The tile is processed as four 64 x 64 quadrants (the same restatement one
 // level down, cross terms as 64^3 DMMA products).  Inside a quadrant the anti-diagonal
-// sweep runs on 8 x 8 leaves: the leaves of one leaf-wave are swept by groups of 8 lanes
-// (lane = row; each row is kept in registers rotated by its row index, so that at step s
-// every lane touches register slot s mod 8; downward pushes travel by warp shuffle, with the
-// lane's L coefficients held in registers), then all warps apply the leaves' feedback to
-// the remaining 8 x 8 blocks of the quadrant with m8n8k4 DMMA.
+// sweep runs on 8 x 8 leaves: each leaf of a leaf-wave is swept by one warp (two entries per
+// lane, errors exchanged through a 16-double shared-memory buffer, branch-free pushes), then
+// all warps apply the leaves' feedback to the remaining 8 x 8 blocks of the quadrant with
+// m8n8k4 DMMA.
 #include "common.cuh"
 #include "dmma_gemm.cuh"
 #include "round_internal.cuh"
@@ -35,6 +34,7 @@ constexpr int T = 128;           // tile edge
 constexpr int Q = 64;            // quadrant edge
 constexpr int QLD = 68;          // shared-memory row stride of quadrant matrices (68 mod 16 == 4)
 constexpr int QMAT = Q * QLD;    // doubles per quadrant matrix
+constexpr int TAB_LD = 24;       // row stride of the leaf coefficient tables (22 used)
 constexpr int BULK_NSTAGE = 4;
 constexpr int TILED_THREADS = 256;
 
@@ -55,7 +55,7 @@ struct TiledKernelParams {
     int l_al16, u_al16;
 };
 
-constexpr size_t SWEEP_SMEM = (size_t)5 * QMAT * sizeof(double) + (size_t)Q * Q * sizeof(int);
+constexpr size_t SWEEP_SMEM = (size_t)(5 * QMAT + 2 * Q * TAB_LD) * sizeof(double) + (size_t)Q * Q * sizeof(int);
 constexpr size_t BULK_SMEM = (size_t)BULK_NSTAGE * SlabLayout<true, false>::STAGE_DOUBLES * sizeof(double);
 constexpr size_t TILED_SMEM = SWEEP_SMEM > BULK_SMEM ? SWEEP_SMEM : BULK_SMEM;
 
@@ -98,17 +98,20 @@ __device__ __forceinline__ int wait_ready_prefix(const unsigned *flags, long str
 }
 
 // ---------------------------------------------------------------------------------------------
-// quadrant <-> shared memory
-__device__ __forceinline__ void load_quadrant_cg(double *dst, const double *src, long ld) {
-    // dense 64 x 64 from a padded workspace buffer (always in range, 16-byte aligned)
-    for (int c = threadIdx.x; c < Q * Q / 2; c += blockDim.x) {
-        int r = c >> 5, cc = (c & 31) * 2;
-        double2 v = __ldcg(reinterpret_cast<const double2 *>(src + (long)r * ld + cc));
-        *reinterpret_cast<double2 *>(dst + r * QLD + cc) = v;
+// quadrant <-> shared memory.  The *_async loaders only issue cp.async copies; the caller
+// commits, waits and barriers once for all operands of a quadrant.
+__device__ __forceinline__ void load_quadrant_async(double *dst, const double *src, long ld) {
+    // dense 64 x 64 from a padded workspace buffer (always in range, 16-byte aligned); L2 only
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+        int c = threadIdx.x + it * TILED_THREADS;
+        cp_async16(dst + (c >> 5) * QLD + (c & 31) * 2, src + (long)(c >> 5) * ld + (c & 31) * 2, 16);
     }
 }
 __device__ __forceinline__ void store_quadrant(double *dst, long ld, const double *src) {
-    for (int c = threadIdx.x; c < Q * Q / 2; c += blockDim.x) {
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+        int c = threadIdx.x + it * TILED_THREADS;
         int r = c >> 5, cc = (c & 31) * 2;
         *reinterpret_cast<double2 *>(dst + (long)r * ld + cc) = *reinterpret_cast<const double2 *>(src + r * QLD + cc);
     }
@@ -116,17 +119,17 @@ __device__ __forceinline__ void store_quadrant(double *dst, long ld, const doubl
 // 64 x 64 block of a user matrix (k x k, leading dimension ld) whose top-left element is
 // (r0, c0); mode 0: everything in range, 1: strictly lower part only, 2: strictly upper only
 // (relative to the matrix diagonal).  Out-of-range and masked elements become zero.
-__device__ __forceinline__ void load_factor_block(double *dst, const double *M, long ld, int k, int r0, int c0,
-                                                  int mode) {
-    for (int c = threadIdx.x; c < Q * Q; c += blockDim.x) {
+__device__ __forceinline__ void load_factor_block_async(double *dst, const double *M, long ld, int k, int r0, int c0,
+                                                        int mode) {
+#pragma unroll
+    for (int it = 0; it < 16; ++it) {
+        int c = threadIdx.x + it * TILED_THREADS;
         int r = c >> 6, cc = c & 63;
         int gr = r0 + r, gc = c0 + cc;
-        double v = 0.0;
         bool take = gr < k && gc < k;
         if (mode == 1) take = take && gc < gr;
         if (mode == 2) take = take && gc > gr;
-        if (take) v = __ldg(M + (long)gr * ld + gc);
-        dst[r * QLD + cc] = v;
+        cp_async8(dst + r * QLD + cc, take ? M + (long)gr * ld + gc : M, take ? 8 : 0);
     }
 }
 
@@ -163,6 +166,35 @@ __device__ __forceinline__ void cross_gemm(double *G, long ld, const double *As,
         }
 }
 
+// One 8 x 8 target block (pb, qb) of the quadrant receives the feedback of leaf-wave `lw`:
+// the downward push of leaf (lw - qb, qb) through L and the rightward push of leaf
+// (pb, lw - pb) through U, as m8n8k4 products on the warp's fragments.  Warp-uniform.
+__device__ __forceinline__ void block_feedback(double *Ys, double *Cs, const double *Ls, const double *Us, int lw,
+                                               int pb, int qb, int g, int t) {
+    const int asrc = lw - qb, bsrc = lw - pb;
+    const bool down = asrc >= 0 && asrc < pb, right = bsrc >= 0 && bsrc < qb;
+    if (!down && !right) return;
+    double *yp = Ys + (pb * 8 + g) * QLD + qb * 8 + t * 2;
+    double2 yv = *reinterpret_cast<double2 *>(yp);
+    if (down) {
+        double p0 = 0.0, p1 = 0.0;
+        dmma_m8n8k4(p0, p1, Ls[(pb * 8 + g) * QLD + asrc * 8 + t], Ys[(asrc * 8 + t) * QLD + qb * 8 + g]);
+        dmma_m8n8k4(p0, p1, Ls[(pb * 8 + g) * QLD + asrc * 8 + 4 + t], Ys[(asrc * 8 + 4 + t) * QLD + qb * 8 + g]);
+        double *cp = Cs + (pb * 8 + g) * QLD + qb * 8 + t * 2;
+        double2 cv = *reinterpret_cast<double2 *>(cp);
+        cv.x += p0;
+        cv.y += p1;
+        *reinterpret_cast<double2 *>(cp) = cv;
+        yv.x += p0;
+        yv.y += p1;
+    }
+    if (right) {
+        dmma_m8n8k4(yv.x, yv.y, Cs[(pb * 8 + g) * QLD + bsrc * 8 + t], Us[(bsrc * 8 + t) * QLD + qb * 8 + g]);
+        dmma_m8n8k4(yv.x, yv.y, Cs[(pb * 8 + g) * QLD + bsrc * 8 + 4 + t], Us[(bsrc * 8 + 4 + t) * QLD + qb * 8 + g]);
+    }
+    *reinterpret_cast<double2 *>(yp) = yv;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Algorithm 3 on one 64 x 64 quadrant held in shared memory.
 //   Ys: in  Y (corrected values, already including the C the quadrant starts with)
@@ -171,115 +203,114 @@ __device__ __forceinline__ void cross_gemm(double *G, long ld, const double *As,
 //   Ls / Us: strictly lower / strictly upper 64 x 64 diagonal blocks of the factors
 //   Zs: out rounded integers
 // row0/col0: global coordinates of the quadrant (for masking the status checks).
+//
+// Leaf-wave lw (leaves (a, lw - a)) runs in two barrier-separated parts:
+//   part 1: each leaf is swept by one warp (phase A); meanwhile every warp applies the feedback
+//           of the PREVIOUS leaf-wave to the blocks of its block row that lie two or more
+//           leaf-waves ahead (interleaved with the sweep steps, which are latency bound);
+//   part 2: every warp applies the feedback of THIS leaf-wave to the one block of its block
+//           row that belongs to the next leaf-wave.
 __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const double *Ls, const double *Us, int *Zs,
-                                               int row0, int col0, const TiledKernelParams &p, double &max_abs_e) {
+                                               double *tabL, double *tabU, int row0, int col0,
+                                               const TiledKernelParams &p, double &max_abs_e) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, t = lane & 3;
+    __shared__ double xch[8 * 2 * 16];
+    __shared__ unsigned long long s_badkey;
+    // coefficient tables of the 8 diagonal leaves (see phase A); also clears the exchange buffers
+    for (int c = tid; c < Q * TAB_LD; c += blockDim.x) {
+        const int r = c / TAB_LD, k = c - r * TAB_LD;       // r: row (L) or column (U) inside the quadrant
+        const int src = k - 7, blk = r & ~7, in = r & 7;    // source index inside the leaf
+        const bool ok = src >= 0 && src < in;
+        tabL[c] = ok ? Ls[r * QLD + blk + src] : 0.0;
+        tabU[c] = ok ? Us[(blk + src) * QLD + r] : 0.0;
+    }
+    if (tid < 8 * 2 * 16) xch[tid] = 0.0;
+    if (tid == 0) s_badkey = ~0ull;
+    unsigned long long badkey = ~0ull;
+
     for (int lw = 0; lw < 15; ++lw) {
         __syncthreads();
-        // ---------------- phase A: sweep the leaves (a, lw - a) of this leaf-wave
-        if (warp < 2) {
-            const int a_lo = max(0, lw - 7), a_hi = min(7, lw);
-            const int grp = tid >> 3, i = tid & 7;          // 8 groups of 8 lanes in warps 0-1
-            const int a = a_lo + grp, b = lw - a;
-            const bool live = a <= a_hi;
-            double y[8], c[8], lrow[8];
-            int z[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                int j = (k - i) & 7;                         // slot k holds column j of the leaf row
-                y[k] = live ? Ys[(a * 8 + i) * QLD + b * 8 + j] : 0.0;
-                c[k] = live ? Cs[(a * 8 + i) * QLD + b * 8 + j] : 0.0;
-                z[k] = 0;
-            }
-#pragma unroll
-            for (int d = 1; d < 8; ++d) lrow[d] = (live && i - d >= 0) ? Ls[(a * 8 + i) * QLD + a * 8 + i - d] : 0.0;
+        // ---------------- part 1
+        const int a_lo = max(0, lw - 7), a_hi = min(7, lw);
+        const int a = a_lo + warp, b = lw - a;
+        if (a <= a_hi) {
+            // Phase A.  Lane l owns entries (i0, j) and (i0 + 4, j) of the 8 x 8 leaf, i0 = l & 3,
+            // j = l >> 2.  At step s the lane whose entry lies on anti-diagonal s rounds it and posts
+            // the error (by column) and the final C value (by row) to a 16-double per-warp exchange
+            // buffer; after a warp barrier EVERY lane applies one downward and one rightward push
+            // to both of its entries (Algorithm 3 lines 8-16 restricted to the leaf).  The pushes
+            // are branch-free: the coefficients come from tables that hold zeros wherever no push
+            // is due (source not on this anti-diagonal, or entry already rounded), so stale
+            // exchange slots are multiplied by zero.
+            const int i0 = lane & 3, j = lane >> 2;
+            double *yp = Ys + (a * 8 + i0) * QLD + b * 8 + j;
+            double *cp = Cs + (a * 8 + i0) * QLD + b * 8 + j;
+            double y0 = yp[0], y1 = yp[4 * QLD], c0 = cp[0], c1 = cp[4 * QLD];
+            // tabL[row][7 + is] = L(row, is) for 0 <= is < row else 0; at step s, is = s - j
+            const double *tl0 = tabL + (a * 8 + i0) * TAB_LD + 7 - j;
+            const double *tl1 = tl0 + 4 * TAB_LD;
+            // tabU[col][7 + js] = U(js, col) for 0 <= js < col else 0; at step s, js = s - i
+            const double *tu0 = tabU + (b * 8 + j) * TAB_LD + 7 - i0;
+            const double *tu1 = tu0 - 4;
+            double *exw = xch + warp * 32;
+            int z0 = 0, z1 = 0;
+            const int t0 = i0 + j, t1 = t0 + 4;
 #pragma unroll
             for (int s = 0; s < 15; ++s) {
-                const int k = s & 7;
-                const int j = s - i;
-                const bool act = live && j >= 0 && j < 8;
-                double e = 0.0;
-                if (act) {
-                    const double yv = y[k];
-                    double zv = rint(yv);
-                    if (!(fabs(yv) < 2147483648.0)) {
-                        int gr = row0 + a * 8 + i, gc = col0 + b * 8 + j;
-                        if (gr < p.m && gc < p.n)
-                            report(p.info, isfinite(yv) ? GPTQ2D_ERR_INT_OVERFLOW : GPTQ2D_ERR_NONFINITE, gr, gc, 0);
-                        zv = 0.0;
+                double *ex = exw + (s & 1) * 16;                        // [0..7] e by column, [8..15] C by row
+                const bool r0 = (t0 == s), r1 = (t1 == s);
+                if (r0 || r1) {
+                    const double yv = r0 ? y0 : y1;
+                    const double zv = rint(yv);
+                    const double e = zv - yv;                           // line 5: E = Z - Y
+                    const double cf = (r0 ? c0 : c1) + e;               // fold, L_ii = 1
+                    ex[j] = e;
+                    ex[8 + i0 + (r0 ? 0 : 4)] = cf;
+                    if (r0) { y0 = e; c0 = cf; z0 = (int)zv; }
+                    else { y1 = e; c1 = cf; z1 = (int)zv; }
+                    if (!(fabs(yv) < 2147483648.0)) {                   // not representable: remember the first
+                        const unsigned long long gr = row0 + a * 8 + i0 + (r0 ? 0 : 4), gc = col0 + b * 8 + j;
+                        const unsigned long long key = ((gr + gc) << 42) | ((isfinite(yv) ? 1ull : 0ull) << 41) |
+                                                       (gr << 20) | gc;
+                        if (gr < (unsigned long long)p.m && gc < (unsigned long long)p.n && key < badkey) badkey = key;
                     }
-                    e = zv - yv;                                           // line 5: E = Z - Y
-                    z[k] = (int)zv;
-                    y[k] = e;                                              // the slot now carries E
-                    c[k] += e;                                             // fold, L_ii = 1
-                    const double cf = c[k];
-                    const double *urow = Us + (b * 8 + j) * QLD + b * 8 + j;
-#pragma unroll
-                    for (int d = 1; d < 8; ++d)                            // push right inside the leaf
-                        if (j + d < 8) y[(k + d) & 7] = fma(cf, urow[d], y[(k + d) & 7]);
                 }
-#pragma unroll
-                for (int d = 1; d < 8; ++d) {                              // fold + push down inside the leaf
-                    const double ed = __shfl_up_sync(0xffffffffu, e, d, 8);
-                    const double mm = lrow[d] * ed;
-                    c[(k + d) & 7] += mm;
-                    y[(k + d) & 7] += mm;
-                }
+                __syncwarp();
+                if (s < 8 && warp + s > lw) block_feedback(Ys, Cs, Ls, Us, lw - 1, warp, s, g, t);   // far feedback
+                const double ed = ex[j], cr0 = ex[8 + i0], cr1 = ex[12 + i0];
+                const double l0 = tl0[s], l1 = tl1[s], u0 = tu0[s], u1 = tu1[s];
+                y0 = fma(l0, ed, y0); c0 = fma(l0, ed, c0); y0 = fma(cr0, u0, y0);   // fold, push down, push right
+                y1 = fma(l1, ed, y1); c1 = fma(l1, ed, c1); y1 = fma(cr1, u1, y1);
             }
-            if (live) {
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    int j = (k - i) & 7;
-                    Ys[(a * 8 + i) * QLD + b * 8 + j] = y[k];
-                    Cs[(a * 8 + i) * QLD + b * 8 + j] = c[k];
-                    Zs[(a * 8 + i) * Q + b * 8 + j] = z[k];
-                    int gr = row0 + a * 8 + i, gc = col0 + b * 8 + j;
-                    if (gr < p.m && gc < p.n) max_abs_e = fmax(max_abs_e, fabs(y[k]));
-                }
+            yp[0] = y0; yp[4 * QLD] = y1; cp[0] = c0; cp[4 * QLD] = c1;
+            Zs[(a * 8 + i0) * Q + b * 8 + j] = z0;
+            Zs[(a * 8 + i0 + 4) * Q + b * 8 + j] = z1;
+            if (col0 + b * 8 + j < p.n) {
+                if (row0 + a * 8 + i0 < p.m) max_abs_e = fmax(max_abs_e, fabs(y0));
+                if (row0 + a * 8 + i0 + 4 < p.m) max_abs_e = fmax(max_abs_e, fabs(y1));
             }
+        } else if (lw > 0) {
+            // no leaf for this warp in this leaf-wave: only the far feedback of the previous one
+#pragma unroll
+            for (int qb = 0; qb < 8; ++qb)
+                if (warp + qb > lw) block_feedback(Ys, Cs, Ls, Us, lw - 1, warp, qb, g, t);
         }
         __syncthreads();
         if (lw == 14) break;
-        // ---------------- phase B: feedback of this leaf-wave to the blocks still to come
+        // ---------------- part 2: feedback of this leaf-wave to the next one
         {
-            const int pb = warp;                                   // warp owns block row pb
-            const int bsrc = lw - pb;                              // leaf (pb, bsrc) pushes right
-            const bool has_right = bsrc >= 0 && bsrc <= 7;
-            double ar0 = 0.0, ar1 = 0.0;
-            if (has_right) {
-                ar0 = Cs[(pb * 8 + g) * QLD + bsrc * 8 + t];
-                ar1 = Cs[(pb * 8 + g) * QLD + bsrc * 8 + 4 + t];
-            }
-            for (int qb = max(0, lw - pb + 1); qb < 8; ++qb) {
-                double *yp = Ys + (pb * 8 + g) * QLD + qb * 8 + t * 2;
-                double2 yv = *reinterpret_cast<double2 *>(yp);
-                const int asrc = lw - qb;                          // leaf (asrc, qb) pushes down
-                if (asrc >= 0 && asrc <= 7) {
-                    double p0 = 0.0, p1 = 0.0;
-#pragma unroll
-                    for (int kk = 0; kk < 8; kk += 4) {
-                        double af = Ls[(pb * 8 + g) * QLD + asrc * 8 + kk + t];
-                        double bf = Ys[(asrc * 8 + kk + t) * QLD + qb * 8 + g];
-                        dmma_m8n8k4(p0, p1, af, bf);
-                    }
-                    double *cp = Cs + (pb * 8 + g) * QLD + qb * 8 + t * 2;
-                    double2 cv = *reinterpret_cast<double2 *>(cp);
-                    cv.x += p0;
-                    cv.y += p1;
-                    *reinterpret_cast<double2 *>(cp) = cv;
-                    yv.x += p0;
-                    yv.y += p1;
-                }
-                if (has_right) {
-                    double b0 = Us[(bsrc * 8 + t) * QLD + qb * 8 + g];
-                    double b1 = Us[(bsrc * 8 + 4 + t) * QLD + qb * 8 + g];
-                    dmma_m8n8k4(yv.x, yv.y, ar0, b0);
-                    dmma_m8n8k4(yv.x, yv.y, ar1, b1);
-                }
-                *reinterpret_cast<double2 *>(yp) = yv;
-            }
+            const int qb = lw + 1 - warp;
+            if (qb >= 0 && qb < 8) block_feedback(Ys, Cs, Ls, Us, lw, warp, qb, g, t);
         }
+    }
+    // status: the earliest (in sweep order) unrepresentable value of the quadrant, if any
+    if (badkey != ~0ull) atomicMin(&s_badkey, badkey);
+    __syncthreads();
+    if (tid == 0 && s_badkey != ~0ull) {
+        const unsigned long long k = s_badkey;
+        report(p.info, ((k >> 41) & 1ull) ? GPTQ2D_ERR_INT_OVERFLOW : GPTQ2D_ERR_NONFINITE,
+               (int)((k >> 20) & 0x1fffffull), (int)(k & 0xfffffull), 0);
     }
 }
 
@@ -288,7 +319,8 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
 // E and C = L E on exit.
 __device__ __forceinline__ void sweep_tile(int I, int J, double *smem, const TiledKernelParams &p, double &max_abs_e) {
     double *Ys = smem, *Cs = smem + QMAT, *Ls = smem + 2 * QMAT, *Us = smem + 3 * QMAT, *Xop = smem + 4 * QMAT;
-    int *Zs = reinterpret_cast<int *>(smem + 5 * QMAT);
+    double *tabL = smem + 5 * QMAT, *tabU = tabL + Q * TAB_LD;
+    int *Zs = reinterpret_cast<int *>(tabU + Q * TAB_LD);
     double *eT = p.Ebuf + (long)I * T * p.np + (long)J * T;
     double *cT = p.Cbuf + (long)I * T * p.np + (long)J * T;
     const int tid = threadIdx.x;
@@ -299,20 +331,29 @@ __device__ __forceinline__ void sweep_tile(int I, int J, double *smem, const Til
         double *eQ = eT + (long)qi * Q * p.np + qj * Q;
         double *cQ = cT + (long)qi * Q * p.np + qj * Q;
         __syncthreads();
-        load_factor_block(Ls, p.L, p.ldl, p.m, row0, row0, 1);
-        load_factor_block(Us, p.U, p.ldu, p.n, col0, col0, 2);
-        load_quadrant_cg(Cs, cQ, p.np);
-        load_quadrant_cg(Ys, eQ, p.np);
+        load_factor_block_async(Ls, p.L, p.ldl, p.m, row0, row0, 1);
+        load_factor_block_async(Us, p.U, p.ldu, p.n, col0, col0, 2);
+        load_quadrant_async(Cs, cQ, p.np);
+        load_quadrant_async(Ys, eQ, p.np);
+        // the operand of the first cross term that follows this quadrant
+        if (q == 0 || q == 2) load_factor_block_async(Xop, p.U, p.ldu, p.n, J * T, J * T + Q, 0);
+        if (q == 1) load_factor_block_async(Xop, p.L, p.ldl, p.m, I * T + Q, I * T, 0);
+        cp_async_commit();
+        cp_async_wait<0>();
         __syncthreads();
-        for (int c = tid; c < Q * Q; c += blockDim.x) {       // Y = X + Rt + Cd
+#pragma unroll
+        for (int it = 0; it < 16; ++it) {                     // Y = X + Rt + Cd
+            int c = tid + it * TILED_THREADS;
             int r = c >> 6, cc = c & 63;
             Ys[r * QLD + cc] += Cs[r * QLD + cc];
         }
-        quadrant_sweep(Ys, Cs, Ls, Us, Zs, row0, col0, p, max_abs_e);
+        quadrant_sweep(Ys, Cs, Ls, Us, Zs, tabL, tabU, row0, col0, p, max_abs_e);
         // results of the quadrant
         store_quadrant(eQ, p.np, Ys);
         store_quadrant(cQ, p.np, Cs);
-        for (int c = tid; c < Q * Q; c += blockDim.x) {
+#pragma unroll
+        for (int it = 0; it < 16; ++it) {
+            int c = tid + it * TILED_THREADS;
             int r = c >> 6, cc = c & 63;
             int gr = row0 + r, gc = col0 + cc;
             if (gr < p.m && gc < p.n) {
@@ -321,18 +362,17 @@ __device__ __forceinline__ void sweep_tile(int I, int J, double *smem, const Til
             }
         }
         // cross terms to the quadrants of this tile that follow
-        if (q == 0 || q == 2) {   // C of the left quadrant pushes right through U[left cols, right cols]
-            load_factor_block(Xop, p.U, p.ldu, p.n, J * T, J * T + Q, 0);
-            __syncthreads();
+        if (q == 0 || q == 2)     // C of the left quadrant pushes right through U[left cols, right cols]
             cross_gemm(eT + (long)qi * Q * p.np + Q, p.np, Cs, Xop);
+        if (q == 0) {
+            __syncthreads();
+            load_factor_block_async(Xop, p.L, p.ldl, p.m, I * T + Q, I * T, 0);
+            cp_async_commit();
+            cp_async_wait<0>();
             __syncthreads();
         }
-        if (q == 0 || q == 1) {   // E of the upper quadrant folds down through L[lower rows, upper rows]
-            load_factor_block(Xop, p.L, p.ldl, p.m, I * T + Q, I * T, 0);
-            __syncthreads();
+        if (q == 0 || q == 1)     // E of the upper quadrant folds down through L[lower rows, upper rows]
             cross_gemm(cT + (long)Q * p.np + qj * Q, p.np, Xop, Ys);
-            __syncthreads();
-        }
     }
 }
 
