@@ -9,14 +9,20 @@
 // sweep.  Cd and Rt are dense contractions and carry all but a T/(m+n) share of the flops,
 // so they run on the fp64 tensor path (dmma_gemm.cuh); tiles with equal I + J are independent.
 //
-// Scheduling.  Every tile has two bulk tasks (Cd and Rt).  Tasks are listed wave by wave
-// (I + J ascending) and claimed in that order from one atomic counter by persistent CTAs
-// (one per SM, cooperatively launched so that all are resident).  A bulk task consumes its
-// source tiles in the order they become available, waiting (bounded) on per-tile ready
-// flags; whichever CTA finishes the second bulk task of a tile runs that tile's in-tile
-// sweep right away and then raises the tile's flag.  A task only ever waits on tiles of
-// earlier waves, whose tasks were claimed earlier, so the earliest unfinished task can
-// always progress.
+// Scheduling.  Every tile has two bulk tasks (Cd and Rt), each split into a FAR part (all
+// source tiles except the adjacent one) and a NEAR step (the adjacent tile, one K = 128
+// chunk).  Far parts are listed wave by wave (I + J ascending) and claimed in that order
+// from one atomic counter by persistent CTAs (one per SM, cooperatively launched so that all
+// are resident); a far part waits (bounded) only on tiles two or more waves back, parks its
+// partial sum in the tile's own workspace region and announces it.  Everything on the
+// critical path runs as an inline continuation with no waiting: the near step runs on
+// whichever CTA completes its second prerequisite (far part parked / adjacent tile swept),
+// the in-tile sweep on whichever CTA completes the tile's second near step; near steps that
+// a swept tile releases go to a global ready ring which every CTA serves first -- at the
+// top of its loop, while it waits, and every few chunks of a far part (it then parks its
+// partial sum and un-parks it afterwards).  A far part only ever waits on tiles of earlier
+// waves, whose far parts were claimed earlier and whose continuations never wait, so the
+// earliest unfinished work can always progress.
 //
 // In-tile sweep.  The tile is processed as four 64 x 64 quadrants (the same restatement one
 // level down, cross terms as 64^3 DMMA products).  Inside a quadrant the anti-diagonal
@@ -47,9 +53,12 @@ struct TiledKernelParams {
     int *Z; long ldz;
     double *Euser; long lde;
     double *Ebuf, *Cbuf;
-    unsigned *counter, *abort;
+    unsigned *counter, *abort, *q_head, *q_tail, *tiles_done;
+    unsigned *q_slots;           // [QCAP] ready continuation tasks
     unsigned *flagS;             // [ntm*ntn] tile swept
-    unsigned *bulk_done;         // [ntm*ntn] number of finished bulk tasks
+    unsigned *bulk_done;         // [ntm*ntn] number of finished bulk contractions (2 -> sweep)
+    unsigned *quad_done;         // [ntm*ntn] finished ones of quadrants 1 and 2 (2 -> quadrant 3)
+    unsigned *near_dep;          // [2][ntm*ntn] arrivals for the near step: far part parked, source tile swept
     double *max_abs_e;
     int *info;
     int l_al16, u_al16;
@@ -58,44 +67,6 @@ struct TiledKernelParams {
 constexpr size_t SWEEP_SMEM = (size_t)(5 * QMAT + 2 * Q * TAB_LD) * sizeof(double) + (size_t)Q * Q * sizeof(int);
 constexpr size_t BULK_SMEM = (size_t)BULK_NSTAGE * SlabLayout<true, false>::STAGE_DOUBLES * sizeof(double);
 constexpr size_t TILED_SMEM = SWEEP_SMEM > BULK_SMEM ? SWEEP_SMEM : BULK_SMEM;
-
-// ---------------------------------------------------------------------------------------------
-// bounded wait until flags[first] is set; returns the index of the first flag in
-// [first, count) that is not set yet (> first), or -1 on abort / timeout.
-__device__ __forceinline__ int wait_ready_prefix(const unsigned *flags, long stride, int first, int count,
-                                                 const TiledKernelParams &p, int where) {
-    __shared__ int s_first;
-    const int tid = threadIdx.x;
-    unsigned long long spins = 0;
-    for (;;) {
-        __syncthreads();
-        if (tid == 0) s_first = count;
-        __syncthreads();
-        for (int idx = first + tid; idx < count; idx += blockDim.x)
-            if (ld_acquire_u32(flags + (long)idx * stride) == 0u) atomicMin(&s_first, idx);
-        __syncthreads();
-        int f = s_first;
-        if (f > first) return f;
-        // nothing ready: thread 0 spins on the first flag
-        __shared__ int s_ok;
-        if (tid == 0) {
-            int ok = 1;
-            while (ld_acquire_u32(flags + (long)first * stride) == 0u) {
-                if (ld_relaxed_u32(p.abort) != 0u) { ok = 0; break; }
-                if (++spins > SPIN_LIMIT) {
-                    report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, where, first, (int)blockIdx.x);
-                    atomicExch(p.abort, 1u);
-                    ok = 0;
-                    break;
-                }
-                __nanosleep(100);
-            }
-            s_ok = ok;
-        }
-        __syncthreads();
-        if (!s_ok) return -1;
-    }
-}
 
 // ---------------------------------------------------------------------------------------------
 // quadrant <-> shared memory.  The *_async loaders only issue cp.async copies; the caller
@@ -315,65 +286,69 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
 }
 
 // ---------------------------------------------------------------------------------------------
-// in-tile sweep of tile (I, J): Ebuf tile holds X + Rt, Cbuf tile holds Cd on entry;
-// E and C = L E on exit.
-__device__ __forceinline__ void sweep_tile(int I, int J, double *smem, const TiledKernelParams &p, double &max_abs_e) {
+// One 64 x 64 quadrant q (0: top-left, 1: top-right, 2: bottom-left, 3: bottom-right) of the
+// in-tile sweep of tile (I, J).  On entry the tile's Ebuf region holds X + Rt and its Cbuf
+// region Cd, both already updated by the cross terms of the quadrants this one depends on;
+// on exit the quadrant's regions hold E and C = L E, Z (and the caller's E) are written, and
+// the cross terms this quadrant owes to later quadrants of the tile have been added to their
+// regions: q0 -> q1 (through U) and q2 (through L); q1 -> q3 (through L); q2 -> q3 (through U).
+// Quadrants 1 and 2 are independent of each other and may run on different CTAs.
+__device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem, const TiledKernelParams &p,
+                                               double &max_abs_e) {
     double *Ys = smem, *Cs = smem + QMAT, *Ls = smem + 2 * QMAT, *Us = smem + 3 * QMAT, *Xop = smem + 4 * QMAT;
     double *tabL = smem + 5 * QMAT, *tabU = tabL + Q * TAB_LD;
     int *Zs = reinterpret_cast<int *>(tabU + Q * TAB_LD);
     double *eT = p.Ebuf + (long)I * T * p.np + (long)J * T;
     double *cT = p.Cbuf + (long)I * T * p.np + (long)J * T;
     const int tid = threadIdx.x;
-#pragma unroll 1
-    for (int q = 0; q < 4; ++q) {
-        const int qi = q >> 1, qj = q & 1;
-        const int row0 = I * T + qi * Q, col0 = J * T + qj * Q;
-        double *eQ = eT + (long)qi * Q * p.np + qj * Q;
-        double *cQ = cT + (long)qi * Q * p.np + qj * Q;
+    const int qi = q >> 1, qj = q & 1;
+    const int row0 = I * T + qi * Q, col0 = J * T + qj * Q;
+    double *eQ = eT + (long)qi * Q * p.np + qj * Q;
+    double *cQ = cT + (long)qi * Q * p.np + qj * Q;
+    __syncthreads();
+    load_factor_block_async(Ls, p.L, p.ldl, p.m, row0, row0, 1);
+    load_factor_block_async(Us, p.U, p.ldu, p.n, col0, col0, 2);
+    load_quadrant_async(Cs, cQ, p.np);
+    load_quadrant_async(Ys, eQ, p.np);
+    // the operand of the first cross term that follows this quadrant
+    if (q == 0 || q == 2) load_factor_block_async(Xop, p.U, p.ldu, p.n, J * T, J * T + Q, 0);
+    if (q == 1) load_factor_block_async(Xop, p.L, p.ldl, p.m, I * T + Q, I * T, 0);
+    cp_async_commit();
+    cp_async_wait<0>();
+    __syncthreads();
+#pragma unroll
+    for (int it = 0; it < 16; ++it) {                     // Y = X + Rt + Cd
+        int c = tid + it * TILED_THREADS;
+        int r = c >> 6, cc = c & 63;
+        Ys[r * QLD + cc] += Cs[r * QLD + cc];
+    }
+    quadrant_sweep(Ys, Cs, Ls, Us, Zs, tabL, tabU, row0, col0, p, max_abs_e);
+    // results of the quadrant
+    store_quadrant(eQ, p.np, Ys);
+    store_quadrant(cQ, p.np, Cs);
+#pragma unroll
+    for (int it = 0; it < 16; ++it) {
+        int c = tid + it * TILED_THREADS;
+        int r = c >> 6, cc = c & 63;
+        int gr = row0 + r, gc = col0 + cc;
+        if (gr < p.m && gc < p.n) {
+            p.Z[(long)gr * p.ldz + gc] = Zs[r * Q + cc];
+            if (p.Euser) p.Euser[(long)gr * p.lde + gc] = Ys[r * QLD + cc];
+        }
+    }
+    // cross terms to the quadrants of this tile that follow
+    if (q == 0 || q == 2)     // C of the left quadrant pushes right through U[left cols, right cols]
+        cross_gemm(eT + (long)qi * Q * p.np + Q, p.np, Cs, Xop);
+    if (q == 0) {
         __syncthreads();
-        load_factor_block_async(Ls, p.L, p.ldl, p.m, row0, row0, 1);
-        load_factor_block_async(Us, p.U, p.ldu, p.n, col0, col0, 2);
-        load_quadrant_async(Cs, cQ, p.np);
-        load_quadrant_async(Ys, eQ, p.np);
-        // the operand of the first cross term that follows this quadrant
-        if (q == 0 || q == 2) load_factor_block_async(Xop, p.U, p.ldu, p.n, J * T, J * T + Q, 0);
-        if (q == 1) load_factor_block_async(Xop, p.L, p.ldl, p.m, I * T + Q, I * T, 0);
+        load_factor_block_async(Xop, p.L, p.ldl, p.m, I * T + Q, I * T, 0);
         cp_async_commit();
         cp_async_wait<0>();
         __syncthreads();
-#pragma unroll
-        for (int it = 0; it < 16; ++it) {                     // Y = X + Rt + Cd
-            int c = tid + it * TILED_THREADS;
-            int r = c >> 6, cc = c & 63;
-            Ys[r * QLD + cc] += Cs[r * QLD + cc];
-        }
-        quadrant_sweep(Ys, Cs, Ls, Us, Zs, tabL, tabU, row0, col0, p, max_abs_e);
-        // results of the quadrant
-        store_quadrant(eQ, p.np, Ys);
-        store_quadrant(cQ, p.np, Cs);
-#pragma unroll
-        for (int it = 0; it < 16; ++it) {
-            int c = tid + it * TILED_THREADS;
-            int r = c >> 6, cc = c & 63;
-            int gr = row0 + r, gc = col0 + cc;
-            if (gr < p.m && gc < p.n) {
-                p.Z[(long)gr * p.ldz + gc] = Zs[r * Q + cc];
-                if (p.Euser) p.Euser[(long)gr * p.lde + gc] = Ys[r * QLD + cc];
-            }
-        }
-        // cross terms to the quadrants of this tile that follow
-        if (q == 0 || q == 2)     // C of the left quadrant pushes right through U[left cols, right cols]
-            cross_gemm(eT + (long)qi * Q * p.np + Q, p.np, Cs, Xop);
-        if (q == 0) {
-            __syncthreads();
-            load_factor_block_async(Xop, p.L, p.ldl, p.m, I * T + Q, I * T, 0);
-            cp_async_commit();
-            cp_async_wait<0>();
-            __syncthreads();
-        }
-        if (q == 0 || q == 1)     // E of the upper quadrant folds down through L[lower rows, upper rows]
-            cross_gemm(cT + (long)Q * p.np + qj * Q, p.np, Xop, Ys);
     }
+    if (q == 0 || q == 1)     // E of the upper quadrant folds down through L[lower rows, upper rows]
+        cross_gemm(cT + (long)Q * p.np + qj * Q, p.np, Xop, Ys);
+    __syncthreads();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -393,96 +368,300 @@ __device__ __forceinline__ void decode_task(int task, int ntm, int ntn, int &typ
     I = J = 0;
 }
 
+// accumulator tile <-> its 128 x 128 region of a padded workspace buffer
+__device__ __forceinline__ void store_acc(const Acc &acc, double *dstT, long np, int wm, int wn, int g, int t) {
+#pragma unroll
+    for (int a = 0; a < 8; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            double2 v;
+            v.x = acc.v[a][b][0];
+            v.y = acc.v[a][b][1];
+            *reinterpret_cast<double2 *>(dstT + (long)(wm * 64 + a * 8 + g) * np + wn * 32 + b * 8 + t * 2) = v;
+        }
+}
+__device__ __forceinline__ void load_acc(Acc &acc, const double *srcT, long np, int wm, int wn, int g, int t) {
+#pragma unroll
+    for (int a = 0; a < 8; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            double2 v = __ldcg(reinterpret_cast<const double2 *>(srcT + (long)(wm * 64 + a * 8 + g) * np + wn * 32 +
+                                                                 b * 8 + t * 2));
+            acc.v[a][b][0] = v.x;
+            acc.v[a][b][1] = v.y;
+        }
+}
+
+constexpr unsigned QCAP = 4096;   // global ring of ready continuation tasks (power of two)
+constexpr int FAR_RUN_CHUNKS = 8; // a far part looks at the ready queue every this many K = 128 chunks
+
+// multi-producer / multi-consumer ring in global memory; slot value 0 = empty.
+__device__ __forceinline__ void ready_push(const TiledKernelParams &p, unsigned entry) {
+    unsigned t = atomicAdd(p.q_tail, 1u);
+    st_release_u32(p.q_slots + (t & (QCAP - 1)), entry | 0x80000000u);
+}
+// thread 0 only.  Returns 0 if the queue is empty (or on abort), else the entry (bit 31 set).
+__device__ __forceinline__ unsigned ready_pop(const TiledKernelParams &p) {
+    for (;;) {
+        unsigned h = ld_relaxed_u32(p.q_head), t = ld_relaxed_u32(p.q_tail);
+        if ((int)(t - h) <= 0) return 0u;
+        if (atomicCAS(p.q_head, h, h + 1u) != h) continue;
+        unsigned *slot = p.q_slots + (h & (QCAP - 1));
+        unsigned long long spins = 0;
+        unsigned e;
+        while ((e = ld_acquire_u32(slot)) == 0u) {          // producer has the ticket but has not written yet
+            if (++spins > SPIN_LIMIT || ld_relaxed_u32(p.abort) != 0u) {
+                report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -3, (int)h, (int)blockIdx.x);
+                atomicExch(p.abort, 1u);
+                return 0u;
+            }
+        }
+        *slot = 0u;
+        return e;
+    }
+}
+__device__ __forceinline__ bool ready_nonempty(const TiledKernelParams &p) {
+    return (int)(ld_relaxed_u32(p.q_tail) - ld_relaxed_u32(p.q_head)) > 0;
+}
+
 __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKernelParams p) {
     extern __shared__ __align__(16) double smem[];
     __shared__ int s_task[4];
+    __shared__ int s_flag;
     __shared__ double s_red[TILED_THREADS / 32];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int wm = warp >> 2, wn = warp & 3, g = lane >> 2, t = lane & 3;
+    const int ntiles = p.ntm * p.ntn;
     double max_abs_e = 0.0;
 
+    // far-part context of this CTA (uniform across the CTA)
+    bool f_valid = false;
+    int f_type = 0, f_I = 0, f_J = 0, f_pos = 0, f_nfar = 0, f_task = 0;
+    // continuation handed over with the accumulator still in registers
+    bool have = false;
+    int type = 0, I = 0, J = 0;
+    unsigned long long idle_spins = 0;
+    Acc acc;
+    acc.zero();
+
     for (;;) {
-        __syncthreads();
-        if (tid == 0) {
-            int task = (int)atomicAdd(p.counter, 1u);
-            int type = 0, I = 0, J = 0;
-            if (task < p.ntasks) decode_task(task, p.ntm, p.ntn, type, I, J);
-            if (ld_relaxed_u32(p.abort) != 0u) task = p.ntasks;
-            s_task[0] = task; s_task[1] = type; s_task[2] = I; s_task[3] = J;
-        }
-        __syncthreads();
-        const int task = s_task[0], type = s_task[1], I = s_task[2], J = s_task[3];
-        if (task >= p.ntasks) break;
-
-        // ---------------- bulk contraction: type 0 = Cd (sources above), 1 = Rt (sources left)
-        Acc acc;
-        acc.zero();
-        const int nsrc = type == 0 ? I : J;
-        const unsigned *flags = type == 0 ? p.flagS + J : p.flagS + (long)I * p.ntn;
-        const long fstride = type == 0 ? p.ntn : 1;
-        Operand A, B;
-        if (type == 0) {
-            A.ptr = p.L + (long)I * T * p.ldl; A.ld = p.ldl; A.mn_valid = min(T, p.m - I * T); A.aligned16 = p.l_al16;
-            B.ptr = p.Ebuf + (long)J * T; B.ld = p.np; B.mn_valid = T; B.aligned16 = true;
-        } else {
-            A.ptr = p.Cbuf + (long)I * T * p.np; A.ld = p.np; A.mn_valid = T; A.aligned16 = true;
-            B.ptr = p.U + (long)J * T; B.ld = p.ldu; B.mn_valid = min(T, p.n - J * T); B.aligned16 = p.u_al16;
-        }
-        bool dead = false;
-        for (int pos = 0; pos < nsrc;) {
-            int upto = wait_ready_prefix(flags, fstride, pos, nsrc, p, task);
-            if (upto < 0) { dead = true; break; }
-            Operand a = A, b = B;
-            a.ptr = A.ptr + (long)pos * T;                 // k offset along the contiguous index
-            b.ptr = B.ptr + (long)pos * T * B.ld;          // k offset along rows
-            gemm_mainloop<true, false, BULK_NSTAGE>(acc, smem, a, b, (upto - pos) * T);
-            pos = upto;
-        }
-        if (dead) break;
-
-        // ---------------- bulk epilogue
-        {
-            double *dstT = (type == 0 ? p.Cbuf : p.Ebuf) + (long)I * T * p.np + (long)J * T;
-#pragma unroll
-            for (int a = 0; a < 8; ++a) {
-                const int r = wm * 64 + a * 8 + g;
-                const int gr = I * T + r;
-#pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    const int c = wn * 32 + b * 8 + t * 2;
-                    const int gc = J * T + c;
-                    double2 v;
-                    v.x = acc.v[a][b][0];
-                    v.y = acc.v[a][b][1];
-                    if (type == 1) {                       // Y0 = X + Rt, zero outside the matrix
-                        double x0 = 0.0, x1 = 0.0;
-                        if (gr < p.m) {
-                            if (gc < p.n) x0 = __ldg(p.X + (long)gr * p.ldx + gc);
-                            if (gc + 1 < p.n) x1 = __ldg(p.X + (long)gr * p.ldx + gc + 1);
-                        }
-                        v.x += x0;
-                        v.y += x1;
+        // ================= A: continuations (near step, quadrant sweeps, releases).  Never waits.
+        // Ready-ring entries: kind 0 / 1 = near step of the Cd / Rt contraction of tile (I, J);
+        // kind 2 = bottom-left quadrant of the in-tile sweep of tile (I, J).
+        for (;;) {
+            int quad = -1;                 // >= 0: next quadrant of tile (I, J) to sweep on this CTA
+            if (!have) {
+                __syncthreads();
+                if (tid == 0) {
+                    unsigned e = ready_pop(p);
+                    s_flag = e != 0u;
+                    s_task[1] = (int)((e >> 29) & 3u); s_task[2] = (int)((e >> 15) & 0x3fffu); s_task[3] = (int)(e & 0x7fffu);
+                }
+                __syncthreads();
+                if (!s_flag) break;
+                type = s_task[1]; I = s_task[2]; J = s_task[3];
+                if (type == 2) {
+                    quad = 2;
+                } else if ((type == 0 ? I : J) > 1) {
+                    load_acc(acc, (type == 0 ? p.Cbuf : p.Ebuf) + (long)I * T * p.np + (long)J * T, p.np, wm, wn, g, t);
+                } else {
+                    acc.zero();
+                }
+            }
+            have = false;
+            if (quad < 0) {
+                // near step: the adjacent source tile (already swept, by construction)
+                const int src = (type == 0 ? I : J) - 1;
+                if (src >= 0) {
+                    Operand a, b;
+                    if (type == 0) {
+                        a.ptr = p.L + (long)I * T * p.ldl + (long)src * T; a.ld = p.ldl; a.mn_valid = min(T, p.m - I * T); a.aligned16 = p.l_al16;
+                        b.ptr = p.Ebuf + (long)src * T * p.np + (long)J * T; b.ld = p.np; b.mn_valid = T; b.aligned16 = true;
+                    } else {
+                        a.ptr = p.Cbuf + (long)I * T * p.np + (long)src * T; a.ld = p.np; a.mn_valid = T; a.aligned16 = true;
+                        b.ptr = p.U + (long)src * T * p.ldu + (long)J * T; b.ld = p.ldu; b.mn_valid = min(T, p.n - J * T); b.aligned16 = p.u_al16;
                     }
-                    *reinterpret_cast<double2 *>(dstT + (long)r * p.np + c) = v;
+                    gemm_mainloop<true, false, BULK_NSTAGE>(acc, smem, a, b, T);
+                }
+                // bulk epilogue: Cd, or Y0 = X + Rt (zero outside the matrix)
+                {
+                    double *dstT = (type == 0 ? p.Cbuf : p.Ebuf) + (long)I * T * p.np + (long)J * T;
+#pragma unroll
+                    for (int a = 0; a < 8; ++a) {
+                        const int r = wm * 64 + a * 8 + g;
+                        const int gr = I * T + r;
+#pragma unroll
+                        for (int b = 0; b < 4; ++b) {
+                            const int c = wn * 32 + b * 8 + t * 2;
+                            const int gc = J * T + c;
+                            double2 v;
+                            v.x = acc.v[a][b][0];
+                            v.y = acc.v[a][b][1];
+                            if (type == 1) {
+                                double x0 = 0.0, x1 = 0.0;
+                                if (gr < p.m) {
+                                    if (gc < p.n) x0 = __ldg(p.X + (long)gr * p.ldx + gc);
+                                    if (gc + 1 < p.n) x1 = __ldg(p.X + (long)gr * p.ldx + gc + 1);
+                                }
+                                v.x += x0;
+                                v.y += x1;
+                            }
+                            *reinterpret_cast<double2 *>(dstT + (long)r * p.np + c) = v;
+                        }
+                    }
+                }
+                __syncthreads();
+                if (tid == 0) {
+                    __threadfence();
+                    unsigned old = atomicAdd(p.bulk_done + (long)I * p.ntn + J, 1u);
+                    __threadfence();
+                    s_flag = (old == 1u) ? 1 : 0;
+                }
+                __syncthreads();
+                if (!s_flag) continue;
+                quad = 0;                  // both contractions of tile (I, J) are complete: sweep it
+            }
+            // in-tile sweep, quadrant by quadrant: 0, then 1 here while 2 is offered to the ready ring
+            // (an idle CTA takes it, otherwise this CTA pops it itself), then 3 on whichever CTA
+            // finishes the second of quadrants 1 and 2.
+            while (quad >= 0) {
+                sweep_quadrant(I, J, quad, smem, p, max_abs_e);
+                if (quad == 0) {
+                    if (tid == 0) {
+                        __threadfence();
+                        ready_push(p, (2u << 29) | ((unsigned)I << 15) | (unsigned)J);
+                    }
+                    quad = 1;
+                } else if (quad == 1 || quad == 2) {
+                    if (tid == 0) {
+                        __threadfence();
+                        unsigned old = atomicAdd(p.quad_done + (long)I * p.ntn + J, 1u);
+                        __threadfence();
+                        s_flag = (old == 1u) ? 1 : 0;
+                    }
+                    __syncthreads();
+                    quad = s_flag ? 3 : -1;
+                } else {
+                    // tile swept: publish it and release the near steps of the tile below and to the right
+                    if (tid == 0) {
+                        __threadfence();
+                        st_release_u32(p.flagS + (long)I * p.ntn + J, 1u);
+                        for (int d = 0; d < 2; ++d) {
+                            const int dI = I + (d == 0 ? 1 : 0), dJ = J + (d == 0 ? 0 : 1);
+                            if (dI >= p.ntm || dJ >= p.ntn) continue;
+                            unsigned old = atomicAdd(p.near_dep + ((long)d * ntiles + (long)dI * p.ntn + dJ), 1u);
+                            if (old == 1u) {      // its far part is parked already: the near step is ready
+                                __threadfence();
+                                ready_push(p, ((unsigned)d << 29) | ((unsigned)dI << 15) | (unsigned)dJ);
+                            }
+                        }
+                        atomicAdd(p.tiles_done, 1u);
+                    }
+                    quad = -1;
                 }
             }
         }
-        __syncthreads();
-        if (tid == 0) {
-            __threadfence();
-            unsigned old = atomicAdd(p.bulk_done + (long)I * p.ntn + J, 1u);
-            __threadfence();
-            s_task[1] = (old == 1u) ? 1 : 0;
-        }
-        __syncthreads();
-        if (s_task[1]) {
-            sweep_tile(I, J, smem, p, max_abs_e);
+        if (ld_relaxed_u32(p.abort) != 0u) break;
+
+        // ================= B: far part of a bulk contraction: every source tile except the adjacent one.
+        if (!f_valid) {
             __syncthreads();
             if (tid == 0) {
-                __threadfence();
-                st_release_u32(p.flagS + (long)I * p.ntn + J, 1u);
+                int task = p.ntasks;
+                if (ld_relaxed_u32(p.counter) < (unsigned)p.ntasks) task = (int)atomicAdd(p.counter, 1u);
+                int ty = 0, fi = 0, fj = 0;
+                if (task < p.ntasks) decode_task(task, p.ntm, p.ntn, ty, fi, fj);
+                s_task[0] = task; s_task[1] = ty; s_task[2] = fi; s_task[3] = fj;
+                s_flag = (ld_relaxed_u32(p.tiles_done) >= (unsigned)ntiles) ? 1 : 0;
+            }
+            __syncthreads();
+            if (s_task[0] >= p.ntasks) {
+                if (s_flag) break;                           // every tile is swept: done
+                if (++idle_spins > SPIN_LIMIT) {             // nothing to claim: wait for continuations
+                    if (tid == 0) {
+                        report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -4, (int)blockIdx.x, 0);
+                        atomicExch(p.abort, 1u);
+                    }
+                    break;
+                }
+                __nanosleep(200);
+                continue;
+            }
+            f_task = s_task[0]; f_type = s_task[1]; f_I = s_task[2]; f_J = s_task[3];
+            f_pos = 0;
+            f_nfar = max(0, (f_type == 0 ? f_I : f_J) - 1);
+            f_valid = true;
+            acc.zero();
+        } else {
+            // coming back from continuations: un-park the partial sum
+            if (f_pos > 0)
+                load_acc(acc, (f_type == 0 ? p.Cbuf : p.Ebuf) + (long)f_I * T * p.np + (long)f_J * T, p.np, wm, wn, g, t);
+            else
+                acc.zero();
+        }
+        bool interrupted = false;
+        {
+            const unsigned *flags = f_type == 0 ? p.flagS + f_J : p.flagS + (long)f_I * p.ntn;
+            const long fstride = f_type == 0 ? p.ntn : 1;
+            Operand A, B;
+            if (f_type == 0) {
+                A.ptr = p.L + (long)f_I * T * p.ldl; A.ld = p.ldl; A.mn_valid = min(T, p.m - f_I * T); A.aligned16 = p.l_al16;
+                B.ptr = p.Ebuf + (long)f_J * T; B.ld = p.np; B.mn_valid = T; B.aligned16 = true;
+            } else {
+                A.ptr = p.Cbuf + (long)f_I * T * p.np; A.ld = p.np; A.mn_valid = T; A.aligned16 = true;
+                B.ptr = p.U + (long)f_J * T; B.ld = p.ldu; B.mn_valid = min(T, p.n - f_J * T); B.aligned16 = p.u_al16;
+            }
+            unsigned long long spins = 0;
+            while (f_pos < f_nfar) {
+                // how many source tiles from f_pos on are swept already; is there ready work to take over
+                __syncthreads();
+                if (tid == 0) { s_task[0] = f_nfar; s_flag = ready_nonempty(p) ? 1 : 0; }
+                __syncthreads();
+                for (int idx = f_pos + tid; idx < f_nfar; idx += blockDim.x)
+                    if (ld_acquire_u32(flags + (long)idx * fstride) == 0u) atomicMin(&s_task[0], idx);
+                __syncthreads();
+                const int upto_ready = s_task[0];
+                const bool work = s_flag != 0;
+                if (upto_ready == f_pos) {                   // next source not swept yet
+                    if (work) { interrupted = true; break; }
+                    if (++spins > SPIN_LIMIT || ld_relaxed_u32(p.abort) != 0u) {
+                        if (tid == 0) {
+                            report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, f_task, f_pos, (int)blockIdx.x);
+                            atomicExch(p.abort, 1u);
+                        }
+                        interrupted = true;
+                        break;
+                    }
+                    __nanosleep(100);
+                    continue;
+                }
+                if (work) { interrupted = true; break; }       // park and serve the critical path first
+                const int upto = min(upto_ready, f_pos + FAR_RUN_CHUNKS);
+                Operand a = A, b = B;
+                a.ptr = A.ptr + (long)f_pos * T;               // k offset along the contiguous index
+                b.ptr = B.ptr + (long)f_pos * T * B.ld;        // k offset along rows
+                gemm_mainloop<true, false, BULK_NSTAGE>(acc, smem, a, b, (upto - f_pos) * T);
+                f_pos = upto;
             }
         }
+        if (ld_relaxed_u32(p.abort) != 0u) break;
+        // park the partial sum in the tile's own output region
+        if (f_pos > 0)
+            store_acc(acc, (f_type == 0 ? p.Cbuf : p.Ebuf) + (long)f_I * T * p.np + (long)f_J * T, p.np, wm, wn, g, t);
+        if (interrupted) continue;                            // back to A, then resume this far part
+        // far part complete: announce it; if the adjacent tile is swept already, go on with the near step
+        __syncthreads();
+        if (tid == 0) {
+            const bool has_src = (f_type == 0 ? f_I : f_J) > 0;
+            __threadfence();
+            unsigned old = atomicAdd(p.near_dep + ((long)f_type * ntiles + (long)f_I * p.ntn + f_J), 1u);
+            __threadfence();
+            s_flag = (old + 1u == (has_src ? 2u : 1u)) ? 1 : 0;
+        }
+        __syncthreads();
+        have = s_flag != 0;
+        type = f_type; I = f_I; J = f_J;
+        f_valid = false;
     }
 
     for (int o = 16; o > 0; o >>= 1) max_abs_e = fmax(max_abs_e, __shfl_xor_sync(0xffffffffu, max_abs_e, o));
@@ -500,7 +679,7 @@ static size_t pad256(size_t x) { return (x + 255) / 256 * 256; }
 
 struct TiledLayout {
     int ntm, ntn;
-    size_t flags_off, done_off, e_off, c_off, total;
+    size_t q_off, flags_off, done_off, quad_off, near_off, e_off, c_off, total;
 };
 static TiledLayout tiled_layout(int m, int n) {
     TiledLayout l;
@@ -508,9 +687,12 @@ static TiledLayout tiled_layout(int m, int n) {
     l.ntn = (n + T - 1) / T;
     size_t tiles = (size_t)l.ntm * l.ntn;
     size_t mat = (size_t)l.ntm * T * (size_t)l.ntn * T * sizeof(double);
-    l.flags_off = 256;
+    l.q_off = 256;
+    l.flags_off = l.q_off + 4096 * sizeof(unsigned);
     l.done_off = l.flags_off + pad256(tiles * sizeof(unsigned));
-    l.e_off = l.done_off + pad256(tiles * sizeof(unsigned));
+    l.quad_off = l.done_off + pad256(tiles * sizeof(unsigned));
+    l.near_off = l.quad_off + pad256(tiles * sizeof(unsigned));
+    l.e_off = l.near_off + pad256(2 * tiles * sizeof(unsigned));
     l.c_off = l.e_off + pad256(mat);
     l.total = l.c_off + pad256(mat);
     return l;
@@ -530,9 +712,15 @@ int launch_round_tiled(const TiledParams &in, void *ws, size_t ws_bytes, cudaStr
     p.Z = in.Z; p.ldz = in.ldz; p.Euser = in.E; p.lde = in.lde;
     p.counter = reinterpret_cast<unsigned *>(w);
     p.abort = reinterpret_cast<unsigned *>(w) + 1;
+    p.q_head = reinterpret_cast<unsigned *>(w) + 2;
+    p.q_tail = reinterpret_cast<unsigned *>(w) + 3;
+    p.tiles_done = reinterpret_cast<unsigned *>(w) + 4;
+    p.q_slots = reinterpret_cast<unsigned *>(w + l.q_off);
     p.max_abs_e = workspace_max_abs_e(ws);
     p.flagS = reinterpret_cast<unsigned *>(w + l.flags_off);
     p.bulk_done = reinterpret_cast<unsigned *>(w + l.done_off);
+    p.near_dep = reinterpret_cast<unsigned *>(w + l.near_off);
+    p.quad_done = reinterpret_cast<unsigned *>(w + l.quad_off);
     p.Ebuf = reinterpret_cast<double *>(w + l.e_off);
     p.Cbuf = reinterpret_cast<double *>(w + l.c_off);
     p.info = in.info;
