@@ -93,6 +93,21 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None}
 
 
+def max_over_ranks(value, dist, device=None):
+    """Whole-job time = the slowest rank's (all-reduce MAX); identity when not distributed."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(m, n, world, ms_per_step):
+    """Replicas only: every rank sweeps its own m x n matrix, so the job rounds world*m*n entries per step."""
+    return world * m * n / (ms_per_step * 1e-3)
+
+
 def workload(index, seed):
     from paper_2607_27042_b200 import workloads as W
     X, A, B = W.make_config(index, seed=seed)
@@ -163,12 +178,9 @@ def run_cuda(args):
     g.check_info(info)
     per_step = [evs[k].elapsed_time(evs[k + 1]) for k in range(args.steps)]
     total_ms = evs[0].elapsed_time(evs[-1])
-    if dist:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dist, "cuda")
     ms_per_step = total_ms / args.steps
-    value = world * m * n / (ms_per_step * 1e-3)
+    value = job_value(m, n, world, ms_per_step)
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies timed)
     e2e = None
@@ -192,12 +204,9 @@ def run_cuda(args):
         a1.record(stream)
         torch.cuda.synchronize()
         e2e_ms = a0.elapsed_time(a1) / nrep
-        if dist:
-            t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks(e2e_ms, dist, "cuda")
         assert torch.equal(hZ, Z.cpu()), "host entry point and device entry point disagree"
-        e2e = {"value": world * m * n / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+        e2e = {"value": job_value(m, n, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": 8 * (m * n + m * m + n * n), "d2h_bytes_per_step": 4 * m * n + 16}
 
     if rank != 0:
