@@ -44,7 +44,8 @@ typedef enum {
                                           info[2] = 0 for A^T A, 1 for B B^T                            */
     GPTQ2D_ERR_NONFINITE = 6,          /* device: NaN/Inf met while rounding; info[1] = row, info[2] = col */
     GPTQ2D_ERR_INT_OVERFLOW = 7,       /* device: |corrected value| >= 2^31; info[1] = row, info[2] = col  */
-    GPTQ2D_ERR_DEVICE_TIMEOUT = 8      /* device: a bounded wait gave up; info[1] = where it waited     */
+    GPTQ2D_ERR_DEVICE_TIMEOUT = 8,     /* device: a bounded wait gave up; info[1] = where it waited     */
+    GPTQ2D_ERR_TOO_LARGE = 9           /* gptq2d_round_static: m or n beyond GPTQ2D_STATIC_MAX_DIM      */
 } gptq2d_status_t;
 
 typedef enum {
@@ -108,6 +109,32 @@ int gptq2d_round_host(int m, int n,
                       int32_t *hZ, double *hE, double *hmin_margin,
                       int precision,
                       void *workspace, size_t workspace_bytes, int *hinfo, void *stream);
+
+/* ---- the sweep without any allocation (the paper has no counterpart: this is a packaging variant
+ * of gptq2d_round, not a different method) ----
+ * For callers that must not allocate device memory -- a step that will be replayed from a CUDA
+ * graph, a framework region that forbids raw cudaMalloc, a latency-critical loop that must stay
+ * away from the allocator -- and therefore cannot hand over a workspace: the scratch of the fp64
+ * tiled sweep lives in a static device array inside the library (GPTQ2D_STATIC_WORKSPACE_BYTES per
+ * GPU that loads the library, held until the process exits).  Same arguments, results and device
+ * status words as gptq2d_round with precision GPTQ2D_FP64, minus the workspace.
+ *   - m, n <= GPTQ2D_STATIC_MAX_DIM, otherwise GPTQ2D_ERR_TOO_LARGE is returned and nothing runs.
+ *   - The call itself allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).
+ *   - The FIRST call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; the call
+ *     clears what must start at zero.  Two calls that overlap on the GPU (different streams, no
+ *     ordering between them) race on it: serialise them.
+ */
+#define GPTQ2D_STATIC_MAX_DIM 512
+#define GPTQ2D_STATIC_WORKSPACE_BYTES (4u * 1024u * 1024u + 64u * 1024u)
+int gptq2d_round_static(int m, int n,
+                        const double *X, long ldx,
+                        const double *L, long ldl, const double *U, long ldu,
+                        int32_t *Z, long ldz,
+                        double *E, long lde, double *min_margin,
+                        int *info, void *stream);
+size_t gptq2d_round_static_max_dim(void);
 
 /* ---- the objective (Eq. 7): obj = || A (Z - X) B ||_F^2 ----
  * obj: device scalar.  A or B may be NULL (identity).

@@ -40,6 +40,7 @@ const char *gptq2d_status_string(int status) {
         case GPTQ2D_ERR_NONFINITE: return "non-finite value met while rounding";
         case GPTQ2D_ERR_INT_OVERFLOW: return "corrected value does not fit int32";
         case GPTQ2D_ERR_DEVICE_TIMEOUT: return "bounded device-side wait expired";
+        case GPTQ2D_ERR_TOO_LARGE: return "problem larger than the static workspace allows";
         default: return "unknown status";
     }
 }

@@ -22,12 +22,14 @@ OK = 0
 STATUS_NAMES = {
     0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_WORKSPACE", 3: "ERR_UNSUPPORTED_DEVICE", 4: "ERR_CUDA",
     5: "ERR_NOT_SPD", 6: "ERR_NONFINITE", 7: "ERR_INT_OVERFLOW", 8: "ERR_DEVICE_TIMEOUT",
+    9: "ERR_TOO_LARGE",
 }
 
 EXPORTS = (
     "gptq2d_status_string", "gptq2d_factor_workspace_bytes", "gptq2d_factor",
     "gptq2d_round_workspace_bytes", "gptq2d_round", "gptq2d_round_host_workspace_bytes",
     "gptq2d_round_host", "gptq2d_objective_workspace_bytes", "gptq2d_objective",
+    "gptq2d_round_static", "gptq2d_round_static_max_dim",
 )
 
 
@@ -63,6 +65,10 @@ def _load():
     lib.gptq2d_round_host.argtypes = [i32, i32, vp, vp, vp, vp, vp, vp, i32, vp, sz, vp, vp]
     lib.gptq2d_objective.restype = i32
     lib.gptq2d_objective.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, sz, vp, vp]
+    lib.gptq2d_round_static.restype = i32
+    lib.gptq2d_round_static.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, vp]
+    lib.gptq2d_round_static_max_dim.restype = sz
+    lib.gptq2d_round_static_max_dim.argtypes = []
     return lib
 
 
@@ -171,6 +177,31 @@ def gptq2d_round(X, L, U, Z=None, E=None, min_margin=None, precision=FP64, works
     if st != OK:
         raise Gptq2dError(st)
     return Z, E, min_margin, info
+
+
+def gptq2d_round_static_max_dim():
+    return int(_lib.gptq2d_round_static_max_dim())
+
+
+def gptq2d_round_static(X, L, U, Z, E=None, min_margin=None, info=None, stream=None):
+    """The fp64 sweep for callers that must not allocate: no workspace argument, the library's
+    static device array is the scratch (m, n <= gptq2d_round_static_max_dim()).
+
+    Every buffer, Z included, is the caller's: this wrapper creates no tensor either.  All calls
+    on a device share the one scratch array, so do not let two of them overlap on the GPU.  The
+    first call on a device performs a one-time symbol look-up; issue it before any stream
+    capture.  A non-zero C status is raised as Gptq2dError; returns Z."""
+    m, n = X.shape
+    pX, ldx = _mat(X, torch.float64, "X")
+    pL, ldl = _mat(L, torch.float64, "L")
+    pU, ldu = _mat(U, torch.float64, "U")
+    pZ, ldz = _mat(Z, torch.int32, "Z")
+    pE, lde = _mat(E, torch.float64, "E")
+    st = _lib.gptq2d_round_static(m, n, pX, ldx, pL, ldl, pU, ldu, pZ, ldz, pE, lde, _ptr(min_margin),
+                                  _ptr(info), _stream_ptr(stream))
+    if st != OK:
+        raise Gptq2dError(st)
+    return Z
 
 
 def gptq2d_round_host(hX, hL, hU, hZ=None, hE=None, hmargin=None, precision=FP64, workspace=None, hinfo=None,
