@@ -141,7 +141,9 @@ __device__ __forceinline__ void mma_slab(Acc &acc, const double *As, const doubl
 
 // acc += A(128 x K) * B(K x 128) over k in [0, K).  `smem` holds NSTAGE stages.
 // All 256 threads of the CTA must call this; ends with every cp.async drained and a
-// __syncthreads(), so the caller may reuse `smem` right away.
+// __syncthreads(), so the caller may reuse `smem` right away.  This is the general loop
+// (ragged edges, unaligned operands); gemm_mainloop_fast below is the one that reaches the
+// tensor peak.
 template <bool A_KCONTIG, bool B_KCONTIG, int NSTAGE>
 __device__ __forceinline__ void gemm_mainloop(Acc &acc, double *smem, const Operand &A, const Operand &B, int K) {
     using SL = SlabLayout<A_KCONTIG, B_KCONTIG>;
@@ -176,6 +178,102 @@ __device__ __forceinline__ void gemm_mainloop(Acc &acc, double *smem, const Oper
     }
     cp_async_wait<0>();
     __syncthreads();
+}
+
+// Per-thread copy plan for one operand: 4 chunks of 16 bytes per slab, pointers advance by a
+// constant per slab.  Valid only for tiles that are fully in range and 16-byte aligned.
+template <bool KCONTIG>
+struct FastCopy {
+    const double *src[4];
+    int dst[4];
+    long step;
+    __device__ __forceinline__ void init(const Operand &op, int tid) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            int c = tid + i * GEMM_THREADS;
+            if (KCONTIG) {
+                int r = c >> 3, kk = (c & 7) * 2;
+                src[i] = op.ptr + (long)r * op.ld + kk;
+                dst[i] = r * LDK + kk;
+            } else {
+                int kr = c >> 6, cc = (c & 63) * 2;
+                src[i] = op.ptr + (long)kr * op.ld + cc;
+                dst[i] = kr * LDN + cc;
+            }
+        }
+        step = KCONTIG ? (long)BK : (long)BK * op.ld;
+    }
+    __device__ __forceinline__ void issue(double *smem, int i, long slab) const {
+        cp_async16(smem + dst[i], src[i] + slab * step, 16);
+    }
+};
+
+// Same contraction as gemm_mainloop for operand tiles that are fully in range and 16-byte aligned
+// and K a multiple of BK: the copies of the next slab are issued one pair per k4-step between the
+// MMAs (every MMA warp would otherwise run all its copy code right after the slab barrier and
+// leave the tensor pipe idle).
+template <bool A_KCONTIG, bool B_KCONTIG, int NSTAGE>
+__device__ __forceinline__ void gemm_mainloop_fast(Acc &acc, double *smem, const Operand &A, const Operand &B, int K) {
+    using SL = SlabLayout<A_KCONTIG, B_KCONTIG>;
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5, lane = tid & 31;
+    const int wm = warp >> 2, wn = warp & 3, g = lane >> 2, t = lane & 3;
+    const int nk = K / BK;
+    FastCopy<A_KCONTIG> ca;
+    FastCopy<B_KCONTIG> cb;
+    ca.init(A, tid);
+    cb.init(B, tid);
+#pragma unroll
+    for (int s = 0; s < NSTAGE - 1; ++s) {
+        if (s < nk) {
+            double *st = smem + s * SL::STAGE_DOUBLES;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { ca.issue(st, i, s); cb.issue(st + SL::A_DOUBLES, i, s); }
+        }
+        cp_async_commit();
+    }
+    for (int kt = 0; kt < nk; ++kt) {
+        cp_async_wait<NSTAGE - 2>();
+        __syncthreads();
+        const int nxt = kt + NSTAGE - 1;
+        const bool more = nxt < nk;
+        double *stn = smem + (nxt % NSTAGE) * SL::STAGE_DOUBLES;
+        const double *As = smem + (kt % NSTAGE) * SL::STAGE_DOUBLES;
+        const double *Bs = As + SL::A_DOUBLES;
+#pragma unroll
+        for (int kk = 0; kk < BK; kk += 4) {
+            double af[8], bf[4];
+#pragma unroll
+            for (int a = 0; a < 8; ++a) {
+                int r = wm * 64 + a * 8 + g;
+                af[a] = A_KCONTIG ? As[r * LDK + kk + t] : As[(kk + t) * LDN + r];
+            }
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                int c = wn * 32 + b * 8 + g;
+                bf[b] = B_KCONTIG ? Bs[c * LDK + kk + t] : Bs[(kk + t) * LDN + c];
+            }
+#pragma unroll
+            for (int a = 0; a < 8; ++a) {
+#pragma unroll
+                for (int b = 0; b < 4; ++b) dmma_m8n8k4(acc.v[a][b][0], acc.v[a][b][1], af[a], bf[b]);
+                if (a == 3 && more) ca.issue(stn, kk / 4, nxt);
+                if (a == 7 && more) cb.issue(stn + SL::A_DOUBLES, kk / 4, nxt);
+            }
+        }
+        cp_async_commit();
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+}
+
+// Picks the interleaved-copy loop when the operand tiles allow it.
+template <bool A_KCONTIG, bool B_KCONTIG, int NSTAGE>
+__device__ __forceinline__ void gemm_tile(Acc &acc, double *smem, const Operand &A, const Operand &B, int K) {
+    if (A.aligned16 && B.aligned16 && A.mn_valid == BM && B.mn_valid == BN && (K % BK) == 0)
+        gemm_mainloop_fast<A_KCONTIG, B_KCONTIG, NSTAGE>(acc, smem, A, B, K);
+    else
+        gemm_mainloop<A_KCONTIG, B_KCONTIG, NSTAGE>(acc, smem, A, B, K);
 }
 
 }  // namespace gptq2d

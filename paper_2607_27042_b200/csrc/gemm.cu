@@ -29,7 +29,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(GemmArgs p) {
 
     Acc acc;
     acc.zero();
-    gemm_mainloop<A_KCONTIG, B_KCONTIG, GEMM_NSTAGE>(acc, smem, A, B, p.K);
+    gemm_tile<A_KCONTIG, B_KCONTIG, GEMM_NSTAGE>(acc, smem, A, B, p.K);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int wm = warp >> 2, wn = warp & 3, g = lane >> 2, t = lane & 3;

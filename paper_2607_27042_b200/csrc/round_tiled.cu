@@ -481,7 +481,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                         a.ptr = p.Cbuf + (long)I * T * p.np + (long)src * T; a.ld = p.np; a.mn_valid = T; a.aligned16 = true;
                         b.ptr = p.U + (long)src * T * p.ldu + (long)J * T; b.ld = p.ldu; b.mn_valid = min(T, p.n - J * T); b.aligned16 = p.u_al16;
                     }
-                    gemm_mainloop<true, false, BULK_NSTAGE>(acc, smem, a, b, T);
+                    gemm_tile<true, false, BULK_NSTAGE>(acc, smem, a, b, T);
                 }
                 // bulk epilogue: Cd, or Y0 = X + Rt (zero outside the matrix)
                 {
@@ -640,7 +640,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                 Operand a = A, b = B;
                 a.ptr = A.ptr + (long)f_pos * T;               // k offset along the contiguous index
                 b.ptr = B.ptr + (long)f_pos * T * B.ld;        // k offset along rows
-                gemm_mainloop<true, false, BULK_NSTAGE>(acc, smem, a, b, (upto - f_pos) * T);
+                gemm_tile<true, false, BULK_NSTAGE>(acc, smem, a, b, (upto - f_pos) * T);
                 f_pos = upto;
             }
         }
