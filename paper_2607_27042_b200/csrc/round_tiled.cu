@@ -420,9 +420,6 @@ __device__ __forceinline__ unsigned ready_pop(const TiledKernelParams &p) {
         return e;
     }
 }
-__device__ __forceinline__ bool ready_nonempty(const TiledKernelParams &p) {
-    return (int)(ld_relaxed_u32(p.q_tail) - ld_relaxed_u32(p.q_head)) > 0;
-}
 
 __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKernelParams p) {
     extern __shared__ __align__(16) double smem[];
@@ -441,6 +438,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
     bool have = false;
     int type = 0, I = 0, J = 0;
     unsigned long long idle_spins = 0;
+    unsigned popped = 0u;          // ready-ring entry taken while a far part was running (uniform)
     Acc acc;
     acc.zero();
 
@@ -453,11 +451,12 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             if (!have) {
                 __syncthreads();
                 if (tid == 0) {
-                    unsigned e = ready_pop(p);
+                    unsigned e = popped ? popped : ready_pop(p);
                     s_flag = e != 0u;
                     s_task[1] = (int)((e >> 29) & 3u); s_task[2] = (int)((e >> 15) & 0x3fffu); s_task[3] = (int)(e & 0x7fffu);
                 }
                 __syncthreads();
+                popped = 0u;
                 if (!s_flag) break;
                 type = s_task[1]; I = s_task[2]; J = s_task[3];
                 if (type == 2) {
@@ -615,13 +614,14 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             while (f_pos < f_nfar) {
                 // how many source tiles from f_pos on are swept already; is there ready work to take over
                 __syncthreads();
-                if (tid == 0) { s_task[0] = f_nfar; s_flag = ready_nonempty(p) ? 1 : 0; }
+                if (tid == 0) { s_task[0] = f_nfar; s_task[1] = (int)ready_pop(p); }
                 __syncthreads();
                 for (int idx = f_pos + tid; idx < f_nfar; idx += blockDim.x)
                     if (ld_acquire_u32(flags + (long)idx * fstride) == 0u) atomicMin(&s_task[0], idx);
                 __syncthreads();
                 const int upto_ready = s_task[0];
-                const bool work = s_flag != 0;
+                popped = (unsigned)s_task[1];
+                const bool work = popped != 0u;
                 if (upto_ready == f_pos) {                   // next source not swept yet
                     if (work) { interrupted = true; break; }
                     if (++spins > SPIN_LIMIT || ld_relaxed_u32(p.abort) != 0u) {
