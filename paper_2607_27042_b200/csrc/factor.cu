@@ -22,15 +22,21 @@ constexpr int FB = 128;
 
 // One CTA.  S: bs x bs Schur complement (lower triangle read).  Writes P (lower, in place),
 // W = P^{-1} (full block, zeros above the diagonal) and diag(P).
+// The block is padded to 128 x 128 with the identity in shared memory.  Cholesky runs from the last
+// index to the first (one column scaling + one rank-one update of the leading part per step, 16 x 16
+// thread tiling); the inverse is built from 32 x 32 diagonal blocks by doubling,
+// W21 = -W22 (P21 W11), with the temporary product kept in the unused upper triangle of the P array.
+__device__ __forceinline__ int tri(int i, int j) { return i * (i + 1) / 2 + j; }   // packed lower triangle
+
 __global__ void __launch_bounds__(256) factor_diag_kernel(double *S, long lds, int bs, double *W, long ldw,
                                                           double *pdiag, int *info, int side, int k0) {
     extern __shared__ double sm[];
-    double *a = sm;               // [128][129]
-    double *w = sm + 128 * 129;   // packed lower triangle: (i, j <= i) at i(i+1)/2 + j
-    const int tid = threadIdx.x;
-    for (int idx = tid; idx < bs * bs; idx += blockDim.x) {
-        int i = idx / bs, j = idx % bs;
-        if (j <= i) a[i * 129 + j] = S[(long)i * lds + j];
+    double *a = sm;               // [128][129]: P in the lower triangle, scratch above it
+    double *w = sm + 128 * 129;   // packed lower triangle of W
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    for (int idx = tid; idx < 128 * 128; idx += blockDim.x) {
+        int i = idx >> 7, j = idx & 127;
+        if (j <= i) a[i * 129 + j] = (i < bs) ? S[(long)i * lds + j] : (i == j ? 1.0 : 0.0);
     }
     __syncthreads();
     for (int k = bs - 1; k >= 0; --k) {
@@ -40,31 +46,57 @@ __global__ void __launch_bounds__(256) factor_diag_kernel(double *S, long lds, i
             if (tid == 0) report(info, GPTQ2D_ERR_NOT_SPD, k0 + k, side, 0);
             d = 1.0;
         }
-        double pk = sqrt(d);
+        const double pk = sqrt(d), rk = 1.0 / pk;
         if (tid == 0) a[k * 129 + k] = pk;
-        for (int i = tid; i < k; i += blockDim.x) a[k * 129 + i] /= pk;     // P[k][i], i < k
+        for (int i = tid; i < k; i += blockDim.x) a[k * 129 + i] *= rk;     // P[k][i], i < k
         __syncthreads();
         // Schur complement of the leading k x k part (lower triangle)
-        for (int idx = tid; idx < k * k; idx += blockDim.x) {
-            int i = idx / k, j = idx % k;
-            if (j <= i) a[i * 129 + j] -= a[k * 129 + i] * a[k * 129 + j];
+        for (int i = ty; i < k; i += 16) {
+            const double pi = a[k * 129 + i];
+            for (int j = tx; j <= i; j += 16) a[i * 129 + j] = fma(-pi, a[k * 129 + j], a[i * 129 + j]);
         }
         __syncthreads();
     }
-    // W = P^{-1}: thread j owns column j (forward substitution down the column)
-    for (int j = tid; j < bs; j += blockDim.x) {
-        w[j * (j + 1) / 2 + j] = 1.0 / a[j * 129 + j];
-        for (int i = j + 1; i < bs; ++i) {
-            double s = 0.0;
-            for (int k = j; k < i; ++k) s = fma(a[i * 129 + k], w[k * (k + 1) / 2 + j], s);
-            w[i * (i + 1) / 2 + j] = -s / a[i * 129 + i];
+    // ---- W = P^{-1}.  Level 0: the four 32 x 32 diagonal blocks, one column per thread.
+    if (tid < 128) {
+        const int r0 = tid & ~31, j = tid & 31;
+        w[tri(r0 + j, r0 + j)] = 1.0 / a[(r0 + j) * 129 + r0 + j];
+        for (int i = j + 1; i < 32; ++i) {
+            double s0 = 0.0, s1 = 0.0;
+            int k = j;
+            for (; k + 1 < i; k += 2) {
+                s0 = fma(a[(r0 + i) * 129 + r0 + k], w[tri(r0 + k, r0 + j)], s0);
+                s1 = fma(a[(r0 + i) * 129 + r0 + k + 1], w[tri(r0 + k + 1, r0 + j)], s1);
+            }
+            if (k < i) s0 = fma(a[(r0 + i) * 129 + r0 + k], w[tri(r0 + k, r0 + j)], s0);
+            w[tri(r0 + i, r0 + j)] = -(s0 + s1) / a[(r0 + i) * 129 + r0 + i];
         }
     }
     __syncthreads();
+    // ---- doubling: blocks of b = 32, then 64
+    for (int b = 32; b < 128; b *= 2) {
+        const int npair = 128 / (2 * b), per = b * b;
+        // T = P21 W11, stored above the diagonal at rows s.., columns s + b ..
+        for (int idx = tid; idx < npair * per; idx += blockDim.x) {
+            const int pr = idx / per, rem = idx - pr * per, r = rem / b, c = rem - r * b, s0 = pr * 2 * b;
+            double acc = 0.0;
+            for (int k = c; k < b; ++k) acc = fma(a[(s0 + b + r) * 129 + s0 + k], w[tri(s0 + k, s0 + c)], acc);
+            a[(s0 + r) * 129 + s0 + b + c] = acc;
+        }
+        __syncthreads();
+        // W21 = -W22 T
+        for (int idx = tid; idx < npair * per; idx += blockDim.x) {
+            const int pr = idx / per, rem = idx - pr * per, r = rem / b, c = rem - r * b, s0 = pr * 2 * b;
+            double acc = 0.0;
+            for (int k = 0; k <= r; ++k) acc = fma(w[tri(s0 + b + r, s0 + b + k)], a[(s0 + k) * 129 + s0 + b + c], acc);
+            w[tri(s0 + b + r, s0 + c)] = -acc;
+        }
+        __syncthreads();
+    }
     for (int idx = tid; idx < bs * bs; idx += blockDim.x) {
-        int i = idx / bs, j = idx % bs;
+        int i = idx / bs, j = idx - i * bs;
         if (j <= i) S[(long)i * lds + j] = a[i * 129 + j];
-        W[(long)i * ldw + j] = (j <= i) ? w[i * (i + 1) / 2 + j] : 0.0;
+        W[(long)i * ldw + j] = (j <= i) ? w[tri(i, j)] : 0.0;
     }
     for (int i = tid; i < bs; i += blockDim.x) pdiag[i] = a[i * 129 + i];
 }
