@@ -9,27 +9,27 @@
 // sweep.  Cd and Rt are dense contractions and carry all but a T/(m+n) share of the flops,
 // so they run on the fp64 tensor path (dmma_gemm.cuh); tiles with equal I + J are independent.
 //
-// Scheduling.  Every tile has two bulk tasks (Cd and Rt), each split into a FAR part (all
-// source tiles except the adjacent one) and a NEAR step (the adjacent tile, one K = 128
-// chunk).  Far parts are listed wave by wave (I + J ascending) and claimed in that order
-// from one atomic counter by persistent CTAs (one per SM, cooperatively launched so that all
-// are resident); a far part waits (bounded) only on tiles two or more waves back, parks its
-// partial sum in the tile's own workspace region and announces it.  Everything on the
-// critical path runs as an inline continuation with no waiting: the near step runs on
-// whichever CTA completes its second prerequisite (far part parked / adjacent tile swept),
-// the in-tile sweep on whichever CTA completes the tile's second near step; near steps that
-// a swept tile releases go to a global ready ring which every CTA serves first -- at the
-// top of its loop, while it waits, and every few chunks of a far part (it then parks its
-// partial sum and un-parks it afterwards).  A far part only ever waits on tiles of earlier
-// waves, whose far parts were claimed earlier and whose continuations never wait, so the
-// earliest unfinished work can always progress.
+// Scheduling.  Two kinds of work, one persistent cooperatively launched grid (one CTA per SM):
+//  * FAR parts.  Each tile's Cd and Rt contractions over every source tile EXCEPT the adjacent
+//    one.  Listed wave by wave (I + J ascending) and claimed in that order from one atomic
+//    counter.  A far part waits (bounded) only on tiles two or more waves back, parks its
+//    partial sum in the tile's own workspace region and then announces it to the tile's four
+//    quadrant tasks.  This is >90 % of the flops and runs on the fp64 tensor path.
+//  * QUADRANT tasks (64 x 64), the critical path.  A quadrant pulls the adjacent tiles'
+//    contributions itself (four 64^3 DMMA products), sweeps, and adds its cross terms to the
+//    later quadrants of its tile.  It counts arrivals from exactly what it needs -- the two
+//    far parts of its tile, the two quadrants above that share its columns, the two quadrants
+//    to the left that share its rows, its predecessors inside the tile -- and the last arrival
+//    puts it on a global ready ring.  Quadrant tasks never wait.
+// Every CTA serves the ready ring first: at the top of its loop, while a far part waits, and
+// every few chunks of a far part (it then parks its partial sum and un-parks it afterwards).
+// A far part only ever waits on tiles of earlier waves, whose far parts were claimed earlier and
+// whose quadrant tasks never wait, so the earliest unfinished work can always progress.
 //
-// In-tile sweep.  The tile is processed as four 64 x 64 quadrants (the same restatement one
-// level down, cross terms as 64^3 DMMA products).  Inside a quadrant the anti-diagonal
-// sweep runs on 8 x 8 leaves: each leaf of a leaf-wave is swept by one warp (two entries per
-// lane, errors exchanged through a 16-double shared-memory buffer, branch-free pushes), then
-// all warps apply the leaves' feedback to the remaining 8 x 8 blocks of the quadrant with
-// m8n8k4 DMMA.
+// In-tile sweep.  Inside a quadrant the anti-diagonal sweep runs on 8 x 8 leaves: each leaf of a
+// leaf-wave is swept by one warp (two entries per lane, errors exchanged through a 16-double
+// shared-memory buffer, branch-free pushes against zero-padded coefficient tables), and the
+// leaves' feedback to the remaining 8 x 8 blocks of the quadrant is m8n8k4 DMMA.
 #include "common.cuh"
 #include "dmma_gemm.cuh"
 #include "round_internal.cuh"
@@ -56,9 +56,8 @@ struct TiledKernelParams {
     unsigned *counter, *abort, *q_head, *q_tail, *tiles_done;
     unsigned *q_slots;           // [QCAP] ready continuation tasks
     unsigned *flagS;             // [ntm*ntn] tile swept
-    unsigned *bulk_done;         // [ntm*ntn] number of finished bulk contractions (2 -> sweep)
-    unsigned *quad_done;         // [ntm*ntn] finished ones of quadrants 1 and 2 (2 -> quadrant 3)
-    unsigned *near_dep;          // [2][ntm*ntn] arrivals for the near step: far part parked, source tile swept
+    unsigned *quad_done;         // [ntm*ntn] swept quadrants of the tile (4 -> tile flag)
+    unsigned *qdep;              // [ntm*ntn][4] arrivals each quadrant task has received
     double *max_abs_e;
     int *info;
     int l_al16, u_al16;
@@ -104,15 +103,21 @@ __device__ __forceinline__ void load_factor_block_async(double *dst, const doubl
     }
 }
 
-// G (global 64 x 64, row stride ld) += As (64 x 64, [m][k]) * Bs (64 x 64, [k][n])
-__device__ __forceinline__ void cross_gemm(double *G, long ld, const double *As, const double *Bs) {
+// 64 x 64 x 64 DMMA product on quadrant operands in shared memory: each warp owns a 16 x 32 piece
+// (2 x 4 fragments); element rows wr*16 + a*8 + (lane>>2), cols wc*32 + b*8 + (lane&3)*2 + {0,1}.
+struct QAcc {
+    double v[2][4][2];
+    __device__ __forceinline__ void zero() {
+#pragma unroll
+        for (int a = 0; a < 2; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) v[a][b][0] = v[a][b][1] = 0.0;
+    }
+};
+// acc += As (64 x 64, [m][k]) * Bs (64 x 64, [k][n])
+__device__ __forceinline__ void quad_mma(QAcc &acc, const double *As, const double *Bs) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int wr = warp >> 1, wc = warp & 1;
-    double acc[2][4][2];
-#pragma unroll
-    for (int a = 0; a < 2; ++a)
-#pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b][0] = acc[a][b][1] = 0.0;
 #pragma unroll 4
     for (int kk = 0; kk < Q; kk += 4) {
         double af[2], bf[4];
@@ -123,18 +128,30 @@ __device__ __forceinline__ void cross_gemm(double *G, long ld, const double *As,
 #pragma unroll
         for (int a = 0; a < 2; ++a)
 #pragma unroll
-            for (int b = 0; b < 4; ++b) dmma_m8n8k4(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
+            for (int b = 0; b < 4; ++b) dmma_m8n8k4(acc.v[a][b][0], acc.v[a][b][1], af[a], bf[b]);
     }
+}
+// D (64 x 64 with row stride ld, global or shared) += acc
+__device__ __forceinline__ void quad_add_to(double *D, long ld, const QAcc &acc, bool global_cg) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const int wr = warp >> 1, wc = warp & 1;
 #pragma unroll
     for (int a = 0; a < 2; ++a)
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
-            double2 *ptr = reinterpret_cast<double2 *>(G + (long)(wr * 16 + a * 8 + g) * ld + wc * 32 + b * 8 + t * 2);
-            double2 v = __ldcg(ptr);
-            v.x += acc[a][b][0];
-            v.y += acc[a][b][1];
+            double2 *ptr = reinterpret_cast<double2 *>(D + (long)(wr * 16 + a * 8 + g) * ld + wc * 32 + b * 8 + t * 2);
+            double2 v = global_cg ? __ldcg(ptr) : *ptr;
+            v.x += acc.v[a][b][0];
+            v.y += acc.v[a][b][1];
             *ptr = v;
         }
+}
+// G (global 64 x 64, row stride ld) += As (64 x 64, [m][k]) * Bs (64 x 64, [k][n])
+__device__ __forceinline__ void cross_gemm(double *G, long ld, const double *As, const double *Bs) {
+    QAcc acc;
+    acc.zero();
+    quad_mma(acc, As, Bs);
+    quad_add_to(G, ld, acc, true);
 }
 
 // One 8 x 8 target block (pb, qb) of the quadrant receives the feedback of leaf-wave `lw`:
@@ -286,13 +303,21 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
 }
 
 // ---------------------------------------------------------------------------------------------
-// One 64 x 64 quadrant q (0: top-left, 1: top-right, 2: bottom-left, 3: bottom-right) of the
-// in-tile sweep of tile (I, J).  On entry the tile's Ebuf region holds X + Rt and its Cbuf
-// region Cd, both already updated by the cross terms of the quadrants this one depends on;
-// on exit the quadrant's regions hold E and C = L E, Z (and the caller's E) are written, and
-// the cross terms this quadrant owes to later quadrants of the tile have been added to their
-// regions: q0 -> q1 (through U) and q2 (through L); q1 -> q3 (through L); q2 -> q3 (through U).
-// Quadrants 1 and 2 are independent of each other and may run on different CTAs.
+// One 64 x 64 quadrant q (0: top-left, 1: top-right, 2: bottom-left, 3: bottom-right) of tile
+// (I, J): the unit of work on the critical path.
+//
+// On entry the quadrant's part of the tile's Cbuf region holds the FAR part of Cd (all source
+// tiles above except the adjacent one) and its Ebuf part the FAR part of Rt, both already
+// updated by the cross terms of the quadrants of this tile it depends on.  The task
+//   1. pulls the adjacent tiles' contributions itself: Cd += L[rows, tile I-1] E[tile I-1, cols]
+//      and Rt += C[rows, tile J-1] U[tile J-1, cols], four 64^3 DMMA products staged through two
+//      pairs of shared-memory buffers (they need only the two quadrants of each neighbour that
+//      share this quadrant's columns / rows, which is what its dependency counter waits for);
+//   2. forms Y = X + Rt + Cd, C = Cd and runs Algorithm 3 on the quadrant;
+//   3. writes E, C = L E, Z (and the caller's E), and adds the cross terms it owes to later
+//      quadrants of the tile: q0 -> q1 (through U) and q2 (through L); q1 -> q3 (through L);
+//      q2 -> q3 (through U).
+// Quadrants 1 and 2 of a tile are independent of each other.
 __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem, const TiledKernelParams &p,
                                                double &max_abs_e) {
     double *Ys = smem, *Cs = smem + QMAT, *Ls = smem + 2 * QMAT, *Us = smem + 3 * QMAT, *Xop = smem + 4 * QMAT;
@@ -305,7 +330,43 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
     const int row0 = I * T + qi * Q, col0 = J * T + qj * Q;
     double *eQ = eT + (long)qi * Q * p.np + qj * Q;
     double *cQ = cT + (long)qi * Q * p.np + qj * Q;
-    __syncthreads();
+
+    // ---- 1. near pulls.  Steps 0,1: Cd halves (k over the two quadrant rows of tile I-1);
+    // steps 2,3: Rt halves (k over the two quadrant columns of tile J-1).  Operands of step k go to
+    // buffer pair k & 1 = {(Ls, Us), (Xop, Cs)}; loads run one step ahead of the products.
+    QAcc accC, accR;
+    accC.zero();
+    accR.zero();
+    {
+        const int first = I > 0 ? 0 : 2, last = J > 0 ? 4 : 2;     // steps [first, last)
+        auto issue = [&](int k) {
+            double *Ab = (k & 1) ? Xop : Ls, *Bb = (k & 1) ? Cs : Us;
+            const int kh = k & 1;
+            if (k < 2) {
+                const int k0 = (I - 1) * T + kh * Q;
+                load_factor_block_async(Ab, p.L, p.ldl, p.m, row0, k0, 0);
+                load_quadrant_async(Bb, p.Ebuf + (long)k0 * p.np + col0, p.np);
+            } else {
+                const int k0 = (J - 1) * T + kh * Q;
+                load_quadrant_async(Ab, p.Cbuf + (long)row0 * p.np + k0, p.np);
+                load_factor_block_async(Bb, p.U, p.ldu, p.n, k0, col0, 0);
+            }
+            cp_async_commit();
+        };
+        __syncthreads();
+        if (first < last) issue(first);
+        if (first + 1 < last) issue(first + 1);
+        for (int k = first; k < last; ++k) {
+            if (k + 1 < last) cp_async_wait<1>(); else cp_async_wait<0>();
+            __syncthreads();
+            const double *Ab = (k & 1) ? Xop : Ls, *Bb = (k & 1) ? Cs : Us;
+            if (k < 2) quad_mma(accC, Ab, Bb); else quad_mma(accR, Ab, Bb);
+            __syncthreads();
+            if (k + 2 < last) issue(k + 2);
+        }
+    }
+
+    // ---- 2. operands of the sweep
     load_factor_block_async(Ls, p.L, p.ldl, p.m, row0, row0, 1);
     load_factor_block_async(Us, p.U, p.ldu, p.n, col0, col0, 2);
     load_quadrant_async(Cs, cQ, p.np);
@@ -314,16 +375,26 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
     if (q == 0 || q == 2) load_factor_block_async(Xop, p.U, p.ldu, p.n, J * T, J * T + Q, 0);
     if (q == 1) load_factor_block_async(Xop, p.L, p.ldl, p.m, I * T + Q, I * T, 0);
     cp_async_commit();
+    double xv[16];
+#pragma unroll
+    for (int it = 0; it < 16; ++it) {                     // X of the quadrant, zero outside the matrix
+        int c = tid + it * TILED_THREADS;
+        int gr = row0 + (c >> 6), gc = col0 + (c & 63);
+        xv[it] = (gr < p.m && gc < p.n) ? __ldg(p.X + (long)gr * p.ldx + gc) : 0.0;
+    }
     cp_async_wait<0>();
+    __syncthreads();
+    quad_add_to(Cs, QLD, accC, false);                    // Cd = far part + cross terms + near pull
+    quad_add_to(Ys, QLD, accR, false);                    // Rt likewise
     __syncthreads();
 #pragma unroll
     for (int it = 0; it < 16; ++it) {                     // Y = X + Rt + Cd
         int c = tid + it * TILED_THREADS;
         int r = c >> 6, cc = c & 63;
-        Ys[r * QLD + cc] += Cs[r * QLD + cc];
+        Ys[r * QLD + cc] += xv[it] + Cs[r * QLD + cc];
     }
     quadrant_sweep(Ys, Cs, Ls, Us, Zs, tabL, tabU, row0, col0, p, max_abs_e);
-    // results of the quadrant
+    // ---- 3. results of the quadrant
     store_quadrant(eQ, p.np, Ys);
     store_quadrant(cQ, p.np, Cs);
 #pragma unroll
@@ -393,7 +464,7 @@ __device__ __forceinline__ void load_acc(Acc &acc, const double *srcT, long np, 
 }
 
 constexpr unsigned QCAP = 4096;   // global ring of ready continuation tasks (power of two)
-constexpr int FAR_RUN_CHUNKS = 8; // a far part looks at the ready queue every this many K = 128 chunks
+constexpr int FAR_RUN_CHUNKS = 16; // a far part looks at the ready queue every this many K = 128 chunks
 
 // multi-producer / multi-consumer ring in global memory; slot value 0 = empty.
 __device__ __forceinline__ void ready_push(const TiledKernelParams &p, unsigned entry) {
@@ -421,6 +492,22 @@ __device__ __forceinline__ unsigned ready_pop(const TiledKernelParams &p) {
     }
 }
 
+// Arrivals a quadrant task waits for: the two far parts of its tile, the two quadrants of the tile
+// above that share its columns, the two quadrants of the tile to the left that share its rows, and
+// its predecessors inside the tile (q1, q2 <- q0; q3 <- q1, q2).
+__device__ __forceinline__ unsigned quadrant_needed(int I, int J, int q) {
+    return 2u + (I > 0 ? 2u : 0u) + (J > 0 ? 2u : 0u) + (q == 0 ? 0u : (q == 3 ? 2u : 1u));
+}
+// thread 0 only; the caller has fenced its own results.  The arrival that completes the count
+// publishes the task on the ready ring.
+__device__ __forceinline__ void quadrant_arrive(const TiledKernelParams &p, int I, int J, int q) {
+    unsigned old = atomicAdd(p.qdep + ((long)I * p.ntn + J) * 4 + q, 1u);
+    if (old + 1u == quadrant_needed(I, J, q)) {
+        __threadfence();
+        ready_push(p, ((unsigned)q << 29) | ((unsigned)I << 15) | (unsigned)J);
+    }
+}
+
 __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKernelParams p) {
     extern __shared__ __align__(16) double smem[];
     __shared__ int s_task[4];
@@ -434,129 +521,37 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
     // far-part context of this CTA (uniform across the CTA)
     bool f_valid = false;
     int f_type = 0, f_I = 0, f_J = 0, f_pos = 0, f_nfar = 0, f_task = 0;
-    // continuation handed over with the accumulator still in registers
-    bool have = false;
-    int type = 0, I = 0, J = 0;
     unsigned long long idle_spins = 0;
     unsigned popped = 0u;          // ready-ring entry taken while a far part was running (uniform)
     Acc acc;
     acc.zero();
 
     for (;;) {
-        // ================= A: continuations (near step, quadrant sweeps, releases).  Never waits.
-        // Ready-ring entries: kind 0 / 1 = near step of the Cd / Rt contraction of tile (I, J);
-        // kind 2 = bottom-left quadrant of the in-tile sweep of tile (I, J).
+        // ================= A: quadrant tasks from the ready ring.  Never waits.
         for (;;) {
-            int quad = -1;                 // >= 0: next quadrant of tile (I, J) to sweep on this CTA
-            if (!have) {
-                __syncthreads();
-                if (tid == 0) {
-                    unsigned e = popped ? popped : ready_pop(p);
-                    s_flag = e != 0u;
-                    s_task[1] = (int)((e >> 29) & 3u); s_task[2] = (int)((e >> 15) & 0x3fffu); s_task[3] = (int)(e & 0x7fffu);
-                }
-                __syncthreads();
-                popped = 0u;
-                if (!s_flag) break;
-                type = s_task[1]; I = s_task[2]; J = s_task[3];
-                if (type == 2) {
-                    quad = 2;
-                } else if ((type == 0 ? I : J) > 1) {
-                    load_acc(acc, (type == 0 ? p.Cbuf : p.Ebuf) + (long)I * T * p.np + (long)J * T, p.np, wm, wn, g, t);
-                } else {
-                    acc.zero();
-                }
+            __syncthreads();
+            if (tid == 0) {
+                unsigned e = popped ? popped : ready_pop(p);
+                s_flag = e != 0u;
+                s_task[1] = (int)((e >> 29) & 3u); s_task[2] = (int)((e >> 15) & 0x3fffu); s_task[3] = (int)(e & 0x7fffu);
             }
-            have = false;
-            if (quad < 0) {
-                // near step: the adjacent source tile (already swept, by construction)
-                const int src = (type == 0 ? I : J) - 1;
-                if (src >= 0) {
-                    Operand a, b;
-                    if (type == 0) {
-                        a.ptr = p.L + (long)I * T * p.ldl + (long)src * T; a.ld = p.ldl; a.mn_valid = min(T, p.m - I * T); a.aligned16 = p.l_al16;
-                        b.ptr = p.Ebuf + (long)src * T * p.np + (long)J * T; b.ld = p.np; b.mn_valid = T; b.aligned16 = true;
-                    } else {
-                        a.ptr = p.Cbuf + (long)I * T * p.np + (long)src * T; a.ld = p.np; a.mn_valid = T; a.aligned16 = true;
-                        b.ptr = p.U + (long)src * T * p.ldu + (long)J * T; b.ld = p.ldu; b.mn_valid = min(T, p.n - J * T); b.aligned16 = p.u_al16;
-                    }
-                    gemm_tile<true, false, BULK_NSTAGE>(acc, smem, a, b, T);
-                }
-                // bulk epilogue: Cd, or Y0 = X + Rt (zero outside the matrix)
-                {
-                    double *dstT = (type == 0 ? p.Cbuf : p.Ebuf) + (long)I * T * p.np + (long)J * T;
-#pragma unroll
-                    for (int a = 0; a < 8; ++a) {
-                        const int r = wm * 64 + a * 8 + g;
-                        const int gr = I * T + r;
-#pragma unroll
-                        for (int b = 0; b < 4; ++b) {
-                            const int c = wn * 32 + b * 8 + t * 2;
-                            const int gc = J * T + c;
-                            double2 v;
-                            v.x = acc.v[a][b][0];
-                            v.y = acc.v[a][b][1];
-                            if (type == 1) {
-                                double x0 = 0.0, x1 = 0.0;
-                                if (gr < p.m) {
-                                    if (gc < p.n) x0 = __ldg(p.X + (long)gr * p.ldx + gc);
-                                    if (gc + 1 < p.n) x1 = __ldg(p.X + (long)gr * p.ldx + gc + 1);
-                                }
-                                v.x += x0;
-                                v.y += x1;
-                            }
-                            *reinterpret_cast<double2 *>(dstT + (long)r * p.np + c) = v;
-                        }
-                    }
-                }
-                __syncthreads();
-                if (tid == 0) {
+            __syncthreads();
+            popped = 0u;
+            if (!s_flag) break;
+            const int q = s_task[1], I = s_task[2], J = s_task[3];
+            sweep_quadrant(I, J, q, smem, p, max_abs_e);
+            if (tid == 0) {
+                __threadfence();
+                const int qi = q >> 1, qj = q & 1;
+                if (q == 0) { quadrant_arrive(p, I, J, 1); quadrant_arrive(p, I, J, 2); }
+                else if (q != 3) quadrant_arrive(p, I, J, 3);
+                if (I + 1 < p.ntm) { quadrant_arrive(p, I + 1, J, qj); quadrant_arrive(p, I + 1, J, 2 + qj); }
+                if (J + 1 < p.ntn) { quadrant_arrive(p, I, J + 1, 2 * qi); quadrant_arrive(p, I, J + 1, 2 * qi + 1); }
+                unsigned done = atomicAdd(p.quad_done + (long)I * p.ntn + J, 1u);
+                if (done == 3u) {          // tile swept: far parts that list it as a source may go on
                     __threadfence();
-                    unsigned old = atomicAdd(p.bulk_done + (long)I * p.ntn + J, 1u);
-                    __threadfence();
-                    s_flag = (old == 1u) ? 1 : 0;
-                }
-                __syncthreads();
-                if (!s_flag) continue;
-                quad = 0;                  // both contractions of tile (I, J) are complete: sweep it
-            }
-            // in-tile sweep, quadrant by quadrant: 0, then 1 here while 2 is offered to the ready ring
-            // (an idle CTA takes it, otherwise this CTA pops it itself), then 3 on whichever CTA
-            // finishes the second of quadrants 1 and 2.
-            while (quad >= 0) {
-                sweep_quadrant(I, J, quad, smem, p, max_abs_e);
-                if (quad == 0) {
-                    if (tid == 0) {
-                        __threadfence();
-                        ready_push(p, (2u << 29) | ((unsigned)I << 15) | (unsigned)J);
-                    }
-                    quad = 1;
-                } else if (quad == 1 || quad == 2) {
-                    if (tid == 0) {
-                        __threadfence();
-                        unsigned old = atomicAdd(p.quad_done + (long)I * p.ntn + J, 1u);
-                        __threadfence();
-                        s_flag = (old == 1u) ? 1 : 0;
-                    }
-                    __syncthreads();
-                    quad = s_flag ? 3 : -1;
-                } else {
-                    // tile swept: publish it and release the near steps of the tile below and to the right
-                    if (tid == 0) {
-                        __threadfence();
-                        st_release_u32(p.flagS + (long)I * p.ntn + J, 1u);
-                        for (int d = 0; d < 2; ++d) {
-                            const int dI = I + (d == 0 ? 1 : 0), dJ = J + (d == 0 ? 0 : 1);
-                            if (dI >= p.ntm || dJ >= p.ntn) continue;
-                            unsigned old = atomicAdd(p.near_dep + ((long)d * ntiles + (long)dI * p.ntn + dJ), 1u);
-                            if (old == 1u) {      // its far part is parked already: the near step is ready
-                                __threadfence();
-                                ready_push(p, ((unsigned)d << 29) | ((unsigned)dI << 15) | (unsigned)dJ);
-                            }
-                        }
-                        atomicAdd(p.tiles_done, 1u);
-                    }
-                    quad = -1;
+                    st_release_u32(p.flagS + (long)I * p.ntn + J, 1u);
+                    atomicAdd(p.tiles_done, 1u);
                 }
             }
         }
@@ -576,7 +571,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             __syncthreads();
             if (s_task[0] >= p.ntasks) {
                 if (s_flag) break;                           // every tile is swept: done
-                if (++idle_spins > SPIN_LIMIT) {             // nothing to claim: wait for continuations
+                if (++idle_spins > SPIN_LIMIT) {             // nothing to claim: wait for ready tasks
                     if (tid == 0) {
                         report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -4, (int)blockIdx.x, 0);
                         atomicExch(p.abort, 1u);
@@ -592,7 +587,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             f_valid = true;
             acc.zero();
         } else {
-            // coming back from continuations: un-park the partial sum
+            // coming back from quadrant tasks: un-park the partial sum
             if (f_pos > 0)
                 load_acc(acc, (f_type == 0 ? p.Cbuf : p.Ebuf) + (long)f_I * T * p.np + (long)f_J * T, p.np, wm, wn, g, t);
             else
@@ -612,7 +607,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             }
             unsigned long long spins = 0;
             while (f_pos < f_nfar) {
-                // how many source tiles from f_pos on are swept already; is there ready work to take over
+                // how many source tiles from f_pos on are swept already; is there a ready task to take over
                 __syncthreads();
                 if (tid == 0) { s_task[0] = f_nfar; s_task[1] = (int)ready_pop(p); }
                 __syncthreads();
@@ -622,8 +617,8 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                 const int upto_ready = s_task[0];
                 popped = (unsigned)s_task[1];
                 const bool work = popped != 0u;
+                if (work) { interrupted = true; break; }       // park and serve the critical path first
                 if (upto_ready == f_pos) {                   // next source not swept yet
-                    if (work) { interrupted = true; break; }
                     if (++spins > SPIN_LIMIT || ld_relaxed_u32(p.abort) != 0u) {
                         if (tid == 0) {
                             report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, f_task, f_pos, (int)blockIdx.x);
@@ -635,7 +630,6 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                     __nanosleep(100);
                     continue;
                 }
-                if (work) { interrupted = true; break; }       // park and serve the critical path first
                 const int upto = min(upto_ready, f_pos + FAR_RUN_CHUNKS);
                 Operand a = A, b = B;
                 a.ptr = A.ptr + (long)f_pos * T;               // k offset along the contiguous index
@@ -645,22 +639,17 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             }
         }
         if (ld_relaxed_u32(p.abort) != 0u) break;
-        // park the partial sum in the tile's own output region
-        if (f_pos > 0)
+        // park the partial sum in the tile's own region (Cd in Cbuf, Rt in Ebuf); a finished far part
+        // always writes it, zeros included, because the quadrant tasks start from it
+        if (f_pos > 0 || !interrupted)
             store_acc(acc, (f_type == 0 ? p.Cbuf : p.Ebuf) + (long)f_I * T * p.np + (long)f_J * T, p.np, wm, wn, g, t);
         if (interrupted) continue;                            // back to A, then resume this far part
-        // far part complete: announce it; if the adjacent tile is swept already, go on with the near step
+        // far part complete: announce it to the four quadrants of its tile
         __syncthreads();
         if (tid == 0) {
-            const bool has_src = (f_type == 0 ? f_I : f_J) > 0;
             __threadfence();
-            unsigned old = atomicAdd(p.near_dep + ((long)f_type * ntiles + (long)f_I * p.ntn + f_J), 1u);
-            __threadfence();
-            s_flag = (old + 1u == (has_src ? 2u : 1u)) ? 1 : 0;
+            for (int q = 0; q < 4; ++q) quadrant_arrive(p, f_I, f_J, q);
         }
-        __syncthreads();
-        have = s_flag != 0;
-        type = f_type; I = f_I; J = f_J;
         f_valid = false;
     }
 
@@ -679,7 +668,7 @@ static size_t pad256(size_t x) { return (x + 255) / 256 * 256; }
 
 struct TiledLayout {
     int ntm, ntn;
-    size_t q_off, flags_off, done_off, quad_off, near_off, e_off, c_off, total;
+    size_t q_off, flags_off, quad_off, qdep_off, e_off, c_off, total;
 };
 static TiledLayout tiled_layout(int m, int n) {
     TiledLayout l;
@@ -689,10 +678,9 @@ static TiledLayout tiled_layout(int m, int n) {
     size_t mat = (size_t)l.ntm * T * (size_t)l.ntn * T * sizeof(double);
     l.q_off = 256;
     l.flags_off = l.q_off + 4096 * sizeof(unsigned);
-    l.done_off = l.flags_off + pad256(tiles * sizeof(unsigned));
-    l.quad_off = l.done_off + pad256(tiles * sizeof(unsigned));
-    l.near_off = l.quad_off + pad256(tiles * sizeof(unsigned));
-    l.e_off = l.near_off + pad256(2 * tiles * sizeof(unsigned));
+    l.quad_off = l.flags_off + pad256(tiles * sizeof(unsigned));
+    l.qdep_off = l.quad_off + pad256(tiles * sizeof(unsigned));
+    l.e_off = l.qdep_off + pad256(4 * tiles * sizeof(unsigned));
     l.c_off = l.e_off + pad256(mat);
     l.total = l.c_off + pad256(mat);
     return l;
@@ -718,9 +706,8 @@ int launch_round_tiled(const TiledParams &in, void *ws, size_t ws_bytes, cudaStr
     p.q_slots = reinterpret_cast<unsigned *>(w + l.q_off);
     p.max_abs_e = workspace_max_abs_e(ws);
     p.flagS = reinterpret_cast<unsigned *>(w + l.flags_off);
-    p.bulk_done = reinterpret_cast<unsigned *>(w + l.done_off);
-    p.near_dep = reinterpret_cast<unsigned *>(w + l.near_off);
     p.quad_done = reinterpret_cast<unsigned *>(w + l.quad_off);
+    p.qdep = reinterpret_cast<unsigned *>(w + l.qdep_off);
     p.Ebuf = reinterpret_cast<double *>(w + l.e_off);
     p.Cbuf = reinterpret_cast<double *>(w + l.c_off);
     p.info = in.info;
