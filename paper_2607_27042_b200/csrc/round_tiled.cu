@@ -103,6 +103,18 @@ __device__ __forceinline__ void load_factor_block_async(double *dst, const doubl
     }
 }
 
+// Whole 64 x 64 block (no triangle mask) with 16-byte copies; needs M 16-byte aligned, ld and c0 even.
+__device__ __forceinline__ void load_full_block_async16(double *dst, const double *M, long ld, int k, int r0, int c0) {
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+        int c = threadIdx.x + it * TILED_THREADS;
+        int r = c >> 5, cc = (c & 31) * 2;
+        int gr = r0 + r, gc = c0 + cc;
+        int nv = (gr < k) ? min(2, max(0, k - gc)) : 0;
+        cp_async16(dst + r * QLD + cc, nv ? M + (long)gr * ld + gc : M, nv * 8);
+    }
+}
+
 // 64 x 64 x 64 DMMA product on quadrant operands in shared memory: each warp owns a 16 x 32 piece
 // (2 x 4 fragments); element rows wr*16 + a*8 + (lane>>2), cols wc*32 + b*8 + (lane&3)*2 + {0,1}.
 struct QAcc {
@@ -339,31 +351,40 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
     accR.zero();
     {
         const int first = I > 0 ? 0 : 2, last = J > 0 ? 4 : 2;     // steps [first, last)
-        auto issue = [&](int k) {
-            double *Ab = (k & 1) ? Xop : Ls, *Bb = (k & 1) ? Cs : Us;
-            const int kh = k & 1;
+        const int ns = last - first;
+        // three buffer pairs, so that up to three steps are in flight; the third pair borrows Ys and
+        // the area of the coefficient tables / Z staging, all unused until the sweep proper
+        auto bufA = [&](int j) { return j == 0 ? Ls : (j == 1 ? Xop : Ys); };
+        auto bufB = [&](int j) { return j == 0 ? Us : (j == 1 ? Cs : tabL); };
+        auto issue = [&](int i) {
+            const int k = first + i, kh = k & 1;
+            double *Ab = bufA(i % 3), *Bb = bufB(i % 3);
             if (k < 2) {
                 const int k0 = (I - 1) * T + kh * Q;
-                load_factor_block_async(Ab, p.L, p.ldl, p.m, row0, k0, 0);
+                if (p.l_al16) load_full_block_async16(Ab, p.L, p.ldl, p.m, row0, k0);
+                else load_factor_block_async(Ab, p.L, p.ldl, p.m, row0, k0, 0);
                 load_quadrant_async(Bb, p.Ebuf + (long)k0 * p.np + col0, p.np);
             } else {
                 const int k0 = (J - 1) * T + kh * Q;
                 load_quadrant_async(Ab, p.Cbuf + (long)row0 * p.np + k0, p.np);
-                load_factor_block_async(Bb, p.U, p.ldu, p.n, k0, col0, 0);
+                if (p.u_al16) load_full_block_async16(Bb, p.U, p.ldu, p.n, k0, col0);
+                else load_factor_block_async(Bb, p.U, p.ldu, p.n, k0, col0, 0);
             }
             cp_async_commit();
         };
         __syncthreads();
-        if (first < last) issue(first);
-        if (first + 1 < last) issue(first + 1);
-        for (int k = first; k < last; ++k) {
-            if (k + 1 < last) cp_async_wait<1>(); else cp_async_wait<0>();
+        for (int i = 0; i < ns && i < 3; ++i) issue(i);
+        for (int i = 0; i < ns; ++i) {
+            const int pending = min(ns, i + 3) - (i + 1);        // groups issued after step i's
+            if (pending >= 2) cp_async_wait<2>(); else if (pending == 1) cp_async_wait<1>(); else cp_async_wait<0>();
             __syncthreads();
-            const double *Ab = (k & 1) ? Xop : Ls, *Bb = (k & 1) ? Cs : Us;
-            if (k < 2) quad_mma(accC, Ab, Bb); else quad_mma(accR, Ab, Bb);
-            __syncthreads();
-            if (k + 2 < last) issue(k + 2);
+            if (first + i < 2) quad_mma(accC, bufA(i % 3), bufB(i % 3)); else quad_mma(accR, bufA(i % 3), bufB(i % 3));
+            if (i + 3 < ns) {
+                __syncthreads();
+                issue(i + 3);
+            }
         }
+        __syncthreads();
     }
 
     // ---- 2. operands of the sweep
@@ -464,7 +485,8 @@ __device__ __forceinline__ void load_acc(Acc &acc, const double *srcT, long np, 
 }
 
 constexpr unsigned QCAP = 4096;   // global ring of ready continuation tasks (power of two)
-constexpr int FAR_RUN_CHUNKS = 16; // a far part looks at the ready queue every this many K = 128 chunks
+constexpr int FAR_RUN_CHUNKS = 16;
+constexpr unsigned IDLE_SLEEP_NS = 400; // a far part looks at the ready queue every this many K = 128 chunks
 
 // multi-producer / multi-consumer ring in global memory; slot value 0 = empty.
 __device__ __forceinline__ void ready_push(const TiledKernelParams &p, unsigned entry) {
@@ -498,13 +520,14 @@ __device__ __forceinline__ unsigned ready_pop(const TiledKernelParams &p) {
 __device__ __forceinline__ unsigned quadrant_needed(int I, int J, int q) {
     return 2u + (I > 0 ? 2u : 0u) + (J > 0 ? 2u : 0u) + (q == 0 ? 0u : (q == 3 ? 2u : 1u));
 }
-// thread 0 only; the caller has fenced its own results.  The arrival that completes the count
+// the caller has fenced the CTA's results (after a barrier).  The arrival that completes the count
 // publishes the task on the ready ring.
 __device__ __forceinline__ void quadrant_arrive(const TiledKernelParams &p, int I, int J, int q) {
     unsigned old = atomicAdd(p.qdep + ((long)I * p.ntn + J) * 4 + q, 1u);
     if (old + 1u == quadrant_needed(I, J, q)) {
+        const unsigned entry = ((unsigned)q << 29) | ((unsigned)I << 15) | (unsigned)J | 0x80000000u;
         __threadfence();
-        ready_push(p, ((unsigned)q << 29) | ((unsigned)I << 15) | (unsigned)J);
+        ready_push(p, entry);
     }
 }
 
@@ -521,7 +544,6 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
     // far-part context of this CTA (uniform across the CTA)
     bool f_valid = false;
     int f_type = 0, f_I = 0, f_J = 0, f_pos = 0, f_nfar = 0, f_task = 0;
-    unsigned long long idle_spins = 0;
     unsigned popped = 0u;          // ready-ring entry taken while a far part was running (uniform)
     Acc acc;
     acc.zero();
@@ -540,18 +562,28 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             if (!s_flag) break;
             const int q = s_task[1], I = s_task[2], J = s_task[3];
             sweep_quadrant(I, J, q, smem, p, max_abs_e);
-            if (tid == 0) {
-                __threadfence();
+            // arrivals at everything this quadrant feeds, one per thread (each is a dependent global
+            // atomic round trip); sweep_quadrant ended with a barrier, so each arriving thread's fence
+            // covers the whole CTA's results
+            if (tid < 8) {
                 const int qi = q >> 1, qj = q & 1;
-                if (q == 0) { quadrant_arrive(p, I, J, 1); quadrant_arrive(p, I, J, 2); }
-                else if (q != 3) quadrant_arrive(p, I, J, 3);
-                if (I + 1 < p.ntm) { quadrant_arrive(p, I + 1, J, qj); quadrant_arrive(p, I + 1, J, 2 + qj); }
-                if (J + 1 < p.ntn) { quadrant_arrive(p, I, J + 1, 2 * qi); quadrant_arrive(p, I, J + 1, 2 * qi + 1); }
-                unsigned done = atomicAdd(p.quad_done + (long)I * p.ntn + J, 1u);
-                if (done == 3u) {          // tile swept: far parts that list it as a source may go on
-                    __threadfence();
-                    st_release_u32(p.flagS + (long)I * p.ntn + J, 1u);
-                    atomicAdd(p.tiles_done, 1u);
+                int aI = -1, aJ = 0, aq = 0;
+                if (tid == 0 && q == 0) { aI = I; aJ = J; aq = 1; }
+                if (tid == 1 && q == 0) { aI = I; aJ = J; aq = 2; }
+                if (tid == 0 && (q == 1 || q == 2)) { aI = I; aJ = J; aq = 3; }
+                if (tid == 2 && I + 1 < p.ntm) { aI = I + 1; aJ = J; aq = qj; }
+                if (tid == 3 && I + 1 < p.ntm) { aI = I + 1; aJ = J; aq = 2 + qj; }
+                if (tid == 4 && J + 1 < p.ntn) { aI = I; aJ = J + 1; aq = 2 * qi; }
+                if (tid == 5 && J + 1 < p.ntn) { aI = I; aJ = J + 1; aq = 2 * qi + 1; }
+                __threadfence();
+                if (aI >= 0) quadrant_arrive(p, aI, aJ, aq);
+                if (tid == 6) {
+                    unsigned done = atomicAdd(p.quad_done + (long)I * p.ntn + J, 1u);
+                    if (done == 3u) {      // tile swept: far parts that list it as a source may go on
+                        __threadfence();
+                        st_release_u32(p.flagS + (long)I * p.ntn + J, 1u);
+                        atomicAdd(p.tiles_done, 1u);
+                    }
                 }
             }
         }
@@ -571,14 +603,22 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             __syncthreads();
             if (s_task[0] >= p.ntasks) {
                 if (s_flag) break;                           // every tile is swept: done
-                if (++idle_spins > SPIN_LIMIT) {             // nothing to claim: wait for ready tasks
-                    if (tid == 0) {
-                        report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -4, (int)blockIdx.x, 0);
-                        atomicExch(p.abort, 1u);
+                // nothing left to claim: thread 0 watches the ready ring until a task shows up or the
+                // sweep is over (bounded), then the CTA goes back to A
+                if (tid == 0) {
+                    unsigned long long sp = 0;
+                    while ((int)(ld_relaxed_u32(p.q_tail) - ld_relaxed_u32(p.q_head)) <= 0) {
+                        if ((sp & 15ull) == 15ull &&
+                            (ld_relaxed_u32(p.tiles_done) >= (unsigned)ntiles || ld_relaxed_u32(p.abort) != 0u))
+                            break;
+                        if (++sp > SPIN_LIMIT) {
+                            report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -4, (int)blockIdx.x, 0);
+                            atomicExch(p.abort, 1u);
+                            break;
+                        }
+                        __nanosleep(IDLE_SLEEP_NS);
                     }
-                    break;
                 }
-                __nanosleep(200);
                 continue;
             }
             f_task = s_task[0]; f_type = s_task[1]; f_I = s_task[2]; f_J = s_task[3];
@@ -646,9 +686,9 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
         if (interrupted) continue;                            // back to A, then resume this far part
         // far part complete: announce it to the four quadrants of its tile
         __syncthreads();
-        if (tid == 0) {
+        if (tid < 4) {
             __threadfence();
-            for (int q = 0; q < 4; ++q) quadrant_arrive(p, f_I, f_J, q);
+            quadrant_arrive(p, f_I, f_J, tid);
         }
         f_valid = false;
     }
