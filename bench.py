@@ -250,6 +250,18 @@ def run_cuda(args):
         "factor_tflops": (2.0 * (m ** 3 + n ** 3) * (1.0 / 2 + 1.0 / 3 + 2.0 / 3)) / (factor_ms * 1e-3) / 1e12,
         "per_step_ms": per_step,
     }
+    if args.fp32:
+        # the optional fp32 mode is judged against the fp64 sweep of the same inputs
+        ws64 = torch.empty(g.gptq2d_round_workspace_bytes(m, n, g.FP64), dtype=torch.uint8, device="cuda")
+        Z64, _, _, info64 = g.gptq2d_round(dX, L, U, precision=g.FP64, workspace=ws64)
+        torch.cuda.synchronize()
+        g.check_info(info64)
+        o32 = float(g.gptq2d_objective(dX, Z, dA, dB).cpu()[0])
+        o64 = float(g.gptq2d_objective(dX, Z64, dA, dB).cpu()[0])
+        out["fp32_mode"] = {"z_mismatch_fraction": float((Z != Z64).double().mean().item()),
+                            "objective_fp32": o32, "objective_fp64": o64, "relative_objective_gap": (o32 - o64) / o64}
+        out["roofline"]["kernel"] = "round_untiled_kernel<float>"
+        out["roofline"]["bound"] = "hbm"
     if not args.no_cpu:
         out["cpu_baseline"], out["cpu_gptq2d"] = cpu_baseline(X, A, B, budget_s=args.cpu_seconds)
     print(json.dumps(out))
