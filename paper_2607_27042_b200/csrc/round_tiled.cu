@@ -166,33 +166,39 @@ __device__ __forceinline__ void cross_gemm(double *G, long ld, const double *As,
     quad_add_to(G, ld, acc, true);
 }
 
-// One 8 x 8 target block (pb, qb) of the quadrant receives the feedback of leaf-wave `lw`:
-// the downward push of leaf (lw - qb, qb) through L and the rightward push of leaf
-// (pb, lw - pb) through U, as m8n8k4 products on the warp's fragments.  Warp-uniform.
-__device__ __forceinline__ void block_feedback(double *Ys, double *Cs, const double *Ls, const double *Us, int lw,
-                                               int pb, int qb, int g, int t) {
-    const int asrc = lw - qb, bsrc = lw - pb;
-    const bool down = asrc >= 0 && asrc < pb, right = bsrc >= 0 && bsrc < qb;
-    if (!down && !right) return;
-    double *yp = Ys + (pb * 8 + g) * QLD + qb * 8 + t * 2;
-    double2 yv = *reinterpret_cast<double2 *>(yp);
-    if (down) {
-        double p0 = 0.0, p1 = 0.0;
-        dmma_m8n8k4(p0, p1, Ls[(pb * 8 + g) * QLD + asrc * 8 + t], Ys[(asrc * 8 + t) * QLD + qb * 8 + g]);
-        dmma_m8n8k4(p0, p1, Ls[(pb * 8 + g) * QLD + asrc * 8 + 4 + t], Ys[(asrc * 8 + 4 + t) * QLD + qb * 8 + g]);
-        double *cp = Cs + (pb * 8 + g) * QLD + qb * 8 + t * 2;
-        double2 cv = *reinterpret_cast<double2 *>(cp);
-        cv.x += p0;
-        cv.y += p1;
-        *reinterpret_cast<double2 *>(cp) = cv;
-        yv.x += p0;
-        yv.y += p1;
+// Leaf (a, b) of the quadrant collects, right before it is swept, all the feedback it is due from
+// the leaves already swept (left-looking): the downward pushes of the leaves above it through L,
+//     P = sum_{a' < a} L[a, a'] E[a', b]       (folded into C and pushed into Y)
+// and the rightward pushes of the leaves to its left through U,
+//     R = sum_{b' < b} C[a, b'] U[b', b]       (pushed into Y),
+// as m8n8k4 products on the warp's fragments (two independent accumulator chains each), then
+// Y += P + R, C += P in place.  E of a swept leaf lives where its Y was, its final C where its C
+// was.  Warp-uniform; all leaves of one leaf-wave do the same amount of work (a + b = lw).
+__device__ __forceinline__ void leaf_pull(double *Ys, double *Cs, const double *Ls, const double *Us, int a, int b,
+                                          int g, int t) {
+    double p0 = 0.0, p1 = 0.0, p2 = 0.0, p3 = 0.0, r0 = 0.0, r1 = 0.0, r2 = 0.0, r3 = 0.0;
+    const double *La = Ls + (a * 8 + g) * QLD + t;           // A fragments: row a*8+g, k = t (+4)
+    const double *Eb = Ys + t * QLD + b * 8 + g;             // B fragments: k = t (+4), col b*8+g
+#pragma unroll 2
+    for (int ap = 0; ap < a; ++ap) {
+        dmma_m8n8k4(p0, p1, La[ap * 8], Eb[(ap * 8) * QLD]);
+        dmma_m8n8k4(p2, p3, La[ap * 8 + 4], Eb[(ap * 8 + 4) * QLD]);
     }
-    if (right) {
-        dmma_m8n8k4(yv.x, yv.y, Cs[(pb * 8 + g) * QLD + bsrc * 8 + t], Us[(bsrc * 8 + t) * QLD + qb * 8 + g]);
-        dmma_m8n8k4(yv.x, yv.y, Cs[(pb * 8 + g) * QLD + bsrc * 8 + 4 + t], Us[(bsrc * 8 + 4 + t) * QLD + qb * 8 + g]);
+    const double *Ca = Cs + (a * 8 + g) * QLD + t;
+    const double *Ub = Us + t * QLD + b * 8 + g;
+#pragma unroll 2
+    for (int bp = 0; bp < b; ++bp) {
+        dmma_m8n8k4(r0, r1, Ca[bp * 8], Ub[(bp * 8) * QLD]);
+        dmma_m8n8k4(r2, r3, Ca[bp * 8 + 4], Ub[(bp * 8 + 4) * QLD]);
     }
+    p0 += p2; p1 += p3;
+    double *yp = Ys + (a * 8 + g) * QLD + b * 8 + t * 2;
+    double *cp = Cs + (a * 8 + g) * QLD + b * 8 + t * 2;
+    double2 yv = *reinterpret_cast<double2 *>(yp), cv = *reinterpret_cast<double2 *>(cp);
+    cv.x += p0; cv.y += p1;
+    yv.x += p0 + (r0 + r2); yv.y += p1 + (r1 + r3);
     *reinterpret_cast<double2 *>(yp) = yv;
+    *reinterpret_cast<double2 *>(cp) = cv;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -204,12 +210,9 @@ __device__ __forceinline__ void block_feedback(double *Ys, double *Cs, const dou
 //   Zs: out rounded integers
 // row0/col0: global coordinates of the quadrant (for masking the status checks).
 //
-// Leaf-wave lw (leaves (a, lw - a)) runs in two barrier-separated parts:
-//   part 1: each leaf is swept by one warp (phase A); meanwhile every warp applies the feedback
-//           of the PREVIOUS leaf-wave to the blocks of its block row that lie two or more
-//           leaf-waves ahead (interleaved with the sweep steps, which are latency bound);
-//   part 2: every warp applies the feedback of THIS leaf-wave to the one block of its block
-//           row that belongs to the next leaf-wave.
+// Leaf-wave lw (leaves (a, lw - a), one per warp): every leaf first pulls the feedback of the
+// leaves swept before it (leaf_pull), then runs the 15 anti-diagonal steps on its 8 x 8 entries.
+// One CTA barrier per leaf-wave.
 __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const double *Ls, const double *Us, int *Zs,
                                                double *tabL, double *tabU, int row0, int col0,
                                                const TiledKernelParams &p, double &max_abs_e) {
@@ -231,10 +234,11 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
 
     for (int lw = 0; lw < 15; ++lw) {
         __syncthreads();
-        // ---------------- part 1
         const int a_lo = max(0, lw - 7), a_hi = min(7, lw);
         const int a = a_lo + warp, b = lw - a;
         if (a <= a_hi) {
+            leaf_pull(Ys, Cs, Ls, Us, a, b, g, t);
+            __syncwarp();
             // Phase A.  Lane l owns entries (i0, j) and (i0 + 4, j) of the 8 x 8 leaf, i0 = l & 3,
             // j = l >> 2.  At step s the lane whose entry lies on anti-diagonal s rounds it and posts
             // the error (by column) and the final C value (by row) to a 16-double per-warp exchange
@@ -277,7 +281,6 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
                     }
                 }
                 __syncwarp();
-                if (s < 8 && warp + s > lw) block_feedback(Ys, Cs, Ls, Us, lw - 1, warp, s, g, t);   // far feedback
                 const double ed = ex[j], cr0 = ex[8 + i0], cr1 = ex[12 + i0];
                 const double l0 = tl0[s], l1 = tl1[s], u0 = tu0[s], u1 = tu1[s];
                 y0 = fma(l0, ed, y0); c0 = fma(l0, ed, c0); y0 = fma(cr0, u0, y0);   // fold, push down, push right
@@ -290,20 +293,9 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
                 if (row0 + a * 8 + i0 < p.m) max_abs_e = fmax(max_abs_e, fabs(y0));
                 if (row0 + a * 8 + i0 + 4 < p.m) max_abs_e = fmax(max_abs_e, fabs(y1));
             }
-        } else if (lw > 0) {
-            // no leaf for this warp in this leaf-wave: only the far feedback of the previous one
-#pragma unroll
-            for (int qb = 0; qb < 8; ++qb)
-                if (warp + qb > lw) block_feedback(Ys, Cs, Ls, Us, lw - 1, warp, qb, g, t);
-        }
-        __syncthreads();
-        if (lw == 14) break;
-        // ---------------- part 2: feedback of this leaf-wave to the next one
-        {
-            const int qb = lw + 1 - warp;
-            if (qb >= 0 && qb < 8) block_feedback(Ys, Cs, Ls, Us, lw, warp, qb, g, t);
         }
     }
+    __syncthreads();
     // status: the earliest (in sweep order) unrepresentable value of the quadrant, if any
     if (badkey != ~0ull) atomicMin(&s_badkey, badkey);
     __syncthreads();
