@@ -176,6 +176,25 @@ def test_mid_size_against_nested_oracle_and_certificate(g, name, make):
     assert torch.equal(Z, Z2) and torch.equal(Z, Z3)
 
 
+# ------------------------------------------------------------------ thin shapes: one row / one column of tiles
+@pytest.mark.parametrize("m,n,seed", [(3, 1500, 0), (1500, 3, 1), (130, 1100, 2), (1100, 130, 3), (1, 700, 4), (700, 1, 5)])
+def test_thin_shapes_against_nested_oracle(g, m, n, seed):
+    for t in range(6):
+        X, A, B = W.gaussian_like(m, n, seed + 1000 * t, samples=2 * max(m, n))
+        L, U, _, _ = O.feedback_factors(A, B)
+        ref = cref.nested(X, L, U)
+        if ref["margin"] >= MARGIN:
+            break
+    else:
+        pytest.fail("no certified seed")
+    Z, E, mm = gpu_round(g, X, L, U)
+    assert np.array_equal(Z, ref["Z"])
+    assert np.max(np.abs(E - ref["E"])) < 1e-8
+    # repeated runs must be bit-identical (the schedule differs from run to run, the arithmetic must not)
+    Z2, E2, _ = gpu_round(g, X, L, U)
+    assert np.array_equal(Z, Z2) and np.array_equal(E, E2)
+
+
 # ------------------------------------------------------------------ invariances on the GPU path
 def test_transpose_and_translation_invariance(g):
     X, A, B = W.general_bases(150, 70, 12)
