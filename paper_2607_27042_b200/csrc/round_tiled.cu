@@ -436,19 +436,24 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
 }
 
 // ---------------------------------------------------------------------------------------------
+// Far parts in claim order: wave by wave (I + J ascending); inside a wave the longest contractions
+// first (the Cd part of tile (I, J) has I - 1 chunks, the Rt part J - 1), so that a wave's far parts
+// finish close together instead of the long ones trailing.
 __device__ __forceinline__ void decode_task(int task, int ntm, int ntn, int &type, int &I, int &J) {
-    type = task & 1;
-    int tt = task >> 1;
+    int tt = task;
     for (int w = 0; w < ntm + ntn - 1; ++w) {
         int lo = max(0, w - ntn + 1), hi = min(ntm - 1, w);
-        int cnt = hi - lo + 1;
+        int cnt = 2 * (hi - lo + 1);
         if (tt < cnt) {
-            I = lo + tt;
+            const int k = tt >> 1;
+            type = tt & 1;
+            I = type == 0 ? hi - k : lo + k;        // Cd parts by descending I, Rt parts by descending J
             J = w - I;
             return;
         }
         tt -= cnt;
     }
+    type = 0;
     I = J = 0;
 }
 
