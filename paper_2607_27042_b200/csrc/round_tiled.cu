@@ -528,166 +528,175 @@ __device__ __forceinline__ void quadrant_arrive(const TiledKernelParams &p, int 
     }
 }
 
+constexpr int FAR_CTX = 2;       // far parts a CTA may hold at once (one live in registers, the others parked)
+
 __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKernelParams p) {
     extern __shared__ __align__(16) double smem[];
     __shared__ int s_task[4];
-    __shared__ int s_flag;
+    __shared__ int s_ctx[FAR_CTX][6];      // far-part contexts, oldest first: type, I, J, pos, nfar, task
+    __shared__ int s_nctx, s_pick, s_state;
+    __shared__ unsigned s_pop;
     __shared__ double s_red[TILED_THREADS / 32];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int wm = warp >> 2, wn = warp & 3, g = lane >> 2, t = lane & 3;
     const int ntiles = p.ntm * p.ntn;
     double max_abs_e = 0.0;
-
-    // far-part context of this CTA (uniform across the CTA)
-    bool f_valid = false;
-    int f_type = 0, f_I = 0, f_J = 0, f_pos = 0, f_nfar = 0, f_task = 0;
-    unsigned popped = 0u;          // ready-ring entry taken while a far part was running (uniform)
+    int cur = -1;                  // context whose accumulator is live in registers (uniform), -1: none
+    unsigned long long spins = 0;
     Acc acc;
     acc.zero();
+    if (tid == 0) s_nctx = 0;
+
+    auto tile_region = [&](int k) {
+        return (s_ctx[k][0] == 0 ? p.Cbuf : p.Ebuf) + (long)s_ctx[k][1] * T * p.np + (long)s_ctx[k][2] * T;
+    };
 
     for (;;) {
-        // ================= A: quadrant tasks from the ready ring.  Never waits.
-        for (;;) {
-            __syncthreads();
-            if (tid == 0) {
-                unsigned e = popped ? popped : ready_pop(p);
-                s_flag = e != 0u;
-                s_task[1] = (int)((e >> 29) & 3u); s_task[2] = (int)((e >> 15) & 0x3fffu); s_task[3] = (int)(e & 0x7fffu);
-            }
-            __syncthreads();
-            popped = 0u;
-            if (!s_flag) break;
-            const int q = s_task[1], I = s_task[2], J = s_task[3];
-            sweep_quadrant(I, J, q, smem, p, max_abs_e);
-            // arrivals at everything this quadrant feeds, one per thread (each is a dependent global
-            // atomic round trip); sweep_quadrant ended with a barrier, so each arriving thread's fence
-            // covers the whole CTA's results
-            if (tid < 8) {
-                const int qi = q >> 1, qj = q & 1;
-                int aI = -1, aJ = 0, aq = 0;
-                if (tid == 0 && q == 0) { aI = I; aJ = J; aq = 1; }
-                if (tid == 1 && q == 0) { aI = I; aJ = J; aq = 2; }
-                if (tid == 0 && (q == 1 || q == 2)) { aI = I; aJ = J; aq = 3; }
-                if (tid == 2 && I + 1 < p.ntm) { aI = I + 1; aJ = J; aq = qj; }
-                if (tid == 3 && I + 1 < p.ntm) { aI = I + 1; aJ = J; aq = 2 + qj; }
-                if (tid == 4 && J + 1 < p.ntn) { aI = I; aJ = J + 1; aq = 2 * qi; }
-                if (tid == 5 && J + 1 < p.ntn) { aI = I; aJ = J + 1; aq = 2 * qi + 1; }
-                __threadfence();
-                if (aI >= 0) quadrant_arrive(p, aI, aJ, aq);
-                if (tid == 6) {
-                    unsigned done = atomicAdd(p.quad_done + (long)I * p.ntn + J, 1u);
-                    if (done == 3u) {      // tile swept: far parts that list it as a source may go on
-                        __threadfence();
-                        st_release_u32(p.flagS + (long)I * p.ntn + J, 1u);
-                        atomicAdd(p.tiles_done, 1u);
+        // ---- thread 0 looks for work: a ready quadrant task first, else the oldest far part that can
+        // go on, else (room and tasks left) a new far part.  s_state: 0 run far part s_pick, 1 serve the
+        // ring, 2 nothing to do right now, 3 all tiles swept, 4 abort.
+        __syncthreads();
+        if (tid == 0) {
+            int state = 2, pick = -1;
+            unsigned e = 0u;
+            if (ld_relaxed_u32(p.abort) != 0u) state = 4;
+            else if ((e = ready_pop(p)) != 0u) state = 1;
+            else {
+                int n = s_nctx;
+                for (int k = 0; k < n && pick < 0; ++k) {
+                    const int ty = s_ctx[k][0], pos = s_ctx[k][3];
+                    const unsigned *fl = ty == 0 ? p.flagS + (long)pos * p.ntn + s_ctx[k][2]
+                                                 : p.flagS + (long)s_ctx[k][1] * p.ntn + pos;
+                    if (pos >= s_ctx[k][4] || ld_acquire_u32(fl) != 0u) pick = k;
+                }
+                if (pick < 0 && n < FAR_CTX && ld_relaxed_u32(p.counter) < (unsigned)p.ntasks) {
+                    int task = (int)atomicAdd(p.counter, 1u);
+                    if (task < p.ntasks) {
+                        int ty, fi, fj;
+                        decode_task(task, p.ntm, p.ntn, ty, fi, fj);
+                        s_ctx[n][0] = ty; s_ctx[n][1] = fi; s_ctx[n][2] = fj; s_ctx[n][3] = 0;
+                        s_ctx[n][4] = max(0, (ty == 0 ? fi : fj) - 1); s_ctx[n][5] = task;
+                        s_nctx = n + 1;
+                        const unsigned *fl = ty == 0 ? p.flagS + fj : p.flagS + (long)fi * p.ntn;
+                        if (s_ctx[n][4] == 0 || ld_acquire_u32(fl) != 0u) pick = n;
                     }
                 }
+                if (pick >= 0) state = 0;
+                else if (s_nctx == 0 && ld_relaxed_u32(p.counter) >= (unsigned)p.ntasks &&
+                         ld_relaxed_u32(p.tiles_done) >= (unsigned)ntiles) state = 3;
             }
+            s_state = state; s_pick = pick; s_pop = e;
         }
-        if (ld_relaxed_u32(p.abort) != 0u) break;
-
-        // ================= B: far part of a bulk contraction: every source tile except the adjacent one.
-        if (!f_valid) {
-            __syncthreads();
-            if (tid == 0) {
-                int task = p.ntasks;
-                if (ld_relaxed_u32(p.counter) < (unsigned)p.ntasks) task = (int)atomicAdd(p.counter, 1u);
-                int ty = 0, fi = 0, fj = 0;
-                if (task < p.ntasks) decode_task(task, p.ntm, p.ntn, ty, fi, fj);
-                s_task[0] = task; s_task[1] = ty; s_task[2] = fi; s_task[3] = fj;
-                s_flag = (ld_relaxed_u32(p.tiles_done) >= (unsigned)ntiles) ? 1 : 0;
-            }
-            __syncthreads();
-            if (s_task[0] >= p.ntasks) {
-                if (s_flag) break;                           // every tile is swept: done
-                // nothing left to claim: thread 0 watches the ready ring until a task shows up or the
-                // sweep is over (bounded), then the CTA goes back to A
+        __syncthreads();
+        const int state = s_state;
+        if (state >= 3) break;
+        if (state == 2) {
+            if (++spins > SPIN_LIMIT) {
                 if (tid == 0) {
-                    unsigned long long sp = 0;
-                    while ((int)(ld_relaxed_u32(p.q_tail) - ld_relaxed_u32(p.q_head)) <= 0) {
-                        if ((sp & 15ull) == 15ull &&
-                            (ld_relaxed_u32(p.tiles_done) >= (unsigned)ntiles || ld_relaxed_u32(p.abort) != 0u))
-                            break;
-                        if (++sp > SPIN_LIMIT) {
-                            report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -4, (int)blockIdx.x, 0);
-                            atomicExch(p.abort, 1u);
-                            break;
+                    report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -4, (int)blockIdx.x, s_nctx);
+                    atomicExch(p.abort, 1u);
+                }
+                break;
+            }
+            __nanosleep(s_nctx == 0 ? IDLE_SLEEP_NS : 100);
+            continue;
+        }
+        spins = 0;
+
+        if (state == 1) {
+            // ================= A: quadrant tasks from the ready ring.  Never waits.  The live far part,
+            // if any, is parked first (the quadrant task needs the shared memory and the registers).
+            if (cur >= 0) {
+                if (s_ctx[cur][3] > 0) store_acc(acc, tile_region(cur), p.np, wm, wn, g, t);
+                cur = -1;
+            }
+            unsigned e = s_pop;
+            while (e != 0u) {
+                const int q = (int)((e >> 29) & 3u), I = (int)((e >> 15) & 0x3fffu), J = (int)(e & 0x7fffu);
+                sweep_quadrant(I, J, q, smem, p, max_abs_e);
+                // arrivals at everything this quadrant feeds, one per thread (each is a dependent global
+                // atomic round trip); sweep_quadrant ended with a barrier, so each arriving thread's fence
+                // covers the whole CTA's results
+                if (tid < 8) {
+                    const int qi = q >> 1, qj = q & 1;
+                    int aI = -1, aJ = 0, aq = 0;
+                    if (tid == 0 && q == 0) { aI = I; aJ = J; aq = 1; }
+                    if (tid == 1 && q == 0) { aI = I; aJ = J; aq = 2; }
+                    if (tid == 0 && (q == 1 || q == 2)) { aI = I; aJ = J; aq = 3; }
+                    if (tid == 2 && I + 1 < p.ntm) { aI = I + 1; aJ = J; aq = qj; }
+                    if (tid == 3 && I + 1 < p.ntm) { aI = I + 1; aJ = J; aq = 2 + qj; }
+                    if (tid == 4 && J + 1 < p.ntn) { aI = I; aJ = J + 1; aq = 2 * qi; }
+                    if (tid == 5 && J + 1 < p.ntn) { aI = I; aJ = J + 1; aq = 2 * qi + 1; }
+                    __threadfence();
+                    if (aI >= 0) quadrant_arrive(p, aI, aJ, aq);
+                    if (tid == 6) {
+                        unsigned done = atomicAdd(p.quad_done + (long)I * p.ntn + J, 1u);
+                        if (done == 3u) {      // tile swept: far parts that list it as a source may go on
+                            __threadfence();
+                            st_release_u32(p.flagS + (long)I * p.ntn + J, 1u);
+                            atomicAdd(p.tiles_done, 1u);
                         }
-                        __nanosleep(IDLE_SLEEP_NS);
                     }
                 }
-                continue;
+                __syncthreads();
+                if (tid == 0) s_pop = ready_pop(p);
+                __syncthreads();
+                e = s_pop;
             }
-            f_task = s_task[0]; f_type = s_task[1]; f_I = s_task[2]; f_J = s_task[3];
-            f_pos = 0;
-            f_nfar = max(0, (f_type == 0 ? f_I : f_J) - 1);
-            f_valid = true;
-            acc.zero();
-        } else {
-            // coming back from quadrant tasks: un-park the partial sum
-            if (f_pos > 0)
-                load_acc(acc, (f_type == 0 ? p.Cbuf : p.Ebuf) + (long)f_I * T * p.np + (long)f_J * T, p.np, wm, wn, g, t);
-            else
-                acc.zero();
+            continue;
         }
-        bool interrupted = false;
-        {
+
+        // ================= B: far part s_pick (every source tile of the contraction except the adjacent one)
+        const int k = s_pick;
+        if (k != cur) {
+            if (cur >= 0 && s_ctx[cur][3] > 0) store_acc(acc, tile_region(cur), p.np, wm, wn, g, t);
+            if (s_ctx[k][3] > 0) load_acc(acc, tile_region(k), p.np, wm, wn, g, t);
+            else acc.zero();
+            cur = k;
+        }
+        const int f_type = s_ctx[k][0], f_I = s_ctx[k][1], f_J = s_ctx[k][2], f_pos = s_ctx[k][3], f_nfar = s_ctx[k][4];
+        int new_pos = f_pos;
+        if (f_pos < f_nfar) {
             const unsigned *flags = f_type == 0 ? p.flagS + f_J : p.flagS + (long)f_I * p.ntn;
             const long fstride = f_type == 0 ? p.ntn : 1;
-            Operand A, B;
+            // how many source tiles from f_pos on are swept already (the first one is)
+            __syncthreads();
+            if (tid == 0) s_task[0] = f_nfar;
+            __syncthreads();
+            for (int idx = f_pos + tid; idx < f_nfar; idx += blockDim.x)
+                if (ld_acquire_u32(flags + (long)idx * fstride) == 0u) atomicMin(&s_task[0], idx);
+            __syncthreads();
+            const int upto = min(s_task[0], f_pos + FAR_RUN_CHUNKS);
+            Operand a, b;
             if (f_type == 0) {
-                A.ptr = p.L + (long)f_I * T * p.ldl; A.ld = p.ldl; A.mn_valid = min(T, p.m - f_I * T); A.aligned16 = p.l_al16;
-                B.ptr = p.Ebuf + (long)f_J * T; B.ld = p.np; B.mn_valid = T; B.aligned16 = true;
+                a.ptr = p.L + (long)f_I * T * p.ldl + (long)f_pos * T; a.ld = p.ldl; a.mn_valid = min(T, p.m - f_I * T); a.aligned16 = p.l_al16;
+                b.ptr = p.Ebuf + (long)f_J * T + (long)f_pos * T * p.np; b.ld = p.np; b.mn_valid = T; b.aligned16 = true;
             } else {
-                A.ptr = p.Cbuf + (long)f_I * T * p.np; A.ld = p.np; A.mn_valid = T; A.aligned16 = true;
-                B.ptr = p.U + (long)f_J * T; B.ld = p.ldu; B.mn_valid = min(T, p.n - f_J * T); B.aligned16 = p.u_al16;
+                a.ptr = p.Cbuf + (long)f_I * T * p.np + (long)f_pos * T; a.ld = p.np; a.mn_valid = T; a.aligned16 = true;
+                b.ptr = p.U + (long)f_J * T + (long)f_pos * T * p.ldu; b.ld = p.ldu; b.mn_valid = min(T, p.n - f_J * T); b.aligned16 = p.u_al16;
             }
-            unsigned long long spins = 0;
-            while (f_pos < f_nfar) {
-                // how many source tiles from f_pos on are swept already; is there a ready task to take over
-                __syncthreads();
-                if (tid == 0) { s_task[0] = f_nfar; s_task[1] = (int)ready_pop(p); }
-                __syncthreads();
-                for (int idx = f_pos + tid; idx < f_nfar; idx += blockDim.x)
-                    if (ld_acquire_u32(flags + (long)idx * fstride) == 0u) atomicMin(&s_task[0], idx);
-                __syncthreads();
-                const int upto_ready = s_task[0];
-                popped = (unsigned)s_task[1];
-                const bool work = popped != 0u;
-                if (work) { interrupted = true; break; }       // park and serve the critical path first
-                if (upto_ready == f_pos) {                   // next source not swept yet
-                    if (++spins > SPIN_LIMIT || ld_relaxed_u32(p.abort) != 0u) {
-                        if (tid == 0) {
-                            report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, f_task, f_pos, (int)blockIdx.x);
-                            atomicExch(p.abort, 1u);
-                        }
-                        interrupted = true;
-                        break;
-                    }
-                    __nanosleep(100);
-                    continue;
-                }
-                const int upto = min(upto_ready, f_pos + FAR_RUN_CHUNKS);
-                Operand a = A, b = B;
-                a.ptr = A.ptr + (long)f_pos * T;               // k offset along the contiguous index
-                b.ptr = B.ptr + (long)f_pos * T * B.ld;        // k offset along rows
-                gemm_tile<true, false, BULK_NSTAGE>(acc, smem, a, b, (upto - f_pos) * T);
-                f_pos = upto;
+            gemm_tile<true, false, BULK_NSTAGE>(acc, smem, a, b, (upto - f_pos) * T);
+            new_pos = upto;
+        }
+        if (new_pos >= f_nfar) {
+            // far part complete: park the sum (zeros included: the quadrant tasks start from it) and
+            // announce it to the four quadrants of its tile; drop the context
+            store_acc(acc, tile_region(k), p.np, wm, wn, g, t);
+            __syncthreads();
+            if (tid < 4) {
+                __threadfence();
+                quadrant_arrive(p, f_I, f_J, tid);
             }
+            if (tid == 0) {
+                const int n = s_nctx;
+                for (int c = k; c + 1 < n; ++c)
+                    for (int f = 0; f < 6; ++f) s_ctx[c][f] = s_ctx[c + 1][f];
+                s_nctx = n - 1;
+            }
+            cur = -1;
+        } else if (tid == 0) {
+            s_ctx[k][3] = new_pos;
         }
-        if (ld_relaxed_u32(p.abort) != 0u) break;
-        // park the partial sum in the tile's own region (Cd in Cbuf, Rt in Ebuf); a finished far part
-        // always writes it, zeros included, because the quadrant tasks start from it
-        if (f_pos > 0 || !interrupted)
-            store_acc(acc, (f_type == 0 ? p.Cbuf : p.Ebuf) + (long)f_I * T * p.np + (long)f_J * T, p.np, wm, wn, g, t);
-        if (interrupted) continue;                            // back to A, then resume this far part
-        // far part complete: announce it to the four quadrants of its tile
-        __syncthreads();
-        if (tid < 4) {
-            __threadfence();
-            quadrant_arrive(p, f_I, f_J, tid);
-        }
-        f_valid = false;
     }
 
     for (int o = 16; o > 0; o >>= 1) max_abs_e = fmax(max_abs_e, __shfl_xor_sync(0xffffffffu, max_abs_e, o));
