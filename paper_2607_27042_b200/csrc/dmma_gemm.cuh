@@ -180,31 +180,33 @@ __device__ __forceinline__ void gemm_mainloop(Acc &acc, double *smem, const Oper
     __syncthreads();
 }
 
-// Per-thread copy plan for one operand: 4 chunks of 16 bytes per slab, pointers advance by a
-// constant per slab.  Valid only for tiles that are fully in range and 16-byte aligned.
+// Per-thread copy plan for one operand: BK/4 chunks of 16 bytes per slab, one base pointer and
+// constant strides (between chunks and between slabs).  Valid only for tiles that are fully in range and 16-byte aligned.
 template <bool KCONTIG>
 struct FastCopy {
-    const double *src[4];
-    int dst[4];
-    long step;
+    // chunk i of this thread: source src0 + i * sstep (+ slab * step), destination dst0 + i * dstep
+    const double *src0;
+    long sstep, step;
+    int dst0, dstep;
     __device__ __forceinline__ void init(const Operand &op, int tid) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            int c = tid + i * GEMM_THREADS;
-            if (KCONTIG) {
-                int r = c >> 3, kk = (c & 7) * 2;
-                src[i] = op.ptr + (long)r * op.ld + kk;
-                dst[i] = r * LDK + kk;
-            } else {
-                int kr = c >> 6, cc = (c & 63) * 2;
-                src[i] = op.ptr + (long)kr * op.ld + cc;
-                dst[i] = kr * LDN + cc;
-            }
+        if (KCONTIG) {
+            int r = tid / (BK / 2), kk = (tid % (BK / 2)) * 2;
+            src0 = op.ptr + (long)r * op.ld + kk;
+            dst0 = r * LDK + kk;
+            sstep = (long)(GEMM_THREADS / (BK / 2)) * op.ld;
+            dstep = (GEMM_THREADS / (BK / 2)) * LDK;
+            step = BK;
+        } else {
+            int kr = tid >> 6, cc = (tid & 63) * 2;
+            src0 = op.ptr + (long)kr * op.ld + cc;
+            dst0 = kr * LDN + cc;
+            sstep = (long)(GEMM_THREADS / 64) * op.ld;
+            dstep = (GEMM_THREADS / 64) * LDN;
+            step = (long)BK * op.ld;
         }
-        step = KCONTIG ? (long)BK : (long)BK * op.ld;
     }
     __device__ __forceinline__ void issue(double *smem, int i, long slab) const {
-        cp_async16(smem + dst[i], src[i] + slab * step, 16);
+        cp_async16(smem + dst0 + i * dstep, src0 + i * sstep + slab * step, 16);
     }
 };
 
@@ -228,7 +230,7 @@ __device__ __forceinline__ void gemm_mainloop_fast(Acc &acc, double *smem, const
         if (s < nk) {
             double *st = smem + s * SL::STAGE_DOUBLES;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) { ca.issue(st, i, s); cb.issue(st + SL::A_DOUBLES, i, s); }
+            for (int i = 0; i < BK / 4; ++i) { ca.issue(st, i, s); cb.issue(st + SL::A_DOUBLES, i, s); }
         }
         cp_async_commit();
     }
