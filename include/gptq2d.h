@@ -45,7 +45,8 @@ typedef enum {
     GPTQ2D_ERR_NONFINITE = 6,          /* device: NaN/Inf met while rounding; info[1] = row, info[2] = col */
     GPTQ2D_ERR_INT_OVERFLOW = 7,       /* device: |corrected value| >= 2^31; info[1] = row, info[2] = col  */
     GPTQ2D_ERR_DEVICE_TIMEOUT = 8,     /* device: a bounded wait gave up; info[1] = where it waited     */
-    GPTQ2D_ERR_TOO_LARGE = 9           /* gptq2d_round_static: m or n beyond GPTQ2D_STATIC_MAX_DIM      */
+    GPTQ2D_ERR_TOO_LARGE = 9           /* gptq2d_round_static: m or n beyond GPTQ2D_STATIC_MAX_DIM;
+                                          gptq2d_round_batched: beyond its count / dimension limits     */
 } gptq2d_status_t;
 
 typedef enum {
@@ -109,6 +110,37 @@ int gptq2d_round_host(int m, int n,
                       int32_t *hZ, double *hE, double *hmin_margin,
                       int precision,
                       void *workspace, size_t workspace_bytes, int *hinfo, void *stream);
+
+/* ---- many independent sweeps in one launch (Section 6: A and B "may come from factors of
+ * Kronecker Hessian approximations", i.e. one (X; A, B) triple per layer; the paper sweeps one
+ * matrix, Algorithm 3, and this call runs that same sweep on `count` matrices at once) ----
+ * A single small or thin matrix cannot fill the GPU: its anti-diagonal dependency chain has
+ * m + n - 1 stages (Section 2, Fig. 1) and few entries per stage.  Here the fp64 tiled sweeps of
+ * all matrices share one persistent kernel, so the tiles that are ready in ANY matrix keep the SMs
+ * busy.  Each matrix gets exactly the Z (and E, min_margin) that gptq2d_round with GPTQ2D_FP64
+ * gives it alone; shapes may differ from matrix to matrix.
+ *   problems:   HOST array of `count` descriptors (device pointers inside, same rules as
+ *               gptq2d_round); read before the call returns, the caller may free it afterwards.
+ *   min_margin: optional DEVICE array of `count` doubles.
+ *   info:       device int[4] shared by all matrices; for NONFINITE / INT_OVERFLOW info[3] is the
+ *               index of the matrix (first error wins; the other matrices are still swept).
+ *   Limits: count <= GPTQ2D_BATCH_MAX_COUNT, every m, n <= GPTQ2D_BATCH_MAX_DIM
+ *           (else GPTQ2D_ERR_TOO_LARGE).  Output regions of different matrices must not overlap.
+ */
+typedef struct gptq2d_problem {
+    int m, n;
+    const double *X; long ldx;
+    const double *L; long ldl;
+    const double *U; long ldu;
+    int32_t *Z; long ldz;
+    double *E; long lde;       /* optional (NULL ok) */
+} gptq2d_problem_t;
+#define GPTQ2D_BATCH_MAX_COUNT 8192
+#define GPTQ2D_BATCH_MAX_DIM 32768
+size_t gptq2d_round_batched_workspace_bytes(int count, const gptq2d_problem_t *problems);
+int gptq2d_round_batched(int count, const gptq2d_problem_t *problems,
+                         double *min_margin,
+                         void *workspace, size_t workspace_bytes, int *info, void *stream);
 
 /* ---- the sweep without any allocation (the paper has no counterpart: this is a packaging variant
  * of gptq2d_round, not a different method) ----

@@ -2,6 +2,7 @@
 #include <cuda_runtime.h>
 #include "common.cuh"
 #include "round_internal.cuh"
+#include <vector>
 
 namespace gptq2d {
 size_t factor_workspace_bytes(int m, int n);
@@ -23,6 +24,27 @@ static int check_device() {
 }
 
 static size_t pad256(size_t x) { return (x + 255) / 256 * 256; }
+
+// host descriptors of a batched call -> internal launch parameters, with the argument checks of gptq2d_round
+static int to_tiled(int count, const gptq2d_problem_t *pr, std::vector<TiledParams> &out) {
+    if (count < 1 || !pr) return GPTQ2D_ERR_INVALID_ARG;
+    if (count > GPTQ2D_BATCH_MAX_COUNT) return GPTQ2D_ERR_TOO_LARGE;
+    out.resize(count);
+    for (int b = 0; b < count; ++b) {
+        const gptq2d_problem_t &q = pr[b];
+        if (q.m < 1 || q.n < 1 || !q.X || !q.L || !q.U || !q.Z) return GPTQ2D_ERR_INVALID_ARG;
+        if (q.ldx < q.n || q.ldl < q.m || q.ldu < q.n || q.ldz < q.n || (q.E && q.lde < q.n)) return GPTQ2D_ERR_INVALID_ARG;
+        if (!aligned(q.X, 8) || !aligned(q.L, 8) || !aligned(q.U, 8) || !aligned(q.Z, 4) || !aligned(q.E, 8))
+            return GPTQ2D_ERR_INVALID_ARG;
+        if (q.m > GPTQ2D_BATCH_MAX_DIM || q.n > GPTQ2D_BATCH_MAX_DIM) return GPTQ2D_ERR_TOO_LARGE;
+        TiledParams t{};
+        t.m = q.m; t.n = q.n;
+        t.X = q.X; t.ldx = q.ldx; t.L = q.L; t.ldl = q.ldl; t.U = q.U; t.ldu = q.ldu;
+        t.Z = q.Z; t.ldz = q.ldz; t.E = q.E; t.lde = q.lde;
+        out[b] = t;
+    }
+    return GPTQ2D_OK;
+}
 }  // namespace gptq2d
 
 using namespace gptq2d;
@@ -111,6 +133,28 @@ int gptq2d_round(int m, int n, const double *X, long ldx, const double *L, long 
         if (cudaGetLastError() != cudaSuccess) return GPTQ2D_ERR_CUDA;
     }
     return GPTQ2D_OK;
+}
+
+size_t gptq2d_round_batched_workspace_bytes(int count, const gptq2d_problem_t *problems) {
+    std::vector<TiledParams> t;
+    if (to_tiled(count, problems, t) != GPTQ2D_OK) return 0;
+    return round_tiled_batched_workspace_bytes(count, t.data());
+}
+
+int gptq2d_round_batched(int count, const gptq2d_problem_t *problems, double *min_margin, void *workspace,
+                         size_t workspace_bytes, int *info, void *stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    std::vector<TiledParams> t;
+    int st = to_tiled(count, problems, t);
+    if (st != GPTQ2D_OK) return st;
+    if (!aligned(min_margin, 8)) return GPTQ2D_ERR_INVALID_ARG;
+    if (!workspace || !aligned(workspace, 256) ||
+        workspace_bytes < round_tiled_batched_workspace_bytes(count, t.data()))
+        return GPTQ2D_ERR_WORKSPACE;
+    st = check_device();
+    if (st != GPTQ2D_OK) return st;
+    if (info && cudaMemsetAsync(info, 0, 4 * sizeof(int), stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+    return launch_round_tiled_batched(count, t.data(), min_margin, info, workspace, workspace_bytes, stream);
 }
 
 size_t gptq2d_round_host_workspace_bytes(int m, int n, int precision) {

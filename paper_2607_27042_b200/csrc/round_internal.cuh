@@ -32,6 +32,12 @@ struct TiledParams {
 };
 size_t round_tiled_workspace_bytes(int m, int n);
 int launch_round_tiled(const TiledParams &p, void *ws, size_t ws_bytes, cudaStream_t stream);
+// many matrices in one launch (fp64 tiled sweep); `info` is shared, `min_margin` (optional) gets one value per matrix
+constexpr int BATCH_MAX_COUNT = 8192;     // matrix index has 13 bits in a ready-ring entry
+constexpr int BATCH_MAX_DIM = 32768;      // tile coordinates have 8 bits there
+size_t round_tiled_batched_workspace_bytes(int count, const TiledParams *problems);
+int launch_round_tiled_batched(int count, const TiledParams *problems, double *min_margin, int *info, void *ws,
+                               size_t ws_bytes, cudaStream_t stream);
 // where the max |E| scalar lives inside either workspace
 inline double *workspace_max_abs_e(void *ws) { return reinterpret_cast<double *>(static_cast<char *>(ws) + 64); }
 

@@ -33,6 +33,7 @@
 #include "common.cuh"
 #include "dmma_gemm.cuh"
 #include "round_internal.cuh"
+#include <vector>
 
 namespace gptq2d {
 
@@ -54,14 +55,22 @@ struct TiledKernelParams {
     double *Euser; long lde;
     double *Ebuf, *Cbuf;
     unsigned *counter, *abort, *q_head, *q_tail, *tiles_done;
-    unsigned *q_slots;           // [QCAP] ready continuation tasks
+    unsigned *q_slots;           // [qmask + 1] ready quadrant tasks
+    unsigned qmask;              // ring size - 1 (power of two)
     unsigned *flagS;             // [ntm*ntn] tile swept
     unsigned *quad_done;         // [ntm*ntn] swept quadrants of the tile (4 -> tile flag)
     unsigned *qdep;              // [ntm*ntn][4] arrivals each quadrant task has received
     double *max_abs_e;
     int *info;
     int l_al16, u_al16;
+    // batched launches only (one descriptor per matrix in device memory; the kernel argument then
+    // carries the shared scheduler words, the totals in ntasks / ntiles_total, and these tables)
+    int batch_index;             // -1: single-matrix launch
+    int ntiles_total;
+    const TiledKernelParams *probs;
+    const unsigned *far_tasks;   // far parts of all matrices in claim order: b << 17 | type << 16 | I << 8 | J
 };
+static_assert(sizeof(TiledKernelParams) % 8 == 0, "descriptors are copied as 8-byte words");
 
 constexpr size_t SWEEP_SMEM = (size_t)(5 * QMAT + 2 * Q * TAB_LD) * sizeof(double) + (size_t)Q * Q * sizeof(int);
 constexpr size_t BULK_SMEM = (size_t)BULK_NSTAGE * SlabLayout<true, false>::STAGE_DOUBLES * sizeof(double);
@@ -302,7 +311,7 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
     if (tid == 0 && s_badkey != ~0ull) {
         const unsigned long long k = s_badkey;
         report(p.info, ((k >> 41) & 1ull) ? GPTQ2D_ERR_INT_OVERFLOW : GPTQ2D_ERR_NONFINITE,
-               (int)((k >> 20) & 0x1fffffull), (int)(k & 0xfffffull), 0);
+               (int)((k >> 20) & 0x1fffffull), (int)(k & 0xfffffull), max(p.batch_index, 0));
     }
 }
 
@@ -481,14 +490,20 @@ __device__ __forceinline__ void load_acc(Acc &acc, const double *srcT, long np, 
         }
 }
 
-constexpr unsigned QCAP = 4096;   // global ring of ready continuation tasks (power of two)
+// Global ring of ready quadrant tasks (size a power of two).  It cannot overflow: a quadrant depends,
+// directly or through others, on the quadrant above it and on the one to its left, so the quadrants
+// of one matrix that are ready at the same time lie on an anti-chain of its 2 ntm x 2 ntn quadrant
+// grid, at most 2 min(ntm, ntn) of them; each enters the ring once.  A single matrix therefore
+// needs at most 512 slots (ntm, ntn <= 256 tiles would be 32768 rows); a batched launch sizes its
+// ring from the sum over its matrices.
+constexpr unsigned QCAP = 4096;
 constexpr int FAR_RUN_CHUNKS = 16;
 constexpr unsigned IDLE_SLEEP_NS = 400; // a far part looks at the ready queue every this many K = 128 chunks
 
 // multi-producer / multi-consumer ring in global memory; slot value 0 = empty.
 __device__ __forceinline__ void ready_push(const TiledKernelParams &p, unsigned entry) {
     unsigned t = atomicAdd(p.q_tail, 1u);
-    st_release_u32(p.q_slots + (t & (QCAP - 1)), entry | 0x80000000u);
+    st_release_u32(p.q_slots + (t & p.qmask), entry | 0x80000000u);
 }
 // thread 0 only.  Returns 0 if the queue is empty (or on abort), else the entry (bit 31 set).
 __device__ __forceinline__ unsigned ready_pop(const TiledKernelParams &p) {
@@ -496,7 +511,7 @@ __device__ __forceinline__ unsigned ready_pop(const TiledKernelParams &p) {
         unsigned h = ld_relaxed_u32(p.q_head), t = ld_relaxed_u32(p.q_tail);
         if ((int)(t - h) <= 0) return 0u;
         if (atomicCAS(p.q_head, h, h + 1u) != h) continue;
-        unsigned *slot = p.q_slots + (h & (QCAP - 1));
+        unsigned *slot = p.q_slots + (h & p.qmask);
         unsigned long long spins = 0;
         unsigned e;
         while ((e = ld_acquire_u32(slot)) == 0u) {          // producer has the ticket but has not written yet
@@ -522,7 +537,10 @@ __device__ __forceinline__ unsigned quadrant_needed(int I, int J, int q) {
 __device__ __forceinline__ void quadrant_arrive(const TiledKernelParams &p, int I, int J, int q) {
     unsigned old = atomicAdd(p.qdep + ((long)I * p.ntn + J) * 4 + q, 1u);
     if (old + 1u == quadrant_needed(I, J, q)) {
-        const unsigned entry = ((unsigned)q << 29) | ((unsigned)I << 15) | (unsigned)J | 0x80000000u;
+        // single matrix: q | I (14 bits) | J (15 bits); batched: q | matrix (13 bits) | I (8 bits) | J (8 bits)
+        const unsigned entry = p.batch_index >= 0
+            ? (((unsigned)q << 29) | ((unsigned)p.batch_index << 16) | ((unsigned)I << 8) | (unsigned)J | 0x80000000u)
+            : (((unsigned)q << 29) | ((unsigned)I << 15) | (unsigned)J | 0x80000000u);
         __threadfence();
         ready_push(p, entry);
     }
@@ -530,25 +548,49 @@ __device__ __forceinline__ void quadrant_arrive(const TiledKernelParams &p, int 
 
 constexpr int FAR_CTX = 2;       // far parts a CTA may hold at once (one live in registers, the others parked)
 
+// The persistent scheduler loop.  BATCHED = false: one matrix, described by the kernel argument
+// itself.  BATCHED = true: many matrices in one launch; the kernel argument holds what they share
+// (claim counter, ready ring, abort word, totals) and each task works on a shared-memory copy of
+// its matrix' descriptor (slots 0..FAR_CTX-1: the far contexts, slot FAR_CTX: the quadrant task).
+template <bool BATCHED>
 __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKernelParams p) {
     extern __shared__ __align__(16) double smem[];
     __shared__ int s_task[4];
-    __shared__ int s_ctx[FAR_CTX][6];      // far-part contexts, oldest first: type, I, J, pos, nfar, task
+    __shared__ int s_ctx[FAR_CTX][7];      // far-part contexts, oldest first: type, I, J, pos, nfar, task, view slot
     __shared__ int s_nctx, s_pick, s_state;
     __shared__ unsigned s_pop;
     __shared__ double s_red[TILED_THREADS / 32];
+    __shared__ TiledKernelParams s_view[BATCHED ? FAR_CTX + 1 : 1];
+    static_assert(!BATCHED || FAR_CTX == 2, "view slots of far contexts are handed out as 0 / 1");
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int wm = warp >> 2, wn = warp & 3, g = lane >> 2, t = lane & 3;
-    const int ntiles = p.ntm * p.ntn;
     double max_abs_e = 0.0;
     int cur = -1;                  // context whose accumulator is live in registers (uniform), -1: none
     unsigned long long spins = 0;
     Acc acc;
     acc.zero();
-    if (tid == 0) s_nctx = 0;
+    if (tid == 0) {
+        s_nctx = 0;
+        if (BATCHED)
+            for (int k = 0; k <= FAR_CTX; ++k) s_view[k].batch_index = -1;
+    }
 
+    // the descriptor a task works on: the kernel argument itself for a single matrix (spelled so that the
+    // compiler sees plain parameter accesses there), a shared-memory copy in a batched launch
+#define VIEW(slot) (BATCHED ? s_view[slot] : p)
+    auto load_view = [&](int slot, int b) {            // thread 0, before the barrier that publishes the task
+        if constexpr (BATCHED) {
+            if (s_view[slot].batch_index != b) {
+                const unsigned long long *src = reinterpret_cast<const unsigned long long *>(p.probs + b);
+                unsigned long long *dst = reinterpret_cast<unsigned long long *>(&s_view[slot]);
+                for (int i = 0; i < (int)(sizeof(TiledKernelParams) / 8); ++i) dst[i] = __ldg(src + i);
+            }
+        }
+    };
+    auto entry_matrix = [&](unsigned e) { return (int)((e >> 16) & 0x1fffu); };
     auto tile_region = [&](int k) {
-        return (s_ctx[k][0] == 0 ? p.Cbuf : p.Ebuf) + (long)s_ctx[k][1] * T * p.np + (long)s_ctx[k][2] * T;
+        const TiledKernelParams &pk = VIEW(s_ctx[k][6]);
+        return (s_ctx[k][0] == 0 ? pk.Cbuf : pk.Ebuf) + (long)s_ctx[k][1] * T * pk.np + (long)s_ctx[k][2] * T;
     };
 
     for (;;) {
@@ -560,30 +602,41 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             int state = 2, pick = -1;
             unsigned e = 0u;
             if (ld_relaxed_u32(p.abort) != 0u) state = 4;
-            else if ((e = ready_pop(p)) != 0u) state = 1;
-            else {
+            else if ((e = ready_pop(p)) != 0u) {
+                state = 1;
+                load_view(FAR_CTX, entry_matrix(e));
+            } else {
                 int n = s_nctx;
                 for (int k = 0; k < n && pick < 0; ++k) {
+                    const TiledKernelParams &pk = VIEW(s_ctx[k][6]);
                     const int ty = s_ctx[k][0], pos = s_ctx[k][3];
-                    const unsigned *fl = ty == 0 ? p.flagS + (long)pos * p.ntn + s_ctx[k][2]
-                                                 : p.flagS + (long)s_ctx[k][1] * p.ntn + pos;
+                    const unsigned *fl = ty == 0 ? pk.flagS + (long)pos * pk.ntn + s_ctx[k][2]
+                                                 : pk.flagS + (long)s_ctx[k][1] * pk.ntn + pos;
                     if (pos >= s_ctx[k][4] || ld_acquire_u32(fl) != 0u) pick = k;
                 }
                 if (pick < 0 && n < FAR_CTX && ld_relaxed_u32(p.counter) < (unsigned)p.ntasks) {
                     int task = (int)atomicAdd(p.counter, 1u);
                     if (task < p.ntasks) {
-                        int ty, fi, fj;
-                        decode_task(task, p.ntm, p.ntn, ty, fi, fj);
+                        int ty, fi, fj, slot = 0;
+                        if constexpr (BATCHED) {
+                            const unsigned ft = __ldg(p.far_tasks + task);
+                            ty = (int)((ft >> 16) & 1u); fi = (int)((ft >> 8) & 255u); fj = (int)(ft & 255u);
+                            slot = n == 0 ? 0 : 1 - s_ctx[0][6];
+                            load_view(slot, (int)(ft >> 17));
+                        } else {
+                            decode_task(task, p.ntm, p.ntn, ty, fi, fj);
+                        }
+                        const TiledKernelParams &pk = VIEW(slot);
                         s_ctx[n][0] = ty; s_ctx[n][1] = fi; s_ctx[n][2] = fj; s_ctx[n][3] = 0;
-                        s_ctx[n][4] = max(0, (ty == 0 ? fi : fj) - 1); s_ctx[n][5] = task;
+                        s_ctx[n][4] = max(0, (ty == 0 ? fi : fj) - 1); s_ctx[n][5] = task; s_ctx[n][6] = slot;
                         s_nctx = n + 1;
-                        const unsigned *fl = ty == 0 ? p.flagS + fj : p.flagS + (long)fi * p.ntn;
+                        const unsigned *fl = ty == 0 ? pk.flagS + fj : pk.flagS + (long)fi * pk.ntn;
                         if (s_ctx[n][4] == 0 || ld_acquire_u32(fl) != 0u) pick = n;
                     }
                 }
                 if (pick >= 0) state = 0;
                 else if (s_nctx == 0 && ld_relaxed_u32(p.counter) >= (unsigned)p.ntasks &&
-                         ld_relaxed_u32(p.tiles_done) >= (unsigned)ntiles) state = 3;
+                         ld_relaxed_u32(p.tiles_done) >= (unsigned)p.ntiles_total) state = 3;
             }
             s_state = state; s_pick = pick; s_pop = e;
         }
@@ -607,13 +660,21 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             // ================= A: quadrant tasks from the ready ring.  Never waits.  The live far part,
             // if any, is parked first (the quadrant task needs the shared memory and the registers).
             if (cur >= 0) {
-                if (s_ctx[cur][3] > 0) store_acc(acc, tile_region(cur), p.np, wm, wn, g, t);
+                if (s_ctx[cur][3] > 0) store_acc(acc, tile_region(cur), VIEW(s_ctx[cur][6]).np, wm, wn, g, t);
                 cur = -1;
             }
             unsigned e = s_pop;
             while (e != 0u) {
-                const int q = (int)((e >> 29) & 3u), I = (int)((e >> 15) & 0x3fffu), J = (int)(e & 0x7fffu);
-                sweep_quadrant(I, J, q, smem, p, max_abs_e);
+                const TiledKernelParams &pq = VIEW(FAR_CTX);
+                const int q = (int)((e >> 29) & 3u);
+                const int I = BATCHED ? (int)((e >> 8) & 255u) : (int)((e >> 15) & 0x3fffu);
+                const int J = BATCHED ? (int)(e & 255u) : (int)(e & 0x7fffu);
+                sweep_quadrant(I, J, q, smem, pq, max_abs_e);
+                if constexpr (BATCHED) {                  // max |E| is kept per matrix: flush after every task
+                    for (int o = 16; o > 0; o >>= 1) max_abs_e = fmax(max_abs_e, __shfl_xor_sync(0xffffffffu, max_abs_e, o));
+                    if (lane == 0 && max_abs_e > 0.0) atomic_max_nonneg_double(pq.max_abs_e, max_abs_e);
+                    max_abs_e = 0.0;
+                }
                 // arrivals at everything this quadrant feeds, one per thread (each is a dependent global
                 // atomic round trip); sweep_quadrant ended with a barrier, so each arriving thread's fence
                 // covers the whole CTA's results
@@ -623,23 +684,27 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                     if (tid == 0 && q == 0) { aI = I; aJ = J; aq = 1; }
                     if (tid == 1 && q == 0) { aI = I; aJ = J; aq = 2; }
                     if (tid == 0 && (q == 1 || q == 2)) { aI = I; aJ = J; aq = 3; }
-                    if (tid == 2 && I + 1 < p.ntm) { aI = I + 1; aJ = J; aq = qj; }
-                    if (tid == 3 && I + 1 < p.ntm) { aI = I + 1; aJ = J; aq = 2 + qj; }
-                    if (tid == 4 && J + 1 < p.ntn) { aI = I; aJ = J + 1; aq = 2 * qi; }
-                    if (tid == 5 && J + 1 < p.ntn) { aI = I; aJ = J + 1; aq = 2 * qi + 1; }
+                    if (tid == 2 && I + 1 < pq.ntm) { aI = I + 1; aJ = J; aq = qj; }
+                    if (tid == 3 && I + 1 < pq.ntm) { aI = I + 1; aJ = J; aq = 2 + qj; }
+                    if (tid == 4 && J + 1 < pq.ntn) { aI = I; aJ = J + 1; aq = 2 * qi; }
+                    if (tid == 5 && J + 1 < pq.ntn) { aI = I; aJ = J + 1; aq = 2 * qi + 1; }
                     __threadfence();
-                    if (aI >= 0) quadrant_arrive(p, aI, aJ, aq);
+                    if (aI >= 0) quadrant_arrive(pq, aI, aJ, aq);
                     if (tid == 6) {
-                        unsigned done = atomicAdd(p.quad_done + (long)I * p.ntn + J, 1u);
+                        unsigned done = atomicAdd(pq.quad_done + (long)I * pq.ntn + J, 1u);
                         if (done == 3u) {      // tile swept: far parts that list it as a source may go on
                             __threadfence();
-                            st_release_u32(p.flagS + (long)I * p.ntn + J, 1u);
+                            st_release_u32(pq.flagS + (long)I * pq.ntn + J, 1u);
                             atomicAdd(p.tiles_done, 1u);
                         }
                     }
                 }
                 __syncthreads();
-                if (tid == 0) s_pop = ready_pop(p);
+                if (tid == 0) {
+                    const unsigned en = ready_pop(p);
+                    if (en != 0u) load_view(FAR_CTX, entry_matrix(en));
+                    s_pop = en;
+                }
                 __syncthreads();
                 e = s_pop;
             }
@@ -648,17 +713,18 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
 
         // ================= B: far part s_pick (every source tile of the contraction except the adjacent one)
         const int k = s_pick;
+        const TiledKernelParams &pk = VIEW(s_ctx[k][6]);
         if (k != cur) {
-            if (cur >= 0 && s_ctx[cur][3] > 0) store_acc(acc, tile_region(cur), p.np, wm, wn, g, t);
-            if (s_ctx[k][3] > 0) load_acc(acc, tile_region(k), p.np, wm, wn, g, t);
+            if (cur >= 0 && s_ctx[cur][3] > 0) store_acc(acc, tile_region(cur), VIEW(s_ctx[cur][6]).np, wm, wn, g, t);
+            if (s_ctx[k][3] > 0) load_acc(acc, tile_region(k), pk.np, wm, wn, g, t);
             else acc.zero();
             cur = k;
         }
         const int f_type = s_ctx[k][0], f_I = s_ctx[k][1], f_J = s_ctx[k][2], f_pos = s_ctx[k][3], f_nfar = s_ctx[k][4];
         int new_pos = f_pos;
         if (f_pos < f_nfar) {
-            const unsigned *flags = f_type == 0 ? p.flagS + f_J : p.flagS + (long)f_I * p.ntn;
-            const long fstride = f_type == 0 ? p.ntn : 1;
+            const unsigned *flags = f_type == 0 ? pk.flagS + f_J : pk.flagS + (long)f_I * pk.ntn;
+            const long fstride = f_type == 0 ? pk.ntn : 1;
             // how many source tiles from f_pos on are swept already (the first one is)
             __syncthreads();
             if (tid == 0) s_task[0] = f_nfar;
@@ -669,11 +735,11 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             const int upto = min(s_task[0], f_pos + FAR_RUN_CHUNKS);
             Operand a, b;
             if (f_type == 0) {
-                a.ptr = p.L + (long)f_I * T * p.ldl + (long)f_pos * T; a.ld = p.ldl; a.mn_valid = min(T, p.m - f_I * T); a.aligned16 = p.l_al16;
-                b.ptr = p.Ebuf + (long)f_J * T + (long)f_pos * T * p.np; b.ld = p.np; b.mn_valid = T; b.aligned16 = true;
+                a.ptr = pk.L + (long)f_I * T * pk.ldl + (long)f_pos * T; a.ld = pk.ldl; a.mn_valid = min(T, pk.m - f_I * T); a.aligned16 = pk.l_al16;
+                b.ptr = pk.Ebuf + (long)f_J * T + (long)f_pos * T * pk.np; b.ld = pk.np; b.mn_valid = T; b.aligned16 = true;
             } else {
-                a.ptr = p.Cbuf + (long)f_I * T * p.np + (long)f_pos * T; a.ld = p.np; a.mn_valid = T; a.aligned16 = true;
-                b.ptr = p.U + (long)f_J * T + (long)f_pos * T * p.ldu; b.ld = p.ldu; b.mn_valid = min(T, p.n - f_J * T); b.aligned16 = p.u_al16;
+                a.ptr = pk.Cbuf + (long)f_I * T * pk.np + (long)f_pos * T; a.ld = pk.np; a.mn_valid = T; a.aligned16 = true;
+                b.ptr = pk.U + (long)f_J * T + (long)f_pos * T * pk.ldu; b.ld = pk.ldu; b.mn_valid = min(T, pk.n - f_J * T); b.aligned16 = pk.u_al16;
             }
             gemm_tile<true, false, BULK_NSTAGE>(acc, smem, a, b, (upto - f_pos) * T);
             new_pos = upto;
@@ -681,16 +747,16 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
         if (new_pos >= f_nfar) {
             // far part complete: park the sum (zeros included: the quadrant tasks start from it) and
             // announce it to the four quadrants of its tile; drop the context
-            store_acc(acc, tile_region(k), p.np, wm, wn, g, t);
+            store_acc(acc, tile_region(k), pk.np, wm, wn, g, t);
             __syncthreads();
             if (tid < 4) {
                 __threadfence();
-                quadrant_arrive(p, f_I, f_J, tid);
+                quadrant_arrive(pk, f_I, f_J, tid);
             }
             if (tid == 0) {
                 const int n = s_nctx;
                 for (int c = k; c + 1 < n; ++c)
-                    for (int f = 0; f < 6; ++f) s_ctx[c][f] = s_ctx[c + 1][f];
+                    for (int f = 0; f < 7; ++f) s_ctx[c][f] = s_ctx[c + 1][f];
                 s_nctx = n - 1;
             }
             cur = -1;
@@ -699,15 +765,19 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
         }
     }
 
-    for (int o = 16; o > 0; o >>= 1) max_abs_e = fmax(max_abs_e, __shfl_xor_sync(0xffffffffu, max_abs_e, o));
-    if (lane == 0) s_red[warp] = max_abs_e;
-    __syncthreads();
-    if (tid == 0) {
-        double v = 0.0;
-        for (int w = 0; w < TILED_THREADS / 32; ++w) v = fmax(v, s_red[w]);
-        if (v > 0.0) atomic_max_nonneg_double(p.max_abs_e, v);
+    if constexpr (!BATCHED) {
+        for (int o = 16; o > 0; o >>= 1) max_abs_e = fmax(max_abs_e, __shfl_xor_sync(0xffffffffu, max_abs_e, o));
+        if (lane == 0) s_red[warp] = max_abs_e;
+        __syncthreads();
+        if (tid == 0) {
+            double v = 0.0;
+            for (int w = 0; w < TILED_THREADS / 32; ++w) v = fmax(v, s_red[w]);
+            if (v > 0.0) atomic_max_nonneg_double(p.max_abs_e, v);
+        }
     }
 }
+
+#undef VIEW
 
 // ---------------------------------------------------------------------------------------------
 static size_t pad256(size_t x) { return (x + 255) / 256 * 256; }
@@ -741,6 +811,8 @@ int launch_round_tiled(const TiledParams &in, void *ws, size_t ws_bytes, cudaStr
     TiledKernelParams p{};
     p.m = in.m; p.n = in.n; p.ntm = l.ntm; p.ntn = l.ntn;
     p.ntasks = 2 * l.ntm * l.ntn;
+    p.ntiles_total = l.ntm * l.ntn;
+    p.batch_index = -1;
     p.np = (long)l.ntn * T;
     p.X = in.X; p.ldx = in.ldx; p.L = in.L; p.ldl = in.ldl; p.U = in.U; p.ldu = in.ldu;
     p.Z = in.Z; p.ldz = in.ldz; p.Euser = in.E; p.lde = in.lde;
@@ -750,6 +822,7 @@ int launch_round_tiled(const TiledParams &in, void *ws, size_t ws_bytes, cudaStr
     p.q_tail = reinterpret_cast<unsigned *>(w) + 3;
     p.tiles_done = reinterpret_cast<unsigned *>(w) + 4;
     p.q_slots = reinterpret_cast<unsigned *>(w + l.q_off);
+    p.qmask = QCAP - 1;
     p.max_abs_e = workspace_max_abs_e(ws);
     p.flagS = reinterpret_cast<unsigned *>(w + l.flags_off);
     p.quad_done = reinterpret_cast<unsigned *>(w + l.quad_off);
@@ -764,14 +837,154 @@ int launch_round_tiled(const TiledParams &in, void *ws, size_t ws_bytes, cudaStr
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return GPTQ2D_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GPTQ2D_ERR_CUDA;
-    if (cudaFuncSetAttribute(round_tiled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TILED_SMEM) !=
+    if (cudaFuncSetAttribute(round_tiled_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TILED_SMEM) !=
         cudaSuccess)
         return GPTQ2D_ERR_CUDA;
     int grid = sms < p.ntasks ? sms : p.ntasks;
     void *args[] = {&p};
-    if (cudaLaunchCooperativeKernel((const void *)round_tiled_kernel, dim3(grid), dim3(TILED_THREADS), args,
+    if (cudaLaunchCooperativeKernel((const void *)round_tiled_kernel<false>, dim3(grid), dim3(TILED_THREADS), args,
                                     TILED_SMEM, stream) != cudaSuccess)
         return GPTQ2D_ERR_CUDA;
+    return GPTQ2D_OK;
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// Batched launch: every matrix keeps its own flags, counters and E / C buffers; claim counter,
+// ready ring and abort word are shared.  Workspace: [header | ring | max|E| per matrix | flags of
+// all matrices] (cleared per call) [descriptors | far-part table] (written per call from the
+// host) [E, C buffers].
+struct BatchedLayout {
+    size_t maxe_off, flags_off, zero_end, desc_off, table_off, bufs_off, total;
+    long ntasks, ntiles;
+    unsigned qcap;
+};
+static BatchedLayout batched_layout(int count, const TiledParams *pr) {
+    BatchedLayout l{};
+    long ready_bound = 1;
+    for (int b = 0; b < count; ++b) {
+        TiledLayout t = tiled_layout(pr[b].m, pr[b].n);
+        ready_bound += 2 * (t.ntm < t.ntn ? t.ntm : t.ntn);
+    }
+    l.qcap = QCAP;
+    while ((long)l.qcap < 2 * ready_bound) l.qcap *= 2;     // twice the bound: slots are never close to reuse
+    l.maxe_off = 256 + (size_t)l.qcap * sizeof(unsigned);
+    l.flags_off = l.maxe_off + pad256((size_t)count * sizeof(double));
+    size_t off = l.flags_off, bufs = 0;
+    for (int b = 0; b < count; ++b) {
+        TiledLayout t = tiled_layout(pr[b].m, pr[b].n);
+        size_t tiles = (size_t)t.ntm * t.ntn;
+        off += 2 * pad256(tiles * sizeof(unsigned)) + pad256(4 * tiles * sizeof(unsigned));
+        bufs += 2 * pad256((size_t)t.ntm * T * (size_t)t.ntn * T * sizeof(double));
+        l.ntiles += (long)tiles;
+    }
+    l.ntasks = 2 * l.ntiles;
+    l.zero_end = off;
+    l.desc_off = off;
+    l.table_off = l.desc_off + pad256((size_t)count * sizeof(TiledKernelParams));
+    l.bufs_off = l.table_off + pad256((size_t)l.ntasks * sizeof(unsigned));
+    l.total = l.bufs_off + bufs;
+    return l;
+}
+
+size_t round_tiled_batched_workspace_bytes(int count, const TiledParams *pr) { return batched_layout(count, pr).total; }
+
+__global__ void batched_margin_kernel(const double *max_abs_e, double *min_margin, int count) {
+    int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < count) min_margin[b] = 0.5 - max_abs_e[b];
+}
+
+int launch_round_tiled_batched(int count, const TiledParams *pr, double *min_margin, int *info, void *ws,
+                               size_t ws_bytes, cudaStream_t stream) {
+    if (count < 1 || count > BATCH_MAX_COUNT) return GPTQ2D_ERR_INVALID_ARG;
+    for (int b = 0; b < count; ++b)
+        if (pr[b].m > BATCH_MAX_DIM || pr[b].n > BATCH_MAX_DIM) return GPTQ2D_ERR_TOO_LARGE;
+    BatchedLayout l = batched_layout(count, pr);
+    if (l.ntasks >= (1l << 31)) return GPTQ2D_ERR_TOO_LARGE;
+    if (ws_bytes < l.total) return GPTQ2D_ERR_WORKSPACE;
+    char *w = static_cast<char *>(ws);
+    unsigned *hdr = reinterpret_cast<unsigned *>(w);
+
+    // descriptors and the far-part table are built here and copied in one piece
+    std::vector<unsigned char> stage(l.bufs_off - l.desc_off, 0);
+    TiledKernelParams *desc = reinterpret_cast<TiledKernelParams *>(stage.data());
+    unsigned *table = reinterpret_cast<unsigned *>(stage.data() + (l.table_off - l.desc_off));
+    size_t foff = l.flags_off, boff = l.bufs_off;
+    int max_waves = 0;
+    for (int b = 0; b < count; ++b) {
+        const TiledParams &in = pr[b];
+        TiledLayout t = tiled_layout(in.m, in.n);
+        size_t tiles = (size_t)t.ntm * t.ntn;
+        size_t mat = pad256((size_t)t.ntm * T * (size_t)t.ntn * T * sizeof(double));
+        TiledKernelParams d{};
+        d.m = in.m; d.n = in.n; d.ntm = t.ntm; d.ntn = t.ntn;
+        d.ntasks = (int)(2 * tiles);
+        d.np = (long)t.ntn * T;
+        d.X = in.X; d.ldx = in.ldx; d.L = in.L; d.ldl = in.ldl; d.U = in.U; d.ldu = in.ldu;
+        d.Z = in.Z; d.ldz = in.ldz; d.Euser = in.E; d.lde = in.lde;
+        d.counter = hdr; d.abort = hdr + 1; d.q_head = hdr + 2; d.q_tail = hdr + 3; d.tiles_done = hdr + 4;
+        d.q_slots = reinterpret_cast<unsigned *>(w + 256);
+        d.qmask = l.qcap - 1;
+        d.flagS = reinterpret_cast<unsigned *>(w + foff); foff += pad256(tiles * sizeof(unsigned));
+        d.quad_done = reinterpret_cast<unsigned *>(w + foff); foff += pad256(tiles * sizeof(unsigned));
+        d.qdep = reinterpret_cast<unsigned *>(w + foff); foff += pad256(4 * tiles * sizeof(unsigned));
+        d.Ebuf = reinterpret_cast<double *>(w + boff); boff += mat;
+        d.Cbuf = reinterpret_cast<double *>(w + boff); boff += mat;
+        d.max_abs_e = reinterpret_cast<double *>(w + l.maxe_off) + b;
+        d.info = info;
+        d.l_al16 = ((reinterpret_cast<uintptr_t>(in.L) & 15) == 0) && ((in.ldl & 1) == 0);
+        d.u_al16 = ((reinterpret_cast<uintptr_t>(in.U) & 15) == 0) && ((in.ldu & 1) == 0);
+        d.batch_index = b;
+        d.ntiles_total = (int)tiles;
+        desc[b] = d;
+        if (t.ntm + t.ntn - 1 > max_waves) max_waves = t.ntm + t.ntn - 1;
+    }
+    // claim order: tile-wave by tile-wave over all matrices; inside a matrix' wave as decode_task lists them
+    long nt = 0;
+    for (int wv = 0; wv < max_waves; ++wv)
+        for (int b = 0; b < count; ++b) {
+            const int ntm = desc[b].ntm, ntn = desc[b].ntn;
+            if (wv >= ntm + ntn - 1) continue;
+            const int lo = wv - ntn + 1 > 0 ? wv - ntn + 1 : 0, hi = wv < ntm - 1 ? wv : ntm - 1;
+            for (int k = 0; k <= hi - lo; ++k)
+                for (int type = 0; type < 2; ++type) {
+                    const int I = type == 0 ? hi - k : lo + k, J = wv - I;
+                    table[nt++] = ((unsigned)b << 17) | ((unsigned)type << 16) | ((unsigned)I << 8) | (unsigned)J;
+                }
+        }
+    if (nt != l.ntasks) return GPTQ2D_ERR_INVALID_ARG;
+
+    TiledKernelParams p{};
+    p.ntasks = (int)l.ntasks;
+    p.ntiles_total = (int)l.ntiles;
+    p.batch_index = -1;
+    p.counter = hdr; p.abort = hdr + 1; p.q_head = hdr + 2; p.q_tail = hdr + 3; p.tiles_done = hdr + 4;
+    p.q_slots = reinterpret_cast<unsigned *>(w + 256);
+    p.qmask = l.qcap - 1;
+    p.info = info;
+    p.probs = reinterpret_cast<const TiledKernelParams *>(w + l.desc_off);
+    p.far_tasks = reinterpret_cast<const unsigned *>(w + l.table_off);
+
+    if (cudaMemsetAsync(w, 0, l.zero_end, stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+    // pageable source: the call returns once the bytes have left `stage`
+    if (cudaMemcpyAsync(w + l.desc_off, stage.data(), stage.size(), cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return GPTQ2D_ERR_CUDA;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+    if (cudaFuncSetAttribute(round_tiled_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)TILED_SMEM) != cudaSuccess)
+        return GPTQ2D_ERR_CUDA;
+    int grid = (long)sms < l.ntasks ? sms : (int)l.ntasks;
+    void *args[] = {&p};
+    if (cudaLaunchCooperativeKernel((const void *)round_tiled_kernel<true>, dim3(grid), dim3(TILED_THREADS), args,
+                                    TILED_SMEM, stream) != cudaSuccess)
+        return GPTQ2D_ERR_CUDA;
+    if (min_margin) {
+        batched_margin_kernel<<<(count + 255) / 256, 256, 0, stream>>>(
+            reinterpret_cast<const double *>(w + l.maxe_off), min_margin, count);
+        if (cudaGetLastError() != cudaSuccess) return GPTQ2D_ERR_CUDA;
+    }
     return GPTQ2D_OK;
 }
 

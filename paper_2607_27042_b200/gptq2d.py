@@ -30,7 +30,20 @@ EXPORTS = (
     "gptq2d_round_workspace_bytes", "gptq2d_round", "gptq2d_round_host_workspace_bytes",
     "gptq2d_round_host", "gptq2d_objective_workspace_bytes", "gptq2d_objective",
     "gptq2d_round_static", "gptq2d_round_static_max_dim",
+    "gptq2d_round_batched_workspace_bytes", "gptq2d_round_batched",
 )
+
+BATCH_MAX_COUNT, BATCH_MAX_DIM = 8192, 32768
+
+
+class Problem(ctypes.Structure):
+    """gptq2d_problem_t: one matrix of a batched sweep (device pointers, leading dimensions in elements)."""
+    _fields_ = [("m", ctypes.c_int), ("n", ctypes.c_int),
+                ("X", ctypes.c_void_p), ("ldx", ctypes.c_long),
+                ("L", ctypes.c_void_p), ("ldl", ctypes.c_long),
+                ("U", ctypes.c_void_p), ("ldu", ctypes.c_long),
+                ("Z", ctypes.c_void_p), ("ldz", ctypes.c_long),
+                ("E", ctypes.c_void_p), ("lde", ctypes.c_long)]
 
 
 class Gptq2dError(RuntimeError):
@@ -69,6 +82,10 @@ def _load():
     lib.gptq2d_round_static.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, vp]
     lib.gptq2d_round_static_max_dim.restype = sz
     lib.gptq2d_round_static_max_dim.argtypes = []
+    lib.gptq2d_round_batched_workspace_bytes.restype = sz
+    lib.gptq2d_round_batched_workspace_bytes.argtypes = [i32, vp]
+    lib.gptq2d_round_batched.restype = i32
+    lib.gptq2d_round_batched.argtypes = [i32, vp, vp, vp, sz, vp, vp]
     return lib
 
 
@@ -202,6 +219,50 @@ def gptq2d_round_static(X, L, U, Z, E=None, min_margin=None, info=None, stream=N
     if st != OK:
         raise Gptq2dError(st)
     return Z
+
+
+def _problems(Xs, Ls, Us, Zs, Es):
+    count = len(Xs)
+    arr = (Problem * count)()
+    for b in range(count):
+        m, n = Xs[b].shape
+        pX, ldx = _mat(Xs[b], torch.float64, "X[%d]" % b)
+        pL, ldl = _mat(Ls[b], torch.float64, "L[%d]" % b)
+        pU, ldu = _mat(Us[b], torch.float64, "U[%d]" % b)
+        pZ, ldz = _mat(Zs[b], torch.int32, "Z[%d]" % b)
+        pE, lde = _mat(None if Es is None else Es[b], torch.float64, "E[%d]" % b)
+        arr[b] = Problem(m, n, pX.value, ldx, pL.value, ldl, pU.value, ldu, pZ.value, ldz,
+                         None if pE is None else pE.value, lde)
+    return arr
+
+
+def gptq2d_round_batched_workspace_bytes(Xs, Ls, Us, Zs, Es=None):
+    arr = _problems(Xs, Ls, Us, Zs, Es)
+    return int(_lib.gptq2d_round_batched_workspace_bytes(len(Xs), ctypes.cast(arr, ctypes.c_void_p)))
+
+
+def gptq2d_round_batched(Xs, Ls, Us, Zs=None, Es=None, min_margin=None, workspace=None, info=None, stream=None,
+                         want_E=False, want_margin=False):
+    """Many independent fp64 sweeps in one launch.  Xs, Ls, Us: sequences of CUDA tensors (shapes may
+    differ between matrices).  Returns (Zs, Es, min_margin, info); min_margin has one entry per matrix."""
+    count = len(Xs)
+    dev = Xs[0].device
+    if Zs is None:
+        Zs = [torch.empty(tuple(x.shape), dtype=torch.int32, device=dev) for x in Xs]
+    if Es is None and want_E:
+        Es = [torch.empty(tuple(x.shape), dtype=torch.float64, device=dev) for x in Xs]
+    if min_margin is None and want_margin:
+        min_margin = torch.empty(count, dtype=torch.float64, device=dev)
+    info = torch.zeros(4, dtype=torch.int32, device=dev) if info is None else info
+    arr = _problems(Xs, Ls, Us, Zs, Es)
+    parr = ctypes.cast(arr, ctypes.c_void_p)
+    if workspace is None:
+        workspace = _workspace(_lib.gptq2d_round_batched_workspace_bytes(count, parr), dev)
+    st = _lib.gptq2d_round_batched(count, parr, _ptr(min_margin), _ptr(workspace), workspace.numel(), _ptr(info),
+                                   _stream_ptr(stream))
+    if st != OK:
+        raise Gptq2dError(st)
+    return Zs, Es, min_margin, info
 
 
 def gptq2d_round_host(hX, hL, hU, hZ=None, hE=None, hmargin=None, precision=FP64, workspace=None, hinfo=None,

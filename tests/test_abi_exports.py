@@ -47,3 +47,43 @@ def test_product_package_does_not_import_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 src = open(os.path.join(dirpath, f)).read()
                 assert "import oracle" not in src and "from oracle" not in src, f
+
+
+def test_batched_entry_argument_checks_need_no_gpu():
+    """Host-side validation of the batched call: made-up (never dereferenced) device addresses."""
+    import ctypes as c
+    from paper_2607_27042_b200 import gptq2d as g
+    lib = g._lib
+
+    def probs(shapes):
+        arr = (g.Problem * len(shapes))()
+        for b, (m, n) in enumerate(shapes):
+            arr[b] = g.Problem(m, n, 0x1000, n, 0x2000, m, 0x3000, n, 0x4000, n, None, 0)
+        return arr
+
+    shapes = [(64, 64), (200, 330), (1, 9)]
+    arr = probs(shapes)
+    total = lib.gptq2d_round_batched_workspace_bytes(3, c.cast(arr, c.c_void_p))
+    # at least the padded E and C buffers of every matrix; no more than that plus bookkeeping
+    bufs = sum(2 * 8 * (-(-m // 128) * 128) * (-(-n // 128) * 128) for m, n in shapes)
+    assert bufs <= total < bufs + (1 << 16)
+    one = [lib.gptq2d_round_batched_workspace_bytes(1, c.cast(probs([s]), c.c_void_p)) for s in shapes]
+    assert total <= sum(one)
+    assert lib.gptq2d_round_batched_workspace_bytes(0, c.cast(arr, c.c_void_p)) == 0
+    # invalid descriptors are rejected before any CUDA call
+    ws = c.c_void_p(0x100000)
+    assert lib.gptq2d_round_batched(0, c.cast(arr, c.c_void_p), None, ws, 1 << 40, None, None) == 1
+    assert lib.gptq2d_round_batched(3, None, None, ws, 1 << 40, None, None) == 1
+    bad = probs(shapes)
+    bad[1].ldx = 100                                   # leading dimension below n
+    assert lib.gptq2d_round_batched(3, c.cast(bad, c.c_void_p), None, ws, 1 << 40, None, None) == 1
+    bad = probs(shapes)
+    bad[2].Z = None
+    assert lib.gptq2d_round_batched(3, c.cast(bad, c.c_void_p), None, ws, 1 << 40, None, None) == 1
+    big = probs([(g.BATCH_MAX_DIM + 1, 8)])
+    assert lib.gptq2d_round_batched(1, c.cast(big, c.c_void_p), None, ws, 1 << 40, None, None) == 9
+    many = probs([(8, 8)] * (g.BATCH_MAX_COUNT + 1))
+    assert lib.gptq2d_round_batched(len(many), c.cast(many, c.c_void_p), None, ws, 1 << 40, None, None) == 9
+    # workspace too small / missing
+    assert lib.gptq2d_round_batched(3, c.cast(arr, c.c_void_p), None, ws, total - 1, None, None) == 2
+    assert lib.gptq2d_round_batched(3, c.cast(arr, c.c_void_p), None, None, total, None, None) == 2
