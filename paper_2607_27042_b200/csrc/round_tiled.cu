@@ -534,7 +534,14 @@ __device__ __forceinline__ unsigned quadrant_needed(int I, int J, int q) {
 }
 // the caller has fenced the CTA's results (after a barrier).  The arrival that completes the count
 // publishes the task on the ready ring.
+// A quadrant that lies wholly outside the matrix (ragged last tile row / column) is never a task:
+// arrivals at it are dropped here, its region of the workspace keeps the zeros the far parts parked
+// there, and nothing inside the matrix depends on it.
+__device__ __forceinline__ bool quadrant_exists(const TiledKernelParams &p, int I, int J, int q) {
+    return I * T + (q >> 1) * Q < p.m && J * T + (q & 1) * Q < p.n;
+}
 __device__ __forceinline__ void quadrant_arrive(const TiledKernelParams &p, int I, int J, int q) {
+    if (!quadrant_exists(p, I, J, q)) return;
     unsigned old = atomicAdd(p.qdep + ((long)I * p.ntn + J) * 4 + q, 1u);
     if (old + 1u == quadrant_needed(I, J, q)) {
         // single matrix: q | I (14 bits) | J (15 bits); batched: q | matrix (13 bits) | I (8 bits) | J (8 bits)
@@ -583,7 +590,11 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             if (s_view[slot].batch_index != b) {
                 const unsigned long long *src = reinterpret_cast<const unsigned long long *>(p.probs + b);
                 unsigned long long *dst = reinterpret_cast<unsigned long long *>(&s_view[slot]);
-                for (int i = 0; i < (int)(sizeof(TiledKernelParams) / 8); ++i) dst[i] = __ldg(src + i);
+                unsigned long long v[sizeof(TiledKernelParams) / 8];
+#pragma unroll
+                for (int i = 0; i < (int)(sizeof(TiledKernelParams) / 8); ++i) v[i] = __ldg(src + i);   // all in flight
+#pragma unroll
+                for (int i = 0; i < (int)(sizeof(TiledKernelParams) / 8); ++i) dst[i] = v[i];
             }
         }
     };
@@ -692,7 +703,8 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                     if (aI >= 0) quadrant_arrive(pq, aI, aJ, aq);
                     if (tid == 6) {
                         unsigned done = atomicAdd(pq.quad_done + (long)I * pq.ntn + J, 1u);
-                        if (done == 3u) {      // tile swept: far parts that list it as a source may go on
+                        const unsigned nquad = (pq.m - I * T > Q ? 2u : 1u) * (pq.n - J * T > Q ? 2u : 1u);
+                        if (done + 1u == nquad) {   // tile swept: far parts that list it as a source may go on
                             __threadfence();
                             st_release_u32(pq.flagS + (long)I * pq.ntn + J, 1u);
                             atomicAdd(p.tiles_done, 1u);

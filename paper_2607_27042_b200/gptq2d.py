@@ -236,26 +236,36 @@ def _problems(Xs, Ls, Us, Zs, Es):
     return arr
 
 
-def gptq2d_round_batched_workspace_bytes(Xs, Ls, Us, Zs, Es=None):
-    arr = _problems(Xs, Ls, Us, Zs, Es)
-    return int(_lib.gptq2d_round_batched_workspace_bytes(len(Xs), ctypes.cast(arr, ctypes.c_void_p)))
+def make_problems(Xs, Ls, Us, Zs, Es=None):
+    """The host descriptor array (gptq2d_problem_t[count]) of a batch; reusable across calls as long as
+    the tensors it points to stay alive and in place."""
+    return _problems(Xs, Ls, Us, Zs, Es)
 
 
-def gptq2d_round_batched(Xs, Ls, Us, Zs=None, Es=None, min_margin=None, workspace=None, info=None, stream=None,
-                         want_E=False, want_margin=False):
+def gptq2d_round_batched_workspace_bytes(Xs=None, Ls=None, Us=None, Zs=None, Es=None, problems=None):
+    arr = _problems(Xs, Ls, Us, Zs, Es) if problems is None else problems
+    return int(_lib.gptq2d_round_batched_workspace_bytes(len(arr), ctypes.cast(arr, ctypes.c_void_p)))
+
+
+def gptq2d_round_batched(Xs=None, Ls=None, Us=None, Zs=None, Es=None, min_margin=None, workspace=None, info=None,
+                         stream=None, want_E=False, want_margin=False, problems=None, device=None):
     """Many independent fp64 sweeps in one launch.  Xs, Ls, Us: sequences of CUDA tensors (shapes may
-    differ between matrices).  Returns (Zs, Es, min_margin, info); min_margin has one entry per matrix."""
-    count = len(Xs)
-    dev = Xs[0].device
-    if Zs is None:
-        Zs = [torch.empty(tuple(x.shape), dtype=torch.int32, device=dev) for x in Xs]
-    if Es is None and want_E:
-        Es = [torch.empty(tuple(x.shape), dtype=torch.float64, device=dev) for x in Xs]
+    differ between matrices), or `problems` = an array from make_problems (then Zs / Es are whatever
+    that array points to).  Returns (Zs, Es, min_margin, info); min_margin has one entry per matrix."""
+    if problems is None:
+        dev = Xs[0].device
+        if Zs is None:
+            Zs = [torch.empty(tuple(x.shape), dtype=torch.int32, device=dev) for x in Xs]
+        if Es is None and want_E:
+            Es = [torch.empty(tuple(x.shape), dtype=torch.float64, device=dev) for x in Xs]
+        problems = _problems(Xs, Ls, Us, Zs, Es)
+    else:
+        dev = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    count = len(problems)
     if min_margin is None and want_margin:
         min_margin = torch.empty(count, dtype=torch.float64, device=dev)
     info = torch.zeros(4, dtype=torch.int32, device=dev) if info is None else info
-    arr = _problems(Xs, Ls, Us, Zs, Es)
-    parr = ctypes.cast(arr, ctypes.c_void_p)
+    parr = ctypes.cast(problems, ctypes.c_void_p)
     if workspace is None:
         workspace = _workspace(_lib.gptq2d_round_batched_workspace_bytes(count, parr), dev)
     st = _lib.gptq2d_round_batched(count, parr, _ptr(min_margin), _ptr(workspace), workspace.numel(), _ptr(info),
