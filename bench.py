@@ -1,6 +1,6 @@
 """Benchmark of the GPTQ-2D sweep (the hot path) on B200.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--config 4] [--fp32]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--config 4] [--fp32] [--batch B]
 
 A step is one full sweep (Algorithm 3: initialisation + all m+n-1 anti-diagonals, i.e. one
 gptq2d_round call) of one synthetic m x n matrix with X, L, U resident in HBM.  The set-up
@@ -269,6 +269,117 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
+def run_batched(args):
+    """--batch K: K matrices of the chosen configuration (same bases, K different X) swept by ONE
+    gptq2d_round_batched launch, against the same K sweeps issued one after the other."""
+    import torch
+    from paper_2607_27042_b200 import gptq2d as g
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist = dist_
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    K = args.batch
+    X, A, B, name = workload(args.config, args.seed + rank)
+    m, n = X.shape
+    dA, dB = (torch.from_numpy(np.ascontiguousarray(a)).cuda() for a in (A, B))
+    L, U, _, _, finfo = g.gptq2d_factor(dA, dB)
+    torch.cuda.synchronize()
+    g.check_info(finfo)
+    stream = torch.cuda.current_stream()
+    rng = np.random.default_rng(args.seed + 7919 * (rank + 1))
+    hXs = [torch.from_numpy(np.ascontiguousarray(X[rng.permutation(m)][:, rng.permutation(n)])).pin_memory()
+           for _ in range(K)]
+    Xs = [h.cuda() for h in hXs]
+    Zs = [torch.empty((m, n), dtype=torch.int32, device="cuda") for _ in range(K)]
+    hZs = [torch.empty((m, n), dtype=torch.int32).pin_memory() for _ in range(K)]
+    probs = g.make_problems(Xs, [L] * K, [U] * K, Zs)
+    ws = torch.empty(g.gptq2d_round_batched_workspace_bytes(problems=probs), dtype=torch.uint8, device="cuda")
+    ws1 = torch.empty(g.gptq2d_round_workspace_bytes(m, n), dtype=torch.uint8, device="cuda")
+    info = torch.zeros(4, dtype=torch.int32, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # larger than the 126 MB L2
+
+    def step():
+        g.gptq2d_round_batched(problems=probs, workspace=ws, info=info, stream=stream)
+
+    def one_by_one():
+        for b in range(K):
+            g.gptq2d_round(Xs[b], L, U, Z=Zs[b], workspace=ws1, info=info, stream=stream)
+
+    def timed(fn, reps):
+        out = []
+        for _ in range(reps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); fn(); b.record(stream)
+            torch.cuda.synchronize()
+            out.append(a.elapsed_time(b))
+        return out
+
+    for _ in range(args.warmup):
+        step()
+    one_by_one()
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    per_step = timed(step, args.steps)
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    g.check_info(info)
+    Zb = [z.clone() for z in Zs]
+    seq = timed(one_by_one, max(2, min(args.steps, 5)))
+    g.check_info(info)
+    assert all(torch.equal(a, b) for a, b in zip(Zb, Zs)), "batched and single sweeps disagree"
+    ms_per_step = max_over_ranks(float(np.mean(per_step)), dist, "cuda")
+    seq_ms = max_over_ranks(float(np.mean(seq)), dist, "cuda")
+
+    def e2e_step():
+        for b in range(K):
+            Xs[b].copy_(hXs[b], non_blocking=True)
+        step()
+        for b in range(K):
+            hZs[b].copy_(Zs[b], non_blocking=True)
+    e2e_ms = max_over_ranks(float(np.mean(timed(e2e_step, max(2, min(args.steps, 5))))), dist, "cuda")
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+    flops = float(K) * m * n * (m + n - 2)
+    achieved = flops / (ms_per_step * 1e-3) / 1e12
+    out = {
+        "metric": METRIC, "value": world * K * m * n / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "%s x %d, one batched launch" % (name, K), "m": m, "n": n, "batch": K,
+                   "seed": args.seed, "replicas": world, "l2": "256 MB written between timed steps",
+                   "timed": "gptq2d_round_batched over %d matrices (same bases, different X)" % K},
+        "clocks": clocks, "gpu_launches": args.steps,
+        "e2e": {"value": world * K * m * n / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": 8 * K * m * n, "d2h_bytes_per_step": 4 * K * m * n,
+                "note": "X copied in from pinned memory and Z copied out every step; L, U resident"},
+        "one_by_one": {"ms_per_step": seq_ms, "value": world * K * m * n / (seq_ms * 1e-3), "unit": UNIT,
+                       "note": "the same %d sweeps as %d gptq2d_round calls on one stream" % (K, K)},
+        "batch_speedup": seq_ms / ms_per_step,
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": FP64_NOMINAL_TFLOPS, "unit": "TFLOP/s",
+                     "frac": achieved / FP64_NOMINAL_TFLOPS, "traffic": None, "kernel": "round_tiled_kernel<true>",
+                     "kernel_ms": ms_per_step, "flops_per_launch": flops},
+        "per_step_ms": per_step,
+    }
+    print(json.dumps(out))
+    if dist:
+        dist.destroy_process_group()
+
+
 def cpu_baseline(X, A, B, budget_s=12.0, want_alg3=True):
     """The oracle as it stands, on the host cores, on a bounded sample of the workload."""
     import oracle as O
@@ -360,10 +471,14 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--ref-coords", type=int, default=16)
+    ap.add_argument("--batch", type=int, default=0,
+                    help="sweep this many matrices of --config in one batched launch (and one by one, for comparison)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.batch > 0:
+        run_batched(args)
     else:
         run_cuda(args)
 
