@@ -108,6 +108,19 @@ def job_value(m, n, world, ms_per_step):
     return world * m * n / (ms_per_step * 1e-3)
 
 
+def host_entry_h2d_bytes(m, n, fp32):
+    """Bytes gptq2d_round_host copies to the device: all of X, L, U in the fp32 mode; in the fp64 mode X
+    plus the rows of L up to the end of each 512 x 512 diagonal block and the columns of U down to it."""
+    if fp32:
+        return 8 * (m * n + m * m + n * n)
+    total = 8 * m * n
+    for r0 in range(0, m, 512):
+        total += 8 * min(512, m - r0) * min(m, r0 + 512)
+    for r0 in range(0, n, 512):
+        total += 8 * min(512, n - r0) * min(n, r0 + 512)
+    return total
+
+
 def workload(index, seed):
     from paper_2607_27042_b200 import workloads as W
     X, A, B = W.make_config(index, seed=seed)
@@ -207,7 +220,10 @@ def run_cuda(args):
         e2e_ms = max_over_ranks(e2e_ms, dist, "cuda")
         assert torch.equal(hZ, Z.cpu()), "host entry point and device entry point disagree"
         e2e = {"value": job_value(m, n, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
-               "h2d_bytes_per_step": 8 * (m * n + m * m + n * n), "d2h_bytes_per_step": 4 * m * n + 16}
+               "h2d_bytes_per_step": host_entry_h2d_bytes(m, n, args.fp32), "d2h_bytes_per_step": 4 * m * n + 16,
+               "note": "fp64: inputs arrive in steps on a second stream while the sweep already runs; of L and U "
+                       "only the triangles (up to the edge of the diagonal tile) are sent; Z is written "
+                       "straight into the pinned host buffer by the kernel (d2h bytes cross the bus all the same)"}
 
     if rank != 0:
         if dist:

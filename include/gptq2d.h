@@ -98,11 +98,21 @@ int gptq2d_round(int m, int n,
                  int precision,
                  void *workspace, size_t workspace_bytes, int *info, void *stream);
 
-/* Same sweep with HOST buffers: X, L, U are copied to the device workspace, the sweep runs, and
- * Z (and E, min_margin if non-NULL) are copied back; all on `stream`, which is synchronised
- * before returning.  hX, hL, hU, hZ, hE are host pointers (pinned memory makes the copies
- * asynchronous and fast), dense row-major (leading dimension = number of columns).
- * hinfo: host int[4], receives the device info words.  The workspace is still a device buffer.
+/* Same sweep with HOST buffers; `stream` is synchronised before returning.  hX, hL, hU, hZ, hE are host
+ * pointers, dense row-major (leading dimension = number of columns); hinfo: host int[4], receives the
+ * device info words.  The workspace is still a device buffer.
+ * GPTQ2D_FP64: the copies overlap the sweep.  The kernel is launched at once and the inputs follow on a
+ *   second stream (one per device, created by the library on first use) in 512 x 512 blocks, in the
+ *   order the anti-diagonal wavefront needs them (Section 2, Fig. 1: entry (i, j) depends on the
+ *   rectangle above and to its left only): step s = the blocks of X on block anti-diagonal s, block
+ *   row s of L up to its diagonal block, block column s of U down to its diagonal block (the opposite
+ *   triangles are never sent).  Each step is announced to the running kernel by a stream-ordered
+ *   32-bit write; a task starts when its step has arrived.  If hZ is pinned, device-mapped memory the
+ *   kernel writes Z straight into it, quadrant by quadrant, and no copy back follows.  Pinned buffers
+ *   make all copies asynchronous and fast; pageable ones work.  If the driver lacks stream memory
+ *   operations the call falls back to copy-then-sweep.  Concurrent calls on one device take turns to
+ *   enqueue (they share the copy stream).
+ * Other precisions: X, L, U are copied first, the sweep runs, Z (and E, min_margin) are copied back.
  */
 size_t gptq2d_round_host_workspace_bytes(int m, int n, int precision);
 int gptq2d_round_host(int m, int n,

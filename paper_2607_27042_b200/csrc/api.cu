@@ -2,6 +2,7 @@
 #include <cuda_runtime.h>
 #include "common.cuh"
 #include "round_internal.cuh"
+#include <mutex>
 #include <vector>
 
 namespace gptq2d {
@@ -24,6 +25,43 @@ static int check_device() {
 }
 
 static size_t pad256(size_t x) { return (x + 255) / 256 * 256; }
+
+// ---- helpers of the pipelined host entry point ------------------------------------------------
+// A second stream (per device, created on first use) carries the host-to-device copies while the
+// sweep kernel already runs on the caller's stream; the copy stream announces each 128-row panel
+// with a stream-ordered 32-bit write (driver entry point looked up through the runtime, so the
+// library has no link-time dependency on the driver library).
+typedef int (*StreamWriteValue32Fn)(cudaStream_t, unsigned long long, unsigned int, unsigned int);
+struct HostPipe {
+    cudaStream_t copy = nullptr;
+    cudaEvent_t inputs_free = nullptr, copies_done = nullptr;
+    StreamWriteValue32Fn write32 = nullptr;
+    bool tried = false;
+    std::mutex enqueue;         // one pipelined call at a time enqueues on the shared copy stream and events
+};
+static std::mutex g_pipe_mutex;
+static HostPipe g_pipe[64];
+
+// NULL if the device cannot do it (then the caller copies everything first, as before)
+static HostPipe *host_pipe() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    HostPipe &hp = g_pipe[dev];
+    if (!hp.tried) {
+        hp.tried = true;
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qr = cudaDriverEntryPointSymbolNotFound;
+        bool ok = cudaGetDriverEntryPoint("cuStreamWriteValue32", &fn, cudaEnableDefault, &qr) == cudaSuccess &&
+                  qr == cudaDriverEntryPointSuccess && fn != nullptr;
+        ok = ok && cudaStreamCreateWithFlags(&hp.copy, cudaStreamNonBlocking) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&hp.inputs_free, cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&hp.copies_done, cudaEventDisableTiming) == cudaSuccess;
+        if (ok) hp.write32 = reinterpret_cast<StreamWriteValue32Fn>(fn);
+        (void)cudaGetLastError();
+    }
+    return hp.write32 ? &hp : nullptr;
+}
 
 // host descriptors of a batched call -> internal launch parameters, with the argument checks of gptq2d_round
 static int to_tiled(int count, const gptq2d_problem_t *pr, std::vector<TiledParams> &out) {
@@ -184,14 +222,89 @@ int gptq2d_round_host(int m, int n, const double *hX, const double *hL, const do
     double *dE = reinterpret_cast<double *>(p); p += pad256((size_t)m * n * 8);
     int *dinfo = reinterpret_cast<int *>(p);
     double *dmargin = reinterpret_cast<double *>(p + 64);
+    HostPipe *hp = (precision == GPTQ2D_FP64) ? host_pipe() : nullptr;
+    std::unique_lock<std::mutex> pipe_lock;
+    bool z_direct = false;
+    if (hp) {
+        pipe_lock = std::unique_lock<std::mutex>(hp->enqueue);
+        // Pipelined: the sweep starts at once and the inputs follow in steps (see below; of L and U only the
+        // triangles the sweep reads).  The kernel holds back each task until its step has arrived.
+        unsigned *dpanels = reinterpret_cast<unsigned *>(p + 128);
+        if (cudaMemsetAsync(dpanels, 0, sizeof(unsigned), stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+        // the copies may overwrite dX, dL, dU only after everything queued on `stream` so far is done
+        if (cudaEventRecord(hp->inputs_free, stream) != cudaSuccess ||
+            cudaStreamWaitEvent(hp->copy, hp->inputs_free, 0) != cudaSuccess)
+            return GPTQ2D_ERR_CUDA;
+        if (hinfo) { hinfo[0] = hinfo[1] = hinfo[2] = hinfo[3] = 0; }
+        if (cudaMemsetAsync(dinfo, 0, 4 * sizeof(int), stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+        TiledParams tp{};
+        tp.m = m; tp.n = n;
+        tp.X = dX; tp.ldx = n; tp.L = dL; tp.ldl = m; tp.U = dU; tp.ldu = n;
+        tp.Z = dZ; tp.ldz = n; tp.E = hE ? dE : nullptr; tp.lde = n; tp.info = dinfo;
+        // Z in pinned, device-mapped host memory is written by the kernel directly, quadrant by quadrant,
+        // as the sweep goes: no copy back at the end
+        cudaPointerAttributes za{};
+        if (cudaPointerGetAttributes(&za, hZ) == cudaSuccess && za.type == cudaMemoryTypeHost && za.devicePointer) {
+            tp.Z = static_cast<int32_t *>(za.devicePointer);
+            z_direct = true;
+        }
+        (void)cudaGetLastError();
+        tp.panels_ready = dpanels;
+        int st = launch_round_tiled(tp, w, inner, stream);
+        if (st != GPTQ2D_OK) return st;
+        if (hmin_margin) {
+            margin_kernel<<<1, 1, 0, stream>>>(workspace_max_abs_e(w), dmargin);
+            if (cudaGetLastError() != cudaSuccess) return GPTQ2D_ERR_CUDA;
+        }
+        // Step s sends the blocks of X on block anti-diagonal s, block row s of L and block column s of U
+        // (COPY_BLOCK x COPY_BLOCK blocks): the order in which the wavefront of the sweep needs them.
+        const int CB = COPY_BLOCK, nbm = (m + CB - 1) / CB, nbn = (n + CB - 1) / CB;
+        auto copy2d = [&](double *dst, const double *src, size_t ld, int rows, int cols) {
+            if (rows <= 0 || cols <= 0) return true;
+            return cudaMemcpy2DAsync(dst, ld * 8, src, ld * 8, (size_t)cols * 8, rows, cudaMemcpyHostToDevice,
+                                     hp->copy) == cudaSuccess;
+        };
+        auto extent = [&](int b, int total) { return total - b * CB < CB ? total - b * CB : CB; };
+        bool ok = true;
+        for (int step = 0; step < nbm + nbn - 1 && ok; ++step) {
+            const int lo = step - nbn + 1 > 0 ? step - nbn + 1 : 0, hi = step < nbm - 1 ? step : nbm - 1;
+            for (int bi = lo; bi <= hi && ok; ++bi) {
+                const int bj = step - bi;
+                const size_t off = (size_t)bi * CB * n + (size_t)bj * CB;
+                ok = copy2d(dX + off, hX + off, n, extent(bi, m), extent(bj, n));
+            }
+            if (step < nbm)       // rows of block row `step`, columns up to the end of the diagonal block
+                ok = ok && copy2d(dL + (size_t)step * CB * m, hL + (size_t)step * CB * m, m, extent(step, m),
+                                  (step + 1) * CB < m ? (step + 1) * CB : m);
+            if (step < nbn)       // columns of block column `step`, rows down to the end of the diagonal block
+                ok = ok && copy2d(dU + (size_t)step * CB, hU + (size_t)step * CB, n,
+                                  (step + 1) * CB < n ? (step + 1) * CB : n, extent(step, n));
+            ok = ok && hp->write32(hp->copy, (unsigned long long)reinterpret_cast<uintptr_t>(dpanels),
+                                   (unsigned)(step + 1), 0u) == 0;
+        }
+        if (!ok) {
+            // the kernel may be waiting for panels that will never come: let it through (its result is
+            // discarded) rather than have it run into its time limit
+            (void)hp->write32(hp->copy, (unsigned long long)reinterpret_cast<uintptr_t>(dpanels), 0x7fffffffu, 0u);
+            (void)cudaStreamSynchronize(stream);
+            return GPTQ2D_ERR_CUDA;
+        }
+        if (cudaEventRecord(hp->copies_done, hp->copy) != cudaSuccess ||
+            cudaStreamWaitEvent(stream, hp->copies_done, 0) != cudaSuccess)
+            return GPTQ2D_ERR_CUDA;
+        pipe_lock.unlock();
+    } else
     if (cudaMemcpyAsync(dX, hX, (size_t)m * n * 8, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
         cudaMemcpyAsync(dL, hL, (size_t)m * m * 8, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
         cudaMemcpyAsync(dU, hU, (size_t)n * n * 8, cudaMemcpyHostToDevice, stream) != cudaSuccess)
         return GPTQ2D_ERR_CUDA;
-    int st = gptq2d_round(m, n, dX, n, dL, m, dU, n, dZ, n, hE ? dE : nullptr, n, hmin_margin ? dmargin : nullptr,
-                          precision, w, inner, dinfo, stream_);
-    if (st != GPTQ2D_OK) return st;
-    if (cudaMemcpyAsync(hZ, dZ, (size_t)m * n * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+    if (!hp) {
+        int st = gptq2d_round(m, n, dX, n, dL, m, dU, n, dZ, n, hE ? dE : nullptr, n, hmin_margin ? dmargin : nullptr,
+                              precision, w, inner, dinfo, stream_);
+        if (st != GPTQ2D_OK) return st;
+    }
+    if (!z_direct && cudaMemcpyAsync(hZ, dZ, (size_t)m * n * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return GPTQ2D_ERR_CUDA;
     if (hE && cudaMemcpyAsync(hE, dE, (size_t)m * n * 8, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
         return GPTQ2D_ERR_CUDA;
     if (hmin_margin && cudaMemcpyAsync(hmin_margin, dmargin, 8, cudaMemcpyDeviceToHost, stream) != cudaSuccess)

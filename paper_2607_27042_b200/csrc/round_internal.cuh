@@ -29,7 +29,15 @@ struct TiledParams {
     double *E; long lde;      // optional user copy of the local errors
     double *max_abs_e;
     int *info;
+    // optional: device word that counts the copy steps of X, L and U that have arrived (the sweep then
+    // starts while the rest is still on its way, see COPY_BLOCK_TILES); NULL = everything is resident
+    const unsigned *panels_ready;
 };
+// Inputs that arrive while the sweep runs come in blocks of COPY_BLOCK_TILES x COPY_BLOCK_TILES tiles of
+// 128 x 128: step s = the blocks of X on block anti-diagonal s, block row s of L (up to the end of its
+// diagonal block), block column s of U (down to the end of its diagonal block).
+constexpr int COPY_BLOCK_TILES_LOG2 = 2;
+constexpr int COPY_BLOCK = 128 << COPY_BLOCK_TILES_LOG2;
 size_t round_tiled_workspace_bytes(int m, int n);
 int launch_round_tiled(const TiledParams &p, void *ws, size_t ws_bytes, cudaStream_t stream);
 // many matrices in one launch (fp64 tiled sweep); `info` is shared, `min_margin` (optional) gets one value per matrix

@@ -69,6 +69,8 @@ struct TiledKernelParams {
     int ntiles_total;
     const TiledKernelParams *probs;
     const unsigned *far_tasks;   // far parts of all matrices in claim order: b << 17 | type << 16 | I << 8 | J
+    // pipelined host entry only: number of 128-row panels of X, L and U that have reached the device
+    const unsigned *panels_ready;
 };
 static_assert(sizeof(TiledKernelParams) % 8 == 0, "descriptors are copied as 8-byte words");
 
@@ -559,7 +561,12 @@ constexpr int FAR_CTX = 2;       // far parts a CTA may hold at once (one live i
 // itself.  BATCHED = true: many matrices in one launch; the kernel argument holds what they share
 // (claim counter, ready ring, abort word, totals) and each task works on a shared-memory copy of
 // its matrix' descriptor (slots 0..FAR_CTX-1: the far contexts, slot FAR_CTX: the quadrant task).
-template <bool BATCHED>
+// PANELS = true (single matrix only): the inputs are still being copied in while the kernel runs, in
+// blocks of COPY_BLOCK_TILES x COPY_BLOCK_TILES tiles and in the order the wavefront needs them: step
+// s brings the blocks of X on block anti-diagonal s, the block row s of L and the block column s of
+// U.  A task on tile (I, J) starts once the copy stream has announced the step of its block
+// (p.panels_ready counts the steps that arrived).
+template <bool BATCHED, bool PANELS>
 __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKernelParams p) {
     extern __shared__ __align__(16) double smem[];
     __shared__ int s_task[4];
@@ -599,6 +606,29 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
         }
     };
     auto entry_matrix = [&](unsigned e) { return (int)((e >> 16) & 0x1fffu); };
+    // thread 0.  Far parts poll (they have other things to do); a popped quadrant task waits, bounded:
+    // the copies make progress on their own.
+    auto panels_arrived = [&](int need) -> bool {
+        if constexpr (PANELS) return ld_acquire_u32(p.panels_ready) >= (unsigned)need;
+        else return true;
+    };
+    auto await_panels = [&](unsigned e) -> unsigned {
+        if constexpr (PANELS) {
+            if (e == 0u) return e;
+            const int need = ((int)((e >> 15) & 0x3fffu) >> COPY_BLOCK_TILES_LOG2) +
+                             ((int)(e & 0x7fffu) >> COPY_BLOCK_TILES_LOG2) + 1;
+            unsigned long long it = 0;
+            while (!panels_arrived(need)) {
+                if (++it > SPIN_LIMIT || ld_relaxed_u32(p.abort) != 0u) {
+                    report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -6, need, (int)blockIdx.x);
+                    atomicExch(p.abort, 1u);
+                    return 0u;
+                }
+                __nanosleep(200);
+            }
+        }
+        return e;
+    };
     auto tile_region = [&](int k) {
         const TiledKernelParams &pk = VIEW(s_ctx[k][6]);
         return (s_ctx[k][0] == 0 ? pk.Cbuf : pk.Ebuf) + (long)s_ctx[k][1] * T * pk.np + (long)s_ctx[k][2] * T;
@@ -613,7 +643,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             int state = 2, pick = -1;
             unsigned e = 0u;
             if (ld_relaxed_u32(p.abort) != 0u) state = 4;
-            else if ((e = ready_pop(p)) != 0u) {
+            else if ((e = await_panels(ready_pop(p))) != 0u) {
                 state = 1;
                 load_view(FAR_CTX, entry_matrix(e));
             } else {
@@ -623,7 +653,10 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                     const int ty = s_ctx[k][0], pos = s_ctx[k][3];
                     const unsigned *fl = ty == 0 ? pk.flagS + (long)pos * pk.ntn + s_ctx[k][2]
                                                  : pk.flagS + (long)s_ctx[k][1] * pk.ntn + pos;
-                    if (pos >= s_ctx[k][4] || ld_acquire_u32(fl) != 0u) pick = k;
+                    // a Cd part reads L in the block row of I, an Rt part U in the block column of J
+                    if ((pos >= s_ctx[k][4] || ld_acquire_u32(fl) != 0u) &&
+                        panels_arrived(((ty == 0 ? s_ctx[k][1] : s_ctx[k][2]) >> COPY_BLOCK_TILES_LOG2) + 1))
+                        pick = k;
                 }
                 if (pick < 0 && n < FAR_CTX && ld_relaxed_u32(p.counter) < (unsigned)p.ntasks) {
                     int task = (int)atomicAdd(p.counter, 1u);
@@ -642,7 +675,8 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                         s_ctx[n][4] = max(0, (ty == 0 ? fi : fj) - 1); s_ctx[n][5] = task; s_ctx[n][6] = slot;
                         s_nctx = n + 1;
                         const unsigned *fl = ty == 0 ? pk.flagS + fj : pk.flagS + (long)fi * pk.ntn;
-                        if (s_ctx[n][4] == 0 || ld_acquire_u32(fl) != 0u) pick = n;
+                        if ((s_ctx[n][4] == 0 || ld_acquire_u32(fl) != 0u) && panels_arrived(((ty == 0 ? fi : fj) >> COPY_BLOCK_TILES_LOG2) + 1))
+                            pick = n;
                     }
                 }
                 if (pick >= 0) state = 0;
@@ -713,7 +747,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                 }
                 __syncthreads();
                 if (tid == 0) {
-                    const unsigned en = ready_pop(p);
+                    const unsigned en = await_panels(ready_pop(p));
                     if (en != 0u) load_view(FAR_CTX, entry_matrix(en));
                     s_pop = en;
                 }
@@ -849,13 +883,14 @@ int launch_round_tiled(const TiledParams &in, void *ws, size_t ws_bytes, cudaStr
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return GPTQ2D_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GPTQ2D_ERR_CUDA;
-    if (cudaFuncSetAttribute(round_tiled_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TILED_SMEM) !=
-        cudaSuccess)
+    p.panels_ready = in.panels_ready;
+    const void *kernel = in.panels_ready ? (const void *)round_tiled_kernel<false, true>
+                                         : (const void *)round_tiled_kernel<false, false>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TILED_SMEM) != cudaSuccess)
         return GPTQ2D_ERR_CUDA;
     int grid = sms < p.ntasks ? sms : p.ntasks;
     void *args[] = {&p};
-    if (cudaLaunchCooperativeKernel((const void *)round_tiled_kernel<false>, dim3(grid), dim3(TILED_THREADS), args,
-                                    TILED_SMEM, stream) != cudaSuccess)
+    if (cudaLaunchCooperativeKernel(kernel, dim3(grid), dim3(TILED_THREADS), args, TILED_SMEM, stream) != cudaSuccess)
         return GPTQ2D_ERR_CUDA;
     return GPTQ2D_OK;
 }
@@ -984,12 +1019,12 @@ int launch_round_tiled_batched(int count, const TiledParams *pr, double *min_mar
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return GPTQ2D_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GPTQ2D_ERR_CUDA;
-    if (cudaFuncSetAttribute(round_tiled_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(round_tiled_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)TILED_SMEM) != cudaSuccess)
         return GPTQ2D_ERR_CUDA;
     int grid = (long)sms < l.ntasks ? sms : (int)l.ntasks;
     void *args[] = {&p};
-    if (cudaLaunchCooperativeKernel((const void *)round_tiled_kernel<true>, dim3(grid), dim3(TILED_THREADS), args,
+    if (cudaLaunchCooperativeKernel((const void *)round_tiled_kernel<true, false>, dim3(grid), dim3(TILED_THREADS), args,
                                     TILED_SMEM, stream) != cudaSuccess)
         return GPTQ2D_ERR_CUDA;
     if (min_margin) {

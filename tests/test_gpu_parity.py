@@ -234,6 +234,34 @@ def test_strided_inputs_and_host_entry(g):
     assert np.array_equal(hZ.numpy().astype(np.int64), ref["Z"])
 
 
+@pytest.mark.parametrize("m,n,seed,pinned", [(1100, 700, 31, True), (700, 1100, 32, False), (1537, 1537, 33, True),
+                                             (513, 40, 34, True)])
+def test_host_entry_streams_inputs_while_sweeping(g, m, n, seed, pinned):
+    """gptq2d_round_host sends X, L, U in 512 x 512 blocks while the kernel already runs (several copy
+    steps, ragged last blocks); Z must be what the device entry point gives on resident inputs, which
+    in turn is checked against the nested CPU oracle and the certificate."""
+    X, A, B = W.general_bases(m, n, seed)
+    L, U, _, _ = O.feedback_factors(A, B)
+    ref = cref.nested(X, L, U)
+    margin, _ = O.certificate_margin(X, ref["Z"], L, U)
+    if margin < MARGIN:
+        pytest.skip("seed not certified")
+    hX, hL, hU = (torch.from_numpy(np.ascontiguousarray(a)) for a in (X, L, U))
+    hZ = torch.full((m, n), -5, dtype=torch.int32)
+    hE = torch.zeros((m, n), dtype=torch.float64)
+    hmargin = torch.zeros(1, dtype=torch.float64)
+    if pinned:
+        hX, hL, hU, hZ, hE, hmargin = (t.pin_memory() for t in (hX, hL, hU, hZ, hE, hmargin))
+    for rep in range(2):                      # the second call reuses the staging buffers of the first
+        hZ.fill_(-5)
+        g.gptq2d_round_host(hX, hL, hU, hZ=hZ, hE=hE, hmargin=hmargin)
+        assert np.array_equal(hZ.numpy().astype(np.int64), ref["Z"]), rep
+        assert abs(float(hmargin[0]) - margin) < 1e-9
+    Zd, Ed, _ = gpu_round(g, X, L, U)
+    assert np.array_equal(Zd, hZ.numpy())
+    assert np.array_equal(Ed, hE.numpy())
+
+
 # ------------------------------------------------------------------ error behaviour (host-made failures only)
 def test_argument_and_data_errors(g):
     X, A, B = W.general_bases(20, 30, 1)
