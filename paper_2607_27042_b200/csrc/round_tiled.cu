@@ -391,13 +391,23 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
     }
 
     // ---- 2. operands of the sweep
-    load_factor_block_async(Ls, p.L, p.ldl, p.m, row0, row0, 1);
-    load_factor_block_async(Us, p.U, p.ldu, p.n, col0, col0, 2);
+    // (the sweep reads the diagonal blocks below / above the diagonal only, so the 16-byte loader, which
+    // does not mask the other triangle, serves as well)
+    if (p.l_al16) load_full_block_async16(Ls, p.L, p.ldl, p.m, row0, row0);
+    else load_factor_block_async(Ls, p.L, p.ldl, p.m, row0, row0, 1);
+    if (p.u_al16) load_full_block_async16(Us, p.U, p.ldu, p.n, col0, col0);
+    else load_factor_block_async(Us, p.U, p.ldu, p.n, col0, col0, 2);
     load_quadrant_async(Cs, cQ, p.np);
     load_quadrant_async(Ys, eQ, p.np);
     // the operand of the first cross term that follows this quadrant
-    if (q == 0 || q == 2) load_factor_block_async(Xop, p.U, p.ldu, p.n, J * T, J * T + Q, 0);
-    if (q == 1) load_factor_block_async(Xop, p.L, p.ldl, p.m, I * T + Q, I * T, 0);
+    if (q == 0 || q == 2) {
+        if (p.u_al16) load_full_block_async16(Xop, p.U, p.ldu, p.n, J * T, J * T + Q);
+        else load_factor_block_async(Xop, p.U, p.ldu, p.n, J * T, J * T + Q, 0);
+    }
+    if (q == 1) {
+        if (p.l_al16) load_full_block_async16(Xop, p.L, p.ldl, p.m, I * T + Q, I * T);
+        else load_factor_block_async(Xop, p.L, p.ldl, p.m, I * T + Q, I * T, 0);
+    }
     cp_async_commit();
     double xv[16];
 #pragma unroll
@@ -436,7 +446,8 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
         cross_gemm(eT + (long)qi * Q * p.np + Q, p.np, Cs, Xop);
     if (q == 0) {
         __syncthreads();
-        load_factor_block_async(Xop, p.L, p.ldl, p.m, I * T + Q, I * T, 0);
+        if (p.l_al16) load_full_block_async16(Xop, p.L, p.ldl, p.m, I * T + Q, I * T);
+        else load_factor_block_async(Xop, p.L, p.ldl, p.m, I * T + Q, I * T, 0);
         cp_async_commit();
         cp_async_wait<0>();
         __syncthreads();
