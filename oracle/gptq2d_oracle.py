@@ -16,7 +16,11 @@ Pins (see tests/test_oracle_pins.py): brute-force conditional minimiser that use
 A and B only; closed forms for 1x1 / 2x2; F == U^T (x) L; B = I column
 independence and an elimination-form GPTQ; A = B = I round-to-nearest; the
 Kronecker-vec identity; transpose symmetry; mutual agreement of Algorithms
-1, 2, 3, 5, 6; the integer-matrix certificate.  No function here is unpinned.
+1, 2, 3, 5, 6; the integer-matrix certificate.  The reverse-order functions at the
+end (Section 2, "Two-sided and Kronecker-factored rounding": the same rounding
+taken from the last row and column) are pinned by their own brute force, by
+F~ == U~^T (x) L~ and by the index-reversal identity with the forward functions.
+No function here is unpinned.
 """
 from __future__ import annotations
 
@@ -30,6 +34,9 @@ __all__ = [
     "sweep_dense_antidiagonal", "sweep_gptq2d", "sweep_nested", "sweep_implicit_y",
     "brute_force_trajectory", "local_errors_from_Z", "certificate_margin",
     "objective", "objective_kron", "objective_from_errors", "gptq_one_sided_elimination",
+    "unit_upper_udu_of_inverse", "feedback_factors_reverse", "adaptive_round_1d_reverse",
+    "vec_sweep_reverse", "sweep_gptq2d_reverse", "brute_force_trajectory_reverse",
+    "certificate_margin_reverse",
 ]
 
 
@@ -329,3 +336,104 @@ def objective_from_errors(E, lamL, lamU):
 
 def _pack(Z, E):
     return {"Z": Z.astype(np.int64), "E": E, "margin": float(0.5 - np.max(np.abs(E))) if E.size else 0.5}
+
+
+# --------------------------------------------------------------------------- reverse order
+# Section 2 ("Two-sided and Kronecker-factored rounding"): the same greedy rounding taken in
+# reverse order, from the last row and column.  Coordinates of vec(X) are visited from the
+# last to the first; everything "lower" becomes "upper".
+def unit_upper_udu_of_inverse(S):
+    """S^{-1} = F lam F^T with F unit UPPER triangular (the factor Algorithm 1 needs when it
+    runs from the last coordinate to the first).  S = R^T R with R upper (ordinary Cholesky)
+    gives S^{-1} = R^{-1} R^{-T}, so F = R^{-1} diag(R) and lam = diag(R)^{-2}."""
+    S = np.asarray(S, dtype=np.float64)
+    R = np.linalg.cholesky(S).T
+    r = np.diag(R).copy()
+    F = sla.solve_triangular(R, np.diag(r), lower=False)
+    F = np.triu(F)
+    np.fill_diagonal(F, 1.0)
+    return F, 1.0 / (r * r)
+
+
+def feedback_factors_reverse(A, B):
+    """L~ unit upper with G^{-1} = L~ lam L~^T and U~ unit lower with H^{-1} = U~^T lam U~.
+    Returns (Lr, Ur, lamL, lamU)."""
+    G, H = gram_pair(A, B)
+    Lr, lamL = unit_upper_udu_of_inverse(G)
+    Urt, lamU = unit_upper_udu_of_inverse(H)
+    return Lr, Urt.T.copy(), lamL, lamU
+
+
+def adaptive_round_1d_reverse(x, F):
+    """Algorithm 1 run from the last coordinate to the first with a unit upper F:
+    z_k = round(y_k); E_k = z_k - y_k; y_{:k+1} += F_{:k+1,k} E_k."""
+    y = np.array(x, dtype=np.float64)
+    d = y.size
+    z = np.zeros(d)
+    E = np.zeros(d)
+    for k in range(d - 1, -1, -1):
+        z[k] = np.rint(y[k])
+        E[k] = z[k] - y[k]
+        y[:k + 1] += F[:k + 1, k] * E[k]
+    return z, E
+
+
+def vec_sweep_reverse(X, A, B):
+    """The definition: reverse Algorithm 1 on vec(X) under the explicit Kronecker Gram."""
+    X = np.asarray(X, dtype=np.float64)
+    m, n = X.shape
+    G, H = gram_pair(A, B)
+    F, _ = unit_upper_udu_of_inverse(kron_gram(G, H))
+    z, E = adaptive_round_1d_reverse(X.reshape(-1, order="F"), F)
+    return _pack(z.reshape(m, n, order="F"), E.reshape(m, n, order="F"))
+
+
+def sweep_gptq2d_reverse(X, Lr, Ur):
+    """Algorithm 3 mirrored for the reverse order: anti-diagonals from the last to the first;
+    every error is folded UP its column of C = L~ E and pushed up its column of Y through L~,
+    then C_ij is pushed LEFT along row i of Y through U~."""
+    Y = np.array(X, dtype=np.float64)
+    m, n = Y.shape
+    Z = np.zeros((m, n))
+    E = np.zeros((m, n))
+    C = np.zeros((m, n))
+    for s in range(m + n - 2, -1, -1):
+        idx = anti_diagonal(s, m, n)
+        for (i, j) in idx:
+            Z[i, j] = np.rint(Y[i, j])
+            E[i, j] = Z[i, j] - Y[i, j]
+            M = Lr[:i + 1, i] * E[i, j]
+            C[:i + 1, j] += M
+            Y[:i, j] += M[:i]
+        for (i, j) in idx:
+            Y[i, :j] += C[i, j] * Ur[j, :j]
+    return _pack(Z, E)
+
+
+def brute_force_trajectory_reverse(X, A, B):
+    """Reverse-order greedy trajectory from the objective alone: coordinates from the last to
+    the first; with the residuals of the already-rounded (later) coordinates fixed, minimise
+    || (B^T (x) A) r ||_2 over the real residuals of the remaining ones."""
+    X = np.asarray(X, dtype=np.float64)
+    m, n = X.shape
+    Mfull = np.kron(np.asarray(B, dtype=np.float64).T, np.asarray(A, dtype=np.float64))
+    x = X.reshape(-1, order="F")
+    d = m * n
+    r = np.zeros(d)
+    z = np.zeros(d)
+    for k in range(d - 1, -1, -1):
+        rhs = -Mfull[:, k + 1:] @ r[k + 1:]
+        sol, *_ = np.linalg.lstsq(Mfull[:, :k + 1], rhs, rcond=None)
+        z[k] = np.rint(x[k] + sol[k])
+        r[k] = z[k] - x[k]
+    return z.reshape(m, n, order="F")
+
+
+def certificate_margin_reverse(X, Z, Lr, Ur):
+    """The certificate for the reverse order: Z = X + L~ E U~, so E = L~^{-1} (Z - X) U~^{-1}
+    and Z is the reverse trajectory iff every |E_ij| < 1/2.  Returns (margin, E)."""
+    R = np.asarray(Z, dtype=np.float64) - np.asarray(X, dtype=np.float64)
+    T = sla.solve_triangular(Lr, R, lower=False, unit_diagonal=True)
+    Et = sla.solve_triangular(Ur.T, T.T, lower=False, unit_diagonal=True)
+    E = Et.T.copy()
+    return float(0.5 - np.max(np.abs(E))), E

@@ -279,3 +279,56 @@ def test_c1_quartic_sweep_and_its_reductions():
     Xi, Ai, Bi = W.make_config(1, seed=0, variant="A=B=I")
     Li, Ui, _, _ = O.feedback_factors(Ai, Bi)
     assert np.array_equal(cref.vec_sweep(Xi, Li, Ui)["Z"], np.rint(Xi).astype(np.int64))
+
+
+# ------------------------------------------------------------------ reverse order (Section 2, related work)
+@pytest.mark.parametrize("m,n,seed", [(1, 1, 0), (2, 2, 1), (3, 4, 2), (4, 3, 3), (1, 6, 4), (6, 1, 5), (4, 4, 6)])
+def test_reverse_order_trajectory_matches_its_brute_force(m, n, seed):
+    """The reverse-order rounding is pinned by a conditional least-squares brute force that uses A and
+    B only (no Gram, no factor), like the forward one; a wrong triangle, a wrong push direction or a
+    transposed factor changes Z."""
+    X, A, B = W.general_bases(m, n, seed)
+    Zb = O.brute_force_trajectory_reverse(X, A, B)
+    ref = O.vec_sweep_reverse(X, A, B)
+    if ref["margin"] < 1e-9:
+        pytest.skip("seed not certified")
+    assert np.array_equal(Zb, ref["Z"])
+    Lr, Ur, _, _ = O.feedback_factors_reverse(A, B)
+    out = O.sweep_gptq2d_reverse(X, Lr, Ur)
+    assert np.array_equal(out["Z"], ref["Z"])
+    assert np.max(np.abs(out["E"] - ref["E"])) < 1e-10
+
+
+def test_reverse_factors_are_unit_triangular_and_factor_the_inverse_grams():
+    X, A, B = W.general_bases(9, 7, 11)
+    Lr, Ur, lamL, lamU = O.feedback_factors_reverse(A, B)
+    G, H = O.gram_pair(A, B)
+    assert np.allclose(np.triu(Lr), Lr) and np.allclose(np.diag(Lr), 1.0)
+    assert np.allclose(np.tril(Ur), Ur) and np.allclose(np.diag(Ur), 1.0)
+    assert np.max(np.abs(Lr @ np.diag(lamL) @ Lr.T @ G - np.eye(9))) < 1e-9
+    assert np.max(np.abs(Ur.T @ np.diag(lamU) @ Ur @ H - np.eye(7))) < 1e-9
+    # Kronecker structure of the reverse feedback factor: F~ = U~^T (x) L~
+    F, _ = O.unit_upper_udu_of_inverse(O.kron_gram(G, H))
+    assert np.max(np.abs(F - np.kron(Ur.T, Lr))) < 1e-9
+
+
+@pytest.mark.parametrize("m,n,seed", [(5, 8, 0), (12, 12, 1), (20, 9, 2)])
+def test_reverse_order_is_the_forward_order_on_the_index_reversed_problem(m, n, seed):
+    """With P the index reversal: reverse(X; A, B) = P forward(P X P; A P, P B) P, and the reverse factors
+    are the reversed forward factors of the reversed bases.  This is what the CUDA path relies on."""
+    X, A, B = W.general_bases(m, n, seed)
+    Lr, Ur, _, _ = O.feedback_factors_reverse(A, B)
+    rev = O.sweep_gptq2d_reverse(X, Lr, Ur)
+    if rev["margin"] < 1e-9:
+        pytest.skip("seed not certified")
+    Lf, Uf, _, _ = O.feedback_factors(A[:, ::-1], B[::-1, :])
+    fwd = O.sweep_gptq2d(X[::-1, ::-1].copy(), Lf, Uf)
+    assert np.array_equal(fwd["Z"][::-1, ::-1], rev["Z"])
+    assert np.max(np.abs(Lf[::-1, ::-1] - Lr)) < 1e-12 and np.max(np.abs(Uf[::-1, ::-1] - Ur)) < 1e-12
+    # it is a different rounding from the forward one on the same inputs (so a no-op "reverse" fails)
+    L, U, _, _ = O.feedback_factors(A, B)
+    assert not np.array_equal(O.sweep_gptq2d(X, L, U)["Z"], rev["Z"])
+    margin, E = O.certificate_margin_reverse(X, rev["Z"], Lr, Ur)
+    assert abs(margin - rev["margin"]) < 1e-10 and np.max(np.abs(E - rev["E"])) < 1e-9
+    bad = rev["Z"].copy(); bad[m // 2, n // 2] += 1
+    assert O.certificate_margin_reverse(X, bad, Lr, Ur)[0] < 0
