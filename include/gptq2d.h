@@ -178,6 +178,33 @@ int gptq2d_round_static(int m, int n,
                         int *info, void *stream);
 size_t gptq2d_round_static_max_dim(void);
 
+/* ---- reverse order (Section 2, "Two-sided and Kronecker-factored rounding": the same greedy
+ * rounding "in reverse order, from the last row and column") ----
+ * Coordinates of vec(X) are visited from the last to the first.  The feedback factors become
+ *   Lr (m x m): unit UPPER triangular, (A^T A)^{-1} = Lr Lambda Lr^T,
+ *   Ur (n x n): unit LOWER triangular, (B B^T)^{-1} = Ur^T Lambda Ur,
+ * and the sweep runs over the anti-diagonals from the last to the first, pushing up and to the left.
+ * With P the index reversal this is the forward problem on (P X P; A P, P B); both calls reverse
+ * their operands into the workspace, run the forward kernels and reverse the results back, so Z, E,
+ * min_margin, dL, dU are in the caller's own indexing.  Only the device status words are not
+ * translated: a row / column / pivot index k reported in `info` is m-1-k (n-1-k) in the caller's
+ * indexing.  Argument rules, status codes and stream behaviour are those of gptq2d_factor /
+ * gptq2d_round (fp64 tiled sweep).
+ */
+size_t gptq2d_factor_reverse_workspace_bytes(int m, int n);
+int gptq2d_factor_reverse(int m, int n,
+                          const double *A, long lda, const double *B, long ldb,
+                          double *Lr, long ldl, double *Ur, long ldu,
+                          double *dL, double *dU,
+                          void *workspace, size_t workspace_bytes, int *info, void *stream);
+size_t gptq2d_round_reverse_workspace_bytes(int m, int n);
+int gptq2d_round_reverse(int m, int n,
+                         const double *X, long ldx,
+                         const double *Lr, long ldl, const double *Ur, long ldu,
+                         int32_t *Z, long ldz,
+                         double *E, long lde, double *min_margin,
+                         void *workspace, size_t workspace_bytes, int *info, void *stream);
+
 /* ---- the objective (Eq. 7): obj = || A (Z - X) B ||_F^2 ----
  * obj: device scalar.  A or B may be NULL (identity).
  */

@@ -31,6 +31,8 @@ EXPORTS = (
     "gptq2d_round_host", "gptq2d_objective_workspace_bytes", "gptq2d_objective",
     "gptq2d_round_static", "gptq2d_round_static_max_dim",
     "gptq2d_round_batched_workspace_bytes", "gptq2d_round_batched",
+    "gptq2d_factor_reverse_workspace_bytes", "gptq2d_factor_reverse",
+    "gptq2d_round_reverse_workspace_bytes", "gptq2d_round_reverse",
 )
 
 BATCH_MAX_COUNT, BATCH_MAX_DIM = 8192, 32768
@@ -82,6 +84,13 @@ def _load():
     lib.gptq2d_round_static.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, vp]
     lib.gptq2d_round_static_max_dim.restype = sz
     lib.gptq2d_round_static_max_dim.argtypes = []
+    for name in ("gptq2d_factor_reverse_workspace_bytes", "gptq2d_round_reverse_workspace_bytes"):
+        getattr(lib, name).restype = sz
+        getattr(lib, name).argtypes = [i32, i32]
+    lib.gptq2d_factor_reverse.restype = i32
+    lib.gptq2d_factor_reverse.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, vp, sz, vp, vp]
+    lib.gptq2d_round_reverse.restype = i32
+    lib.gptq2d_round_reverse.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, sz, vp, vp]
     lib.gptq2d_round_batched_workspace_bytes.restype = sz
     lib.gptq2d_round_batched_workspace_bytes.argtypes = [i32, vp]
     lib.gptq2d_round_batched.restype = i32
@@ -191,6 +200,61 @@ def gptq2d_round(X, L, U, Z=None, E=None, min_margin=None, precision=FP64, works
     pE, lde = _mat(E, torch.float64, "E")
     st = _lib.gptq2d_round(m, n, pX, ldx, pL, ldl, pU, ldu, pZ, ldz, pE, lde, _ptr(min_margin), int(precision),
                            _ptr(workspace), workspace.numel(), _ptr(info), _stream_ptr(stream))
+    if st != OK:
+        raise Gptq2dError(st)
+    return Z, E, min_margin, info
+
+
+def gptq2d_factor_reverse_workspace_bytes(m, n):
+    return int(_lib.gptq2d_factor_reverse_workspace_bytes(m, n))
+
+
+def gptq2d_round_reverse_workspace_bytes(m, n):
+    return int(_lib.gptq2d_round_reverse_workspace_bytes(m, n))
+
+
+def gptq2d_factor_reverse(A, B, Lr=None, Ur=None, dL=None, dU=None, workspace=None, info=None, stream=None,
+                          m=None, n=None):
+    """Factors for the reverse order: Lr unit upper, Ur unit lower.  Returns (Lr, Ur, dL, dU, info)."""
+    m = A.shape[0] if A is not None else m
+    n = B.shape[0] if B is not None else n
+    dev = (A if A is not None else B).device if (A is not None or B is not None) else torch.device("cuda")
+    Lr = torch.empty((m, m), dtype=torch.float64, device=dev) if Lr is None else Lr
+    Ur = torch.empty((n, n), dtype=torch.float64, device=dev) if Ur is None else Ur
+    dL = torch.empty(m, dtype=torch.float64, device=dev) if dL is None else dL
+    dU = torch.empty(n, dtype=torch.float64, device=dev) if dU is None else dU
+    info = torch.zeros(4, dtype=torch.int32, device=dev) if info is None else info
+    workspace = _workspace(gptq2d_factor_reverse_workspace_bytes(m, n), dev) if workspace is None else workspace
+    pA, lda = _mat(A, torch.float64, "A")
+    pB, ldb = _mat(B, torch.float64, "B")
+    pL, ldl = _mat(Lr, torch.float64, "Lr")
+    pU, ldu = _mat(Ur, torch.float64, "Ur")
+    st = _lib.gptq2d_factor_reverse(m, n, pA, lda, pB, ldb, pL, ldl, pU, ldu, _ptr(dL), _ptr(dU),
+                                    _ptr(workspace), workspace.numel(), _ptr(info), _stream_ptr(stream))
+    if st != OK:
+        raise Gptq2dError(st)
+    return Lr, Ur, dL, dU, info
+
+
+def gptq2d_round_reverse(X, Lr, Ur, Z=None, E=None, min_margin=None, workspace=None, info=None, stream=None,
+                         want_E=False, want_margin=False):
+    """The sweep in reverse order (from the last row and column).  Returns (Z, E, min_margin, info)."""
+    m, n = X.shape
+    dev = X.device
+    Z = torch.empty((m, n), dtype=torch.int32, device=dev) if Z is None else Z
+    if E is None and want_E:
+        E = torch.empty((m, n), dtype=torch.float64, device=dev)
+    if min_margin is None and want_margin:
+        min_margin = torch.empty(1, dtype=torch.float64, device=dev)
+    info = torch.zeros(4, dtype=torch.int32, device=dev) if info is None else info
+    workspace = _workspace(gptq2d_round_reverse_workspace_bytes(m, n), dev) if workspace is None else workspace
+    pX, ldx = _mat(X, torch.float64, "X")
+    pL, ldl = _mat(Lr, torch.float64, "Lr")
+    pU, ldu = _mat(Ur, torch.float64, "Ur")
+    pZ, ldz = _mat(Z, torch.int32, "Z")
+    pE, lde = _mat(E, torch.float64, "E")
+    st = _lib.gptq2d_round_reverse(m, n, pX, ldx, pL, ldl, pU, ldu, pZ, ldz, pE, lde, _ptr(min_margin),
+                                   _ptr(workspace), workspace.numel(), _ptr(info), _stream_ptr(stream))
     if st != OK:
         raise Gptq2dError(st)
     return Z, E, min_margin, info
