@@ -162,7 +162,7 @@ def run_cuda(args):
     g.check_info(finfo)
     del fws
 
-    precision = g.FP32 if args.fp32 else g.FP64
+    precision = g.FP32 if args.fp32 else (g.FP64_PULL if args.pull else g.FP64)
     ws = torch.empty(g.gptq2d_round_workspace_bytes(m, n, precision), dtype=torch.uint8, device="cuda")
     Z = torch.empty((m, n), dtype=torch.int32, device="cuda")
     info = torch.zeros(4, dtype=torch.int32, device="cuda")
@@ -278,6 +278,14 @@ def run_cuda(args):
                             "objective_fp32": o32, "objective_fp64": o64, "relative_objective_gap": (o32 - o64) / o64}
         out["roofline"]["kernel"] = "round_untiled_kernel<float>"
         out["roofline"]["bound"] = "hbm"
+    if args.pull:
+        # every entry streams 2 (i + j) words: 8 m n (m + n) bytes in all
+        pull_bytes = 8.0 * m * n * (m + n)
+        gbs = pull_bytes / (kernel_ms * 1e-3) / 1e9
+        out["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                           "frac": gbs / peaks["hbm_gbs"], "traffic": None, "kernel": "round_pull_kernel",
+                           "kernel_ms": kernel_ms, "bytes_per_launch": pull_bytes,
+                           "note": "algorithmic bytes of the pull form, 8 m n (m + n); part of them hit in L2"}
     if not args.no_cpu:
         out["cpu_baseline"], out["cpu_gptq2d"] = cpu_baseline(X, A, B, budget_s=args.cpu_seconds)
     print(json.dumps(out))
@@ -483,6 +491,8 @@ def main():
     ap.add_argument("--config", type=int, default=4, help="configuration index 0..4 (4 = 8192 x 8192 headline)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--fp32", action="store_true", help="time the fp32 mode instead")
+    ap.add_argument("--pull", action="store_true",
+                    help="time the untiled pull-form kernel (Algorithm 6) instead: the memory-bound comparison point")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)

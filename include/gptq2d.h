@@ -53,7 +53,10 @@ typedef enum {
     GPTQ2D_FP64 = 0,   /* all sweep arithmetic in fp64 (tiled wavefront kernel)                       */
     GPTQ2D_FP32 = 1,   /* X, L, U rounded to fp32 and all sweep arithmetic in fp32 (Algorithm 3 as
                           written, one grid-wide barrier per anti-diagonal); Z may differ from FP64  */
-    GPTQ2D_FP64_UNTILED = 2 /* fp64 with the untiled Algorithm-3 kernel; a cross-check, not fast      */
+    GPTQ2D_FP64_UNTILED = 2, /* fp64 with the untiled Algorithm-3 kernel; a cross-check, not fast     */
+    GPTQ2D_FP64_PULL = 3    /* fp64, implicit-Y form (Algorithm 6, Eq. 19-20) with C pulled as well: every
+                               entry reconstructs its corrected value from L, E, C, U at rounding time;
+                               untiled and bound by memory bandwidth: the comparison point, not fast   */
 } gptq2d_precision_t;
 
 /* Human-readable name of a status code (static storage). */

@@ -132,6 +132,7 @@ size_t gptq2d_round_workspace_bytes(int m, int n, int precision) {
     if (precision == GPTQ2D_FP64) return round_tiled_workspace_bytes(m, n);
     if (precision == GPTQ2D_FP32) return round_untiled_workspace_bytes(m, n, true);
     if (precision == GPTQ2D_FP64_UNTILED) return round_untiled_workspace_bytes(m, n, false);
+    if (precision == GPTQ2D_FP64_PULL) return round_pull_workspace_bytes(m, n);
     return 0;
 }
 
@@ -144,7 +145,8 @@ int gptq2d_round(int m, int n, const double *X, long ldx, const double *L, long 
     if (!aligned(X, 8) || !aligned(L, 8) || !aligned(U, 8) || !aligned(Z, 4) || !aligned(E, 8) ||
         !aligned(min_margin, 8))
         return GPTQ2D_ERR_INVALID_ARG;
-    if (precision != GPTQ2D_FP64 && precision != GPTQ2D_FP32 && precision != GPTQ2D_FP64_UNTILED)
+    if (precision != GPTQ2D_FP64 && precision != GPTQ2D_FP32 && precision != GPTQ2D_FP64_UNTILED &&
+        precision != GPTQ2D_FP64_PULL)
         return GPTQ2D_ERR_INVALID_ARG;
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < gptq2d_round_workspace_bytes(m, n, precision))
         return GPTQ2D_ERR_WORKSPACE;
@@ -158,6 +160,12 @@ int gptq2d_round(int m, int n, const double *X, long ldx, const double *L, long 
         p.X = X; p.ldx = ldx; p.L = L; p.ldl = ldl; p.U = U; p.ldu = ldu;
         p.Z = Z; p.ldz = ldz; p.E = E; p.lde = lde; p.info = info;
         st = launch_round_tiled(p, workspace, workspace_bytes, stream);
+    } else if (precision == GPTQ2D_FP64_PULL) {
+        PullParams p{};
+        p.m = m; p.n = n;
+        p.X = X; p.ldx = ldx; p.L = L; p.ldl = ldl; p.U = U; p.ldu = ldu;
+        p.Z = Z; p.ldz = ldz; p.E = E; p.lde = lde; p.info = info;
+        st = launch_round_pull(p, workspace, stream);
     } else {
         UntiledParams p{};
         p.m = m; p.n = n;

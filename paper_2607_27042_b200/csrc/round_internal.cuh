@@ -20,6 +20,21 @@ struct UntiledParams {
 size_t round_untiled_workspace_bytes(int m, int n, bool fp32);
 int launch_round_untiled(const UntiledParams &p, bool fp32, void *ws, cudaStream_t stream);
 
+struct PullParams {
+    int m, n;
+    const double *X; long ldx;
+    const double *L; long ldl;
+    const double *U; long ldu;
+    int *Z; long ldz;
+    double *E; long lde;      // optional
+    double *max_abs_e;
+    int *info;
+    double *C, *Et, *Ut;      // workspace: C = L E (m x n), E transposed (n x m), U transposed (n x n)
+    GridSync sync;
+};
+size_t round_pull_workspace_bytes(int m, int n);
+int launch_round_pull(const PullParams &p, void *ws, cudaStream_t stream);
+
 struct TiledParams {
     int m, n;
     const double *X; long ldx;

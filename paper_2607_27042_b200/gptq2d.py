@@ -16,7 +16,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libgptq2d.so")
 
-FP64, FP32, FP64_UNTILED = 0, 1, 2
+FP64, FP32, FP64_UNTILED, FP64_PULL = 0, 1, 2, 3
 
 OK = 0
 STATUS_NAMES = {

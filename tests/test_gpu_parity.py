@@ -51,7 +51,7 @@ def oracle_small(X, L, U):
 
 
 # ------------------------------------------------------------------ the sweep, oracle factors
-@pytest.mark.parametrize("precision", [0, 2])
+@pytest.mark.parametrize("precision", [0, 2, 3])
 @pytest.mark.parametrize("m,n,seed", [(1, 1, 0), (1, 9, 1), (9, 1, 2), (8, 8, 3), (17, 5, 4), (64, 64, 5),
                                       (65, 63, 6), (100, 130, 7), (129, 257, 8), (200, 75, 9)])
 def test_sweep_small_and_ragged_general_bases(g, m, n, seed, precision):
@@ -71,7 +71,7 @@ def test_c0_bit_exact_against_explicit_kronecker_oracle(g):
     ref = O.vec_sweep_explicit(X, A, B)           # the definition, 4096 x 4096 Kronecker Gram
     assert ref["margin"] >= MARGIN
     L, U, _, _ = O.feedback_factors(A, B)
-    for precision in (0, 2):
+    for precision in (0, 2, 3):
         Z, E, mm = gpu_round(g, X, L, U, precision)
         assert np.array_equal(Z, ref["Z"])
     # end to end with the library's own factors
@@ -98,7 +98,7 @@ def test_c1_bit_exact_and_reductions(g, variant):
         assert np.array_equal(ref["Z"], np.rint(X).astype(np.int64))
     if variant == "B=I":
         assert torch.equal(Ud.cpu(), torch.eye(256, dtype=torch.float64))
-    for precision in (0, 2):
+    for precision in (0, 2, 3):
         Z, E, mm, info = g.gptq2d_round(dev(X), Ld, Ud, precision=precision, want_E=True, want_margin=True)
         torch.cuda.synchronize()
         g.check_info(info)
@@ -172,8 +172,9 @@ def test_mid_size_against_nested_oracle_and_certificate(g, name, make):
     # two runs and the untiled kernel must agree bit for bit (a missing fence would not)
     Z2, _, _, _ = g.gptq2d_round(dev(X), Ld, Ud)
     Z3, _, _, _ = g.gptq2d_round(dev(X), Ld, Ud, precision=2)
+    Z4, _, _, _ = g.gptq2d_round(dev(X), Ld, Ud, precision=3)          # pull form (Algorithm 6)
     torch.cuda.synchronize()
-    assert torch.equal(Z, Z2) and torch.equal(Z, Z3)
+    assert torch.equal(Z, Z2) and torch.equal(Z, Z3) and torch.equal(Z, Z4)
 
 
 # ------------------------------------------------------------------ thin shapes: one row / one column of tiles
