@@ -7,6 +7,7 @@
 
 namespace gptq2d {
 size_t factor_workspace_bytes(int m, int n);
+size_t factor_side_workspace_bytes(int k);
 int factor_one_side(int k, const double *M, long ldm, int side, double *out, long ldo, double *dinv, void *ws,
                     int *info, cudaStream_t stream);
 size_t objective_workspace_bytes(int m, int n);
@@ -26,9 +27,10 @@ static int check_device() {
 
 static size_t pad256(size_t x) { return (x + 255) / 256 * 256; }
 
-// ---- helpers of the pipelined host entry point ------------------------------------------------
-// A second stream (per device, created on first use) carries the host-to-device copies while the
-// sweep kernel already runs on the caller's stream; the copy stream announces each 128-row panel
+// ---- the library's second stream ---------------------------------------------------------------
+// A second stream (per device, created on first use).  In the host entry point it carries the
+// host-to-device copies while the sweep kernel already runs on the caller's stream; in gptq2d_factor
+// it carries the B side.  In the host entry point the copy stream announces each 128-row panel
 // with a stream-ordered 32-bit write (driver entry point looked up through the runtime, so the
 // library has no link-time dependency on the driver library).
 typedef int (*StreamWriteValue32Fn)(cudaStream_t, unsigned long long, unsigned int, unsigned int);
@@ -122,9 +124,27 @@ int gptq2d_factor(int m, int n, const double *A, long lda, const double *B, long
     int st = check_device();
     if (st != GPTQ2D_OK) return st;
     if (info && cudaMemsetAsync(info, 0, 4 * sizeof(int), stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+    // The two sides are independent.  Each has a serial spine (one small diagonal-block kernel per 128
+    // rows, between the panel and trailing updates) that leaves most SMs idle, so the B side runs on a
+    // second stream and its GEMMs fill the gaps of the A side and vice versa.
+    char *wsB = static_cast<char *>(workspace) + factor_side_workspace_bytes(m);
+    HostPipe *hp = (A && B) ? host_pipe() : nullptr;
+    if (!hp) {
+        st = factor_one_side(m, A, lda, 0, L, ldl, dL, workspace, info, stream);
+        if (st != GPTQ2D_OK) return st;
+        return factor_one_side(n, B, ldb, 1, U, ldu, dU, wsB, info, stream);
+    }
+    std::unique_lock<std::mutex> lock(hp->enqueue);
+    if (cudaEventRecord(hp->inputs_free, stream) != cudaSuccess ||
+        cudaStreamWaitEvent(hp->copy, hp->inputs_free, 0) != cudaSuccess)
+        return GPTQ2D_ERR_CUDA;
     st = factor_one_side(m, A, lda, 0, L, ldl, dL, workspace, info, stream);
-    if (st != GPTQ2D_OK) return st;
-    return factor_one_side(n, B, ldb, 1, U, ldu, dU, workspace, info, stream);
+    int st2 = factor_one_side(n, B, ldb, 1, U, ldu, dU, wsB, info, hp->copy);
+    // join even if an enqueue failed, so that nothing of this call is left running behind the caller's stream
+    if (cudaEventRecord(hp->copies_done, hp->copy) != cudaSuccess ||
+        cudaStreamWaitEvent(stream, hp->copies_done, 0) != cudaSuccess)
+        return GPTQ2D_ERR_CUDA;
+    return st != GPTQ2D_OK ? st : st2;
 }
 
 size_t gptq2d_round_workspace_bytes(int m, int n, int precision) {

@@ -143,12 +143,15 @@ __global__ void identity_kernel(double *out, long ldo, int k, double *dinv) {
 
 static inline long round_up(long x, long a) { return (x + a - 1) / a * a; }
 
-size_t factor_workspace_bytes(int m, int n) {
-    long k = m > n ? m : n;
+// one side: three k x k matrices (Gram / Cholesky factor, its inverse, a product buffer) and the pivots
+size_t factor_side_workspace_bytes(int k) {
     long ld = round_up(k, 16);
     size_t mat = (size_t)ld * (size_t)round_up(k, 16) * sizeof(double);
-    return 3 * mat + (size_t)round_up(k, 32) * sizeof(double) + 256;
+    size_t b = 3 * mat + (size_t)round_up(k, 32) * sizeof(double) + 256;
+    return (b + 255) / 256 * 256;
 }
+// the two sides are factorised at the same time (two streams), each in its own part of the workspace
+size_t factor_workspace_bytes(int m, int n) { return factor_side_workspace_bytes(m) + factor_side_workspace_bytes(n); }
 
 #define CK(x)                                          \
     do {                                               \
