@@ -263,6 +263,30 @@ def test_host_entry_streams_inputs_while_sweeping(g, m, n, seed, pinned):
     assert np.array_equal(Ed, hE.numpy())
 
 
+def test_two_streams_two_workspaces(g):
+    """Calls on different streams with their own workspaces may be in flight together (the persistent
+    launches take turns on the device); neither disturbs the other's result."""
+    cases = []
+    for (m, n, seed) in [(300, 515, 41), (515, 300, 42)]:
+        X, A, B = W.general_bases(m, n, seed)
+        L, U, _, _ = O.feedback_factors(A, B)
+        ref = cref.nested(X, L, U)
+        cases.append((dev(X), dev(L), dev(U), ref["Z"], O.certificate_margin(X, ref["Z"], L, U)[0]))
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    outs = []
+    for rep in range(3):
+        for (dX, dL, dU, _, _), st in zip(cases, streams):
+            with torch.cuda.stream(st):
+                outs.append(g.gptq2d_round(dX, dL, dU, stream=st))
+    torch.cuda.synchronize()
+    for k, (Z, _, _, info) in enumerate(outs):
+        g.check_info(info)
+        _, _, _, Zref, margin = cases[k % 2]
+        if margin >= MARGIN:
+            assert np.array_equal(Z.cpu().numpy().astype(np.int64), Zref)
+
+
 # ------------------------------------------------------------------ error behaviour (host-made failures only)
 def test_argument_and_data_errors(g):
     X, A, B = W.general_bases(20, 30, 1)
