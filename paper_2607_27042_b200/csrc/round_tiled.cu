@@ -15,16 +15,22 @@
 //    counter.  A far part waits (bounded) only on tiles two or more waves back, parks its
 //    partial sum in the tile's own workspace region and then announces it to the tile's four
 //    quadrant tasks.  This is >90 % of the flops and runs on the fp64 tensor path.
-//  * QUADRANT tasks (64 x 64), the critical path.  A quadrant pulls the adjacent tiles'
-//    contributions itself (four 64^3 DMMA products), sweeps, and adds its cross terms to the
-//    later quadrants of its tile.  It counts arrivals from exactly what it needs -- the two
-//    far parts of its tile, the two quadrants above that share its columns, the two quadrants
-//    to the left that share its rows, its predecessors inside the tile -- and the last arrival
-//    puts it on a global ready ring.  Quadrant tasks never wait.
+//  * QUADRANT tasks (64 x 64), the critical path.  In the grid of quadrants, (r, c) needs all
+//    quadrants above it in its column and to its left in its row.  What complete quadrants of the
+//    adjacent tiles (and of its own tile) contribute it pulls itself when it starts (up to four
+//    64^3 DMMA products).  The quadrant right above and the one right to the left are NOT waited
+//    for: every quadrant publishes its 8 x 8 leaves leaf-wave by leaf-wave (results to the
+//    workspace, a progress word per quadrant), and its two neighbours take them in as they come,
+//    running nine leaf-waves behind (block b of a neighbour is final after its leaf-wave 7 + b).
+//    A task counts arrivals from the two far parts of its tile, from (r-2, c) and (r, c-2) being
+//    complete, and from (r-1, c) and (r, c-1) having reached their third leaf-wave; the last arrival
+//    puts it on a global ready ring.  A running quadrant task waits -- bounded -- only on its two
+//    neighbours, which are running by then (or done).
 // Every CTA serves the ready ring first: at the top of its loop, while a far part waits, and
 // every few chunks of a far part (it then parks its partial sum and un-parks it afterwards).
 // A far part only ever waits on tiles of earlier waves, whose far parts were claimed earlier and
-// whose quadrant tasks never wait, so the earliest unfinished work can always progress.
+// whose quadrant tasks wait on running tasks only, so the earliest unfinished work can always
+// progress.
 //
 // In-tile sweep.  Inside a quadrant the anti-diagonal sweep runs on 8 x 8 leaves: each leaf of a
 // leaf-wave is swept by one warp (two entries per lane, errors exchanged through a 16-double
@@ -60,6 +66,7 @@ struct TiledKernelParams {
     unsigned *flagS;             // [ntm*ntn] tile swept
     unsigned *quad_done;         // [ntm*ntn] swept quadrants of the tile (4 -> tile flag)
     unsigned *qdep;              // [ntm*ntn][4] arrivals each quadrant task has received
+    unsigned *qprog;             // [ntm*ntn][4] leaf-waves each quadrant has published (15: complete)
     double *max_abs_e;
     int *info;
     int l_al16, u_al16;
@@ -74,12 +81,12 @@ struct TiledKernelParams {
 };
 static_assert(sizeof(TiledKernelParams) % 8 == 0, "descriptors are copied as 8-byte words");
 
-constexpr size_t SWEEP_SMEM = (size_t)(5 * QMAT + 2 * Q * TAB_LD) * sizeof(double) + (size_t)Q * Q * sizeof(int);
+constexpr size_t SWEEP_SMEM = (size_t)(5 * QMAT + 2 * Q * TAB_LD + 2 * (64 * 12) + 2 * (8 * QLD)) * sizeof(double);
 constexpr size_t BULK_SMEM = (size_t)BULK_NSTAGE * SlabLayout<true, false>::STAGE_DOUBLES * sizeof(double);
 constexpr size_t TILED_SMEM = SWEEP_SMEM > BULK_SMEM ? SWEEP_SMEM : BULK_SMEM;
 
 // ---------------------------------------------------------------------------------------------
-// quadrant <-> shared memory.  The *_async loaders only issue cp.async copies; the caller
+// workspace / factors -> shared memory.  The *_async loaders only issue cp.async copies; the caller
 // commits, waits and barriers once for all operands of a quadrant.
 __device__ __forceinline__ void load_quadrant_async(double *dst, const double *src, long ld) {
     // dense 64 x 64 from a padded workspace buffer (always in range, 16-byte aligned); L2 only
@@ -87,14 +94,6 @@ __device__ __forceinline__ void load_quadrant_async(double *dst, const double *s
     for (int it = 0; it < 8; ++it) {
         int c = threadIdx.x + it * TILED_THREADS;
         cp_async16(dst + (c >> 5) * QLD + (c & 31) * 2, src + (long)(c >> 5) * ld + (c & 31) * 2, 16);
-    }
-}
-__device__ __forceinline__ void store_quadrant(double *dst, long ld, const double *src) {
-#pragma unroll
-    for (int it = 0; it < 8; ++it) {
-        int c = threadIdx.x + it * TILED_THREADS;
-        int r = c >> 5, cc = (c & 31) * 2;
-        *reinterpret_cast<double2 *>(dst + (long)r * ld + cc) = *reinterpret_cast<const double2 *>(src + r * QLD + cc);
     }
 }
 // 64 x 64 block of a user matrix (k x k, leading dimension ld) whose top-left element is
@@ -169,14 +168,6 @@ __device__ __forceinline__ void quad_add_to(double *D, long ld, const QAcc &acc,
             *ptr = v;
         }
 }
-// G (global 64 x 64, row stride ld) += As (64 x 64, [m][k]) * Bs (64 x 64, [k][n])
-__device__ __forceinline__ void cross_gemm(double *G, long ld, const double *As, const double *Bs) {
-    QAcc acc;
-    acc.zero();
-    quad_mma(acc, As, Bs);
-    quad_add_to(G, ld, acc, true);
-}
-
 // Leaf (a, b) of the quadrant collects, right before it is swept, all the feedback it is due from
 // the leaves already swept (left-looking): the downward pushes of the leaves above it through L,
 //     P = sum_{a' < a} L[a, a'] E[a', b]       (folded into C and pushed into Y)
@@ -213,24 +204,70 @@ __device__ __forceinline__ void leaf_pull(double *Ys, double *Cs, const double *
 }
 
 // ---------------------------------------------------------------------------------------------
+// Streaming between neighbouring quadrants.  A quadrant does not wait for the quadrant above it
+// (and the one to its left) to finish: column block b of the E above is final once that quadrant
+// has swept its leaf-waves 0 .. 7+b, row block a of the C to the left once leaf-waves 0 .. 7+a are
+// done, and leaf-wave lw of this quadrant needs exactly blocks 0 .. lw of both.  Every quadrant
+// therefore publishes its leaves wave by wave (E, C to the workspace, a progress word per
+// quadrant), and its two neighbours run nine leaf-waves behind it.
+constexpr int STG_E_LD = 12;                 // staged 64 x 8 column block of E, [k][n], 12 = 8 + 4 pad
+constexpr int STG_E = Q * STG_E_LD;          // doubles per staged E block
+constexpr int STG_C = 8 * QLD;               // staged 8 x 64 row block of C, [m][k]
+constexpr int GO_WAVE = 2;                   // a quadrant lets its two neighbours start at this leaf-wave
+
+struct Stream {
+    const unsigned *prog_above, *prog_left;  // progress words of the two neighbours (NULL: none)
+    unsigned *prog_self;
+    const double *e_above;                   // Ebuf at (first row of the quadrant above, first column of this one)
+    const double *c_left;                    // Cbuf at (first row of this quadrant, first column of the one to the left)
+    int I, J, q;
+};
+
+// Called by one warp: lane 0 polls both neighbours' progress words until each has reached `need`
+// (bounded; on expiry the launch is aborted and the caller carries on with whatever is there).
+__device__ __forceinline__ void await_progress(const TiledKernelParams &p, const unsigned *wa, const unsigned *wl,
+                                               unsigned need) {
+    if ((threadIdx.x & 31) == 0) {
+        unsigned long long it = 0;
+        for (;;) {
+            const unsigned va = wa ? ld_acquire_u32(wa) : need, vl = wl ? ld_acquire_u32(wl) : need;
+            if (va >= need && vl >= need) break;
+            if (++it > SPIN_LIMIT || ld_relaxed_u32(p.abort) != 0u) {
+                report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -8, (int)need, (int)blockIdx.x);
+                atomicExch(p.abort, 1u);
+                break;
+            }
+            __nanosleep(40);
+        }
+    }
+    __syncwarp();
+}
+
+__device__ __forceinline__ void quadrant_arrive(const TiledKernelParams &p, int I, int J, int q);
+
 // Algorithm 3 on one 64 x 64 quadrant held in shared memory.
-//   Ys: in  Y (corrected values, already including the C the quadrant starts with)
-//       out E (local errors)
-//   Cs: in  C at entry; out final C = L E rows of the quadrant
-//   Ls / Us: strictly lower / strictly upper 64 x 64 diagonal blocks of the factors
-//   Zs: out rounded integers
-// row0/col0: global coordinates of the quadrant (for masking the status checks).
+//   Ys: in  Y (corrected values from everything but the two streaming neighbours); out E
+//   Cs: in  C likewise; out final C = L E rows of the quadrant
+//   LU: the 64 x 64 diagonal blocks of both factors in one matrix: strictly lower part from L,
+//       strictly upper part from U (the sweep never reads the other triangles)
+//   Lfa: L[rows of this quadrant, rows of the quadrant above];  Ufl: U[columns of the quadrant to
+//        the left, columns of this quadrant]
+//   stg: staging for the streamed blocks, two of each kind
+// row0/col0: global coordinates of the quadrant.
 //
-// Leaf-wave lw (leaves (a, lw - a), one per warp): every leaf first pulls the feedback of the
-// leaves swept before it (leaf_pull), then runs the 15 anti-diagonal steps on its 8 x 8 entries.
-// One CTA barrier per leaf-wave.
-__device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const double *Ls, const double *Us, int *Zs,
-                                               double *tabL, double *tabU, int row0, int col0,
-                                               const TiledKernelParams &p, double &max_abs_e) {
+// Leaf-wave lw (leaves (a, lw - a), one per warp).  For lw <= 7, all warps first add what block lw
+// of the neighbours feeds into this quadrant (pull phase), and request block lw + 1.  Then every
+// leaf pulls the feedback of the leaves swept before it (leaf_pull), runs the 15 anti-diagonal
+// steps on its 8 x 8 entries and stores its results.
+__device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const double *LU, const double *Lfa,
+                                               const double *Ufl, double *stg, double *tabL, double *tabU, int row0,
+                                               int col0, const Stream &sm, const TiledKernelParams &p,
+                                               double &max_abs_e) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, t = lane & 3;
     __shared__ double xch[8 * 2 * 16];
     __shared__ unsigned long long s_badkey;
+    const double *Ls = LU, *Us = LU;
     // coefficient tables of the 8 diagonal leaves (see phase A); also clears the exchange buffers
     for (int c = tid; c < Q * TAB_LD; c += blockDim.x) {
         const int r = c / TAB_LD, k = c - r * TAB_LD;       // r: row (L) or column (U) inside the quadrant
@@ -242,9 +279,87 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
     if (tid < 8 * 2 * 16) xch[tid] = 0.0;
     if (tid == 0) s_badkey = ~0ull;
     unsigned long long badkey = ~0ull;
+    const bool fresh = sm.prog_above != nullptr || sm.prog_left != nullptr;
+    double *stgE = stg, *stgC = stg + 2 * STG_E;
+    // Warp 7 (idle in every leaf-wave but the eighth) is the streaming warp: it fetches the next block of
+    // the neighbours' results while the other warps sweep their leaves: 8 + 8 pieces of 16 bytes per lane.
+    auto fetch_block = [&](int blk) {
+        await_progress(p, sm.prog_above, sm.prog_left, (unsigned)(blk + 8));
+        if (sm.prog_above) {        // E above: 64 rows x 8 columns [8 blk, 8 blk + 8)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int piece = lane + 32 * i, r = piece >> 2, c2 = (piece & 3) * 2;
+                cp_async16(stgE + (blk & 1) * STG_E + r * STG_E_LD + c2, sm.e_above + (long)r * p.np + blk * 8 + c2, 16);
+            }
+        }
+        if (sm.prog_left) {         // C to the left: rows [8 blk, 8 blk + 8) x 64 columns
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int piece = lane + 32 * i, r = piece >> 5, c2 = (piece & 31) * 2;
+                cp_async16(stgC + (blk & 1) * STG_C + r * QLD + c2, sm.c_left + (long)(blk * 8 + r) * p.np + c2, 16);
+            }
+        }
+        cp_async_commit();
+        cp_async_wait<0>();
+    };
+    if (fresh && warp == 7) fetch_block(0);
 
     for (int lw = 0; lw < 15; ++lw) {
         __syncthreads();
+        if (fresh && lw <= 7) {
+            // ---- pull phase: warp w adds P = Lfa[row block w, :] E_above[:, block lw] to C and Y of leaf
+            // (w, lw), and R = C_left[block lw, :] Ufl[:, column block w] to Y of leaf (lw, w)
+            if (sm.prog_above) {
+                double p0 = 0.0, p1 = 0.0, p2 = 0.0, p3 = 0.0;
+                const double *A = Lfa + (warp * 8 + g) * QLD + t;
+                const double *B = stgE + (lw & 1) * STG_E + t * STG_E_LD + g;
+#pragma unroll 4
+                for (int kk = 0; kk < Q; kk += 8) {
+                    dmma_m8n8k4(p0, p1, A[kk], B[kk * STG_E_LD]);
+                    dmma_m8n8k4(p2, p3, A[kk + 4], B[(kk + 4) * STG_E_LD]);
+                }
+                p0 += p2; p1 += p3;
+                double2 *yq = reinterpret_cast<double2 *>(Ys + (warp * 8 + g) * QLD + lw * 8 + t * 2);
+                double2 *cq = reinterpret_cast<double2 *>(Cs + (warp * 8 + g) * QLD + lw * 8 + t * 2);
+                double2 yv = *yq, cv = *cq;
+                yv.x += p0; yv.y += p1; cv.x += p0; cv.y += p1;
+                *yq = yv; *cq = cv;
+            }
+            __syncwarp();
+            if (sm.prog_left) {
+                double r0 = 0.0, r1 = 0.0, r2 = 0.0, r3 = 0.0;
+                const double *A = stgC + (lw & 1) * STG_C + g * QLD + t;
+                const double *B = Ufl + t * QLD + warp * 8 + g;
+#pragma unroll 4
+                for (int kk = 0; kk < Q; kk += 8) {
+                    dmma_m8n8k4(r0, r1, A[kk], B[kk * QLD]);
+                    dmma_m8n8k4(r2, r3, A[kk + 4], B[(kk + 4) * QLD]);
+                }
+                r0 += r2; r1 += r3;
+                double2 *yq = reinterpret_cast<double2 *>(Ys + (lw * 8 + g) * QLD + warp * 8 + t * 2);
+                double2 yv = *yq;
+                yv.x += r0; yv.y += r1;
+                *yq = yv;
+            }
+            __syncthreads();
+        }
+        if (warp == 7) {
+            // ---- publish what the previous leaf-waves stored (the barriers above order those stores before
+            // this thread's fence), then fetch the next block of the neighbours
+            if (lane == 0 && lw > 0) {
+                __threadfence();
+                st_release_u32(sm.prog_self, (unsigned)lw);
+                if (lw == GO_WAVE) {
+                    const int qi = sm.q >> 1, qj = sm.q & 1;
+                    if (qi == 0) quadrant_arrive(p, sm.I, sm.J, sm.q + 2);
+                    else if (sm.I + 1 < p.ntm) quadrant_arrive(p, sm.I + 1, sm.J, sm.q - 2);
+                    if (qj == 0) quadrant_arrive(p, sm.I, sm.J, sm.q + 1);
+                    else if (sm.J + 1 < p.ntn) quadrant_arrive(p, sm.I, sm.J + 1, sm.q - 1);
+                }
+            }
+            __syncwarp();
+            if (fresh && lw < 7) fetch_block(lw + 1);
+        }
         const int a_lo = max(0, lw - 7), a_hi = min(7, lw);
         const int a = a_lo + warp, b = lw - a;
         if (a <= a_hi) {
@@ -298,15 +413,33 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
                 y1 = fma(l1, ed, y1); c1 = fma(l1, ed, c1); y1 = fma(cr1, u1, y1);
             }
             yp[0] = y0; yp[4 * QLD] = y1; cp[0] = c0; cp[4 * QLD] = c1;
-            Zs[(a * 8 + i0) * Q + b * 8 + j] = z0;
-            Zs[(a * 8 + i0 + 4) * Q + b * 8 + j] = z1;
-            if (col0 + b * 8 + j < p.n) {
-                if (row0 + a * 8 + i0 < p.m) max_abs_e = fmax(max_abs_e, fabs(y0));
-                if (row0 + a * 8 + i0 + 4 < p.m) max_abs_e = fmax(max_abs_e, fabs(y1));
+            // results of the leaf: E and C to the workspace (for the neighbours and for the far parts of
+            // later tiles), Z (and the caller's E) to the output
+            {
+                const int gr = row0 + a * 8 + i0, gc = col0 + b * 8 + j;
+                const long at = (long)gr * p.np + gc;
+                p.Ebuf[at] = y0; p.Ebuf[at + 4 * p.np] = y1;
+                p.Cbuf[at] = c0; p.Cbuf[at + 4 * p.np] = c1;
+                if (gc < p.n) {
+                    if (gr < p.m) {
+                        p.Z[(long)gr * p.ldz + gc] = z0;
+                        if (p.Euser) p.Euser[(long)gr * p.lde + gc] = y0;
+                        max_abs_e = fmax(max_abs_e, fabs(y0));
+                    }
+                    if (gr + 4 < p.m) {
+                        p.Z[(long)(gr + 4) * p.ldz + gc] = z1;
+                        if (p.Euser) p.Euser[(long)(gr + 4) * p.lde + gc] = y1;
+                        max_abs_e = fmax(max_abs_e, fabs(y1));
+                    }
+                }
             }
         }
     }
     __syncthreads();
+    if (tid == 0) {                      // everything is stored: the quadrant is complete
+        __threadfence();
+        st_release_u32(sm.prog_self, 15u);
+    }
     // status: the earliest (in sweep order) unrepresentable value of the quadrant, if any
     if (badkey != ~0ull) atomicMin(&s_badkey, badkey);
     __syncthreads();
@@ -317,58 +450,62 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
     }
 }
 
+// 64 x 64 diagonal blocks of both factors into one shared-memory matrix: below the diagonal
+// L[r0 + i][r0 + k], above it U[c0 + k][c0 + j], zeros on it and outside the matrices.
+__device__ __forceinline__ void load_lu_diag_async(double *dst, const TiledKernelParams &p, int r0, int c0) {
+#pragma unroll
+    for (int it = 0; it < 16; ++it) {
+        const int c = threadIdx.x + it * TILED_THREADS;
+        const int i = c >> 6, j = c & 63;
+        const bool lower = j < i, upper = j > i;
+        const bool take = lower ? (r0 + i < p.m) : (upper && c0 + j < p.n);     // r0 + j < r0 + i, c0 + i < c0 + j
+        const double *src = lower ? p.L + (long)(r0 + i) * p.ldl + r0 + j : p.U + (long)(c0 + i) * p.ldu + c0 + j;
+        cp_async8(dst + i * QLD + j, take ? src : p.L, take ? 8 : 0);
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // One 64 x 64 quadrant q (0: top-left, 1: top-right, 2: bottom-left, 3: bottom-right) of tile
-// (I, J): the unit of work on the critical path.
+// (I, J): the unit of work on the critical path.  In the grid of quadrants it sits at
+// (r, c) = (2 I + q / 2, 2 J + q % 2).
 //
 // On entry the quadrant's part of the tile's Cbuf region holds the FAR part of Cd (all source
-// tiles above except the adjacent one) and its Ebuf part the FAR part of Rt, both already
-// updated by the cross terms of the quadrants of this tile it depends on.  The task
-//   1. pulls the adjacent tiles' contributions itself: Cd += L[rows, tile I-1] E[tile I-1, cols]
-//      and Rt += C[rows, tile J-1] U[tile J-1, cols], four 64^3 DMMA products staged through two
-//      pairs of shared-memory buffers (they need only the two quadrants of each neighbour that
-//      share this quadrant's columns / rows, which is what its dependency counter waits for);
-//   2. forms Y = X + Rt + Cd, C = Cd and runs Algorithm 3 on the quadrant;
-//   3. writes E, C = L E, Z (and the caller's E), and adds the cross terms it owes to later
-//      quadrants of the tile: q0 -> q1 (through U) and q2 (through L); q1 -> q3 (through L);
-//      q2 -> q3 (through U).
-// Quadrants 1 and 2 of a tile are independent of each other.
+// tiles above except the adjacent one) and its Ebuf part the FAR part of Rt.  The task
+//   1. pulls what the adjacent tiles and its own tile contribute from quadrants that are COMPLETE
+//      (rows r' <= r - 2, columns c' <= c - 2 of the quadrant grid): up to four 64^3 DMMA products;
+//   2. forms Y = X + Rt + Cd, C = Cd and runs Algorithm 3 on the quadrant, taking the contributions
+//      of the quadrant right above it and of the one right to its left block by block as they
+//      finish (quadrant_sweep), and publishing its own leaves wave by wave.
 __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem, const TiledKernelParams &p,
                                                double &max_abs_e) {
-    double *Ys = smem, *Cs = smem + QMAT, *Ls = smem + 2 * QMAT, *Us = smem + 3 * QMAT, *Xop = smem + 4 * QMAT;
+    double *Ys = smem, *Cs = smem + QMAT, *LU = smem + 2 * QMAT, *Lfa = smem + 3 * QMAT, *Ufl = smem + 4 * QMAT;
     double *tabL = smem + 5 * QMAT, *tabU = tabL + Q * TAB_LD;
-    int *Zs = reinterpret_cast<int *>(tabU + Q * TAB_LD);
-    double *eT = p.Ebuf + (long)I * T * p.np + (long)J * T;
-    double *cT = p.Cbuf + (long)I * T * p.np + (long)J * T;
+    double *stg = tabU + Q * TAB_LD;
     const int tid = threadIdx.x;
     const int qi = q >> 1, qj = q & 1;
     const int row0 = I * T + qi * Q, col0 = J * T + qj * Q;
-    double *eQ = eT + (long)qi * Q * p.np + qj * Q;
-    double *cQ = cT + (long)qi * Q * p.np + qj * Q;
+    double *eQ = p.Ebuf + (long)row0 * p.np + col0;
+    double *cQ = p.Cbuf + (long)row0 * p.np + col0;
 
-    // ---- 1. near pulls.  Steps 0,1: Cd halves (k over the two quadrant rows of tile I-1);
-    // steps 2,3: Rt halves (k over the two quadrant columns of tile J-1).  Operands of step k go to
-    // buffer pair k & 1 = {(Ls, Us), (Xop, Cs)}; loads run one step ahead of the products.
+    // ---- 1. pulls from complete quadrants.  Rows of the adjacent tile above that are not the 64 rows
+    // right above this quadrant: one block for a top quadrant, two for a bottom one; columns likewise.
     QAcc accC, accR;
     accC.zero();
     accR.zero();
     {
-        const int first = I > 0 ? 0 : 2, last = J > 0 ? 4 : 2;     // steps [first, last)
-        const int ns = last - first;
-        // three buffer pairs, so that up to three steps are in flight; the third pair borrows Ys and
-        // the area of the coefficient tables / Z staging, all unused until the sweep proper
-        auto bufA = [&](int j) { return j == 0 ? Ls : (j == 1 ? Xop : Ys); };
-        auto bufB = [&](int j) { return j == 0 ? Us : (j == 1 ? Cs : tabL); };
+        const int nsa = I > 0 ? 1 + qi : 0, nsl = J > 0 ? 1 + qj : 0, ns = nsa + nsl;
+        // three buffer pairs, so that up to three steps are in flight; all unused until the sweep proper
+        auto bufA = [&](int j) { return j == 0 ? Lfa : (j == 1 ? LU : Ys); };
+        auto bufB = [&](int j) { return j == 0 ? Ufl : (j == 1 ? Cs : tabL); };
         auto issue = [&](int i) {
-            const int k = first + i, kh = k & 1;
             double *Ab = bufA(i % 3), *Bb = bufB(i % 3);
-            if (k < 2) {
-                const int k0 = (I - 1) * T + kh * Q;
+            if (i < nsa) {
+                const int k0 = (I - 1) * T + i * Q;
                 if (p.l_al16) load_full_block_async16(Ab, p.L, p.ldl, p.m, row0, k0);
                 else load_factor_block_async(Ab, p.L, p.ldl, p.m, row0, k0, 0);
                 load_quadrant_async(Bb, p.Ebuf + (long)k0 * p.np + col0, p.np);
             } else {
-                const int k0 = (J - 1) * T + kh * Q;
+                const int k0 = (J - 1) * T + (i - nsa) * Q;
                 load_quadrant_async(Ab, p.Cbuf + (long)row0 * p.np + k0, p.np);
                 if (p.u_al16) load_full_block_async16(Bb, p.U, p.ldu, p.n, k0, col0);
                 else load_factor_block_async(Bb, p.U, p.ldu, p.n, k0, col0, 0);
@@ -381,7 +518,7 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
             const int pending = min(ns, i + 3) - (i + 1);        // groups issued after step i's
             if (pending >= 2) cp_async_wait<2>(); else if (pending == 1) cp_async_wait<1>(); else cp_async_wait<0>();
             __syncthreads();
-            if (first + i < 2) quad_mma(accC, bufA(i % 3), bufB(i % 3)); else quad_mma(accR, bufA(i % 3), bufB(i % 3));
+            if (i < nsa) quad_mma(accC, bufA(i % 3), bufB(i % 3)); else quad_mma(accR, bufA(i % 3), bufB(i % 3));
             if (i + 3 < ns) {
                 __syncthreads();
                 issue(i + 3);
@@ -391,23 +528,26 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
     }
 
     // ---- 2. operands of the sweep
-    // (the sweep reads the diagonal blocks below / above the diagonal only, so the 16-byte loader, which
-    // does not mask the other triangle, serves as well)
-    if (p.l_al16) load_full_block_async16(Ls, p.L, p.ldl, p.m, row0, row0);
-    else load_factor_block_async(Ls, p.L, p.ldl, p.m, row0, row0, 1);
-    if (p.u_al16) load_full_block_async16(Us, p.U, p.ldu, p.n, col0, col0);
-    else load_factor_block_async(Us, p.U, p.ldu, p.n, col0, col0, 2);
+    Stream sm;
+    sm.I = I; sm.J = J; sm.q = q;
+    const long tq = ((long)I * p.ntn + J) * 4;
+    sm.prog_self = p.qprog + tq + q;
+    sm.prog_above = nullptr; sm.prog_left = nullptr; sm.e_above = nullptr; sm.c_left = nullptr;
+    if (row0 > 0) {
+        sm.prog_above = qi ? p.qprog + tq + (q - 2) : p.qprog + ((long)(I - 1) * p.ntn + J) * 4 + (q + 2);
+        sm.e_above = p.Ebuf + (long)(row0 - Q) * p.np + col0;
+        if (p.l_al16) load_full_block_async16(Lfa, p.L, p.ldl, p.m, row0, row0 - Q);
+        else load_factor_block_async(Lfa, p.L, p.ldl, p.m, row0, row0 - Q, 0);
+    }
+    if (col0 > 0) {
+        sm.prog_left = qj ? p.qprog + tq + (q - 1) : p.qprog + ((long)I * p.ntn + (J - 1)) * 4 + (q + 1);
+        sm.c_left = p.Cbuf + (long)row0 * p.np + (col0 - Q);
+        if (p.u_al16) load_full_block_async16(Ufl, p.U, p.ldu, p.n, col0 - Q, col0);
+        else load_factor_block_async(Ufl, p.U, p.ldu, p.n, col0 - Q, col0, 0);
+    }
+    load_lu_diag_async(LU, p, row0, col0);
     load_quadrant_async(Cs, cQ, p.np);
     load_quadrant_async(Ys, eQ, p.np);
-    // the operand of the first cross term that follows this quadrant
-    if (q == 0 || q == 2) {
-        if (p.u_al16) load_full_block_async16(Xop, p.U, p.ldu, p.n, J * T, J * T + Q);
-        else load_factor_block_async(Xop, p.U, p.ldu, p.n, J * T, J * T + Q, 0);
-    }
-    if (q == 1) {
-        if (p.l_al16) load_full_block_async16(Xop, p.L, p.ldl, p.m, I * T + Q, I * T);
-        else load_factor_block_async(Xop, p.L, p.ldl, p.m, I * T + Q, I * T, 0);
-    }
     cp_async_commit();
     double xv[16];
 #pragma unroll
@@ -418,7 +558,7 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
     }
     cp_async_wait<0>();
     __syncthreads();
-    quad_add_to(Cs, QLD, accC, false);                    // Cd = far part + cross terms + near pull
+    quad_add_to(Cs, QLD, accC, false);                    // Cd = far part + pulls from complete quadrants
     quad_add_to(Ys, QLD, accR, false);                    // Rt likewise
     __syncthreads();
 #pragma unroll
@@ -427,33 +567,7 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
         int r = c >> 6, cc = c & 63;
         Ys[r * QLD + cc] += xv[it] + Cs[r * QLD + cc];
     }
-    quadrant_sweep(Ys, Cs, Ls, Us, Zs, tabL, tabU, row0, col0, p, max_abs_e);
-    // ---- 3. results of the quadrant
-    store_quadrant(eQ, p.np, Ys);
-    store_quadrant(cQ, p.np, Cs);
-#pragma unroll
-    for (int it = 0; it < 16; ++it) {
-        int c = tid + it * TILED_THREADS;
-        int r = c >> 6, cc = c & 63;
-        int gr = row0 + r, gc = col0 + cc;
-        if (gr < p.m && gc < p.n) {
-            p.Z[(long)gr * p.ldz + gc] = Zs[r * Q + cc];
-            if (p.Euser) p.Euser[(long)gr * p.lde + gc] = Ys[r * QLD + cc];
-        }
-    }
-    // cross terms to the quadrants of this tile that follow
-    if (q == 0 || q == 2)     // C of the left quadrant pushes right through U[left cols, right cols]
-        cross_gemm(eT + (long)qi * Q * p.np + Q, p.np, Cs, Xop);
-    if (q == 0) {
-        __syncthreads();
-        if (p.l_al16) load_full_block_async16(Xop, p.L, p.ldl, p.m, I * T + Q, I * T);
-        else load_factor_block_async(Xop, p.L, p.ldl, p.m, I * T + Q, I * T, 0);
-        cp_async_commit();
-        cp_async_wait<0>();
-        __syncthreads();
-    }
-    if (q == 0 || q == 1)     // E of the upper quadrant folds down through L[lower rows, upper rows]
-        cross_gemm(cT + (long)Q * p.np + qj * Q, p.np, Xop, Ys);
+    quadrant_sweep(Ys, Cs, LU, Lfa, Ufl, stg, tabL, tabU, row0, col0, sm, p, max_abs_e);
     __syncthreads();
 }
 
@@ -539,14 +653,13 @@ __device__ __forceinline__ unsigned ready_pop(const TiledKernelParams &p) {
     }
 }
 
-// Arrivals a quadrant task waits for: the two far parts of its tile, the two quadrants of the tile
-// above that share its columns, the two quadrants of the tile to the left that share its rows, and
-// its predecessors inside the tile (q1, q2 <- q0; q3 <- q1, q2).
+// Arrivals a quadrant task at (r, c) of the quadrant grid waits for: the two far parts of its tile,
+// the quadrants at (r - 2, c) and (r, c - 2) being complete (everything further up / left is then
+// complete as well), and the quadrants at (r - 1, c) and (r, c - 1) having reached GO_WAVE.
 __device__ __forceinline__ unsigned quadrant_needed(int I, int J, int q) {
-    return 2u + (I > 0 ? 2u : 0u) + (J > 0 ? 2u : 0u) + (q == 0 ? 0u : (q == 3 ? 2u : 1u));
+    const int r = 2 * I + (q >> 1), c = 2 * J + (q & 1);
+    return 2u + (r >= 2 ? 1u : 0u) + (c >= 2 ? 1u : 0u) + (r >= 1 ? 1u : 0u) + (c >= 1 ? 1u : 0u);
 }
-// the caller has fenced the CTA's results (after a barrier).  The arrival that completes the count
-// publishes the task on the ready ring.
 // A quadrant that lies wholly outside the matrix (ragged last tile row / column) is never a task:
 // arrivals at it are dropped here, its region of the workspace keeps the zeros the far parts parked
 // there, and nothing inside the matrix depends on it.
@@ -735,17 +848,12 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                 // atomic round trip); sweep_quadrant ended with a barrier, so each arriving thread's fence
                 // covers the whole CTA's results
                 if (tid < 8) {
-                    const int qi = q >> 1, qj = q & 1;
-                    int aI = -1, aJ = 0, aq = 0;
-                    if (tid == 0 && q == 0) { aI = I; aJ = J; aq = 1; }
-                    if (tid == 1 && q == 0) { aI = I; aJ = J; aq = 2; }
-                    if (tid == 0 && (q == 1 || q == 2)) { aI = I; aJ = J; aq = 3; }
-                    if (tid == 2 && I + 1 < pq.ntm) { aI = I + 1; aJ = J; aq = qj; }
-                    if (tid == 3 && I + 1 < pq.ntm) { aI = I + 1; aJ = J; aq = 2 + qj; }
-                    if (tid == 4 && J + 1 < pq.ntn) { aI = I; aJ = J + 1; aq = 2 * qi; }
-                    if (tid == 5 && J + 1 < pq.ntn) { aI = I; aJ = J + 1; aq = 2 * qi + 1; }
+                    // completion: the quadrants two below / two to the right may pull from this one
+                    int aI = -1, aJ = 0;
+                    if (tid == 2 && I + 1 < pq.ntm) { aI = I + 1; aJ = J; }
+                    if (tid == 4 && J + 1 < pq.ntn) { aI = I; aJ = J + 1; }
                     __threadfence();
-                    if (aI >= 0) quadrant_arrive(pq, aI, aJ, aq);
+                    if (aI >= 0) quadrant_arrive(pq, aI, aJ, q);
                     if (tid == 6) {
                         unsigned done = atomicAdd(pq.quad_done + (long)I * pq.ntn + J, 1u);
                         const unsigned nquad = (pq.m - I * T > Q ? 2u : 1u) * (pq.n - J * T > Q ? 2u : 1u);
@@ -841,7 +949,7 @@ static size_t pad256(size_t x) { return (x + 255) / 256 * 256; }
 
 struct TiledLayout {
     int ntm, ntn;
-    size_t q_off, flags_off, quad_off, qdep_off, e_off, c_off, total;
+    size_t q_off, flags_off, quad_off, qdep_off, qprog_off, e_off, c_off, total;
 };
 static TiledLayout tiled_layout(int m, int n) {
     TiledLayout l;
@@ -853,7 +961,8 @@ static TiledLayout tiled_layout(int m, int n) {
     l.flags_off = l.q_off + 4096 * sizeof(unsigned);
     l.quad_off = l.flags_off + pad256(tiles * sizeof(unsigned));
     l.qdep_off = l.quad_off + pad256(tiles * sizeof(unsigned));
-    l.e_off = l.qdep_off + pad256(4 * tiles * sizeof(unsigned));
+    l.qprog_off = l.qdep_off + pad256(4 * tiles * sizeof(unsigned));
+    l.e_off = l.qprog_off + pad256(4 * tiles * sizeof(unsigned));
     l.c_off = l.e_off + pad256(mat);
     l.total = l.c_off + pad256(mat);
     return l;
@@ -884,6 +993,7 @@ int launch_round_tiled(const TiledParams &in, void *ws, size_t ws_bytes, cudaStr
     p.flagS = reinterpret_cast<unsigned *>(w + l.flags_off);
     p.quad_done = reinterpret_cast<unsigned *>(w + l.quad_off);
     p.qdep = reinterpret_cast<unsigned *>(w + l.qdep_off);
+    p.qprog = reinterpret_cast<unsigned *>(w + l.qprog_off);
     p.Ebuf = reinterpret_cast<double *>(w + l.e_off);
     p.Cbuf = reinterpret_cast<double *>(w + l.c_off);
     p.info = in.info;
@@ -932,7 +1042,7 @@ static BatchedLayout batched_layout(int count, const TiledParams *pr) {
     for (int b = 0; b < count; ++b) {
         TiledLayout t = tiled_layout(pr[b].m, pr[b].n);
         size_t tiles = (size_t)t.ntm * t.ntn;
-        off += 2 * pad256(tiles * sizeof(unsigned)) + pad256(4 * tiles * sizeof(unsigned));
+        off += 2 * pad256(tiles * sizeof(unsigned)) + 2 * pad256(4 * tiles * sizeof(unsigned));
         bufs += 2 * pad256((size_t)t.ntm * T * (size_t)t.ntn * T * sizeof(double));
         l.ntiles += (long)tiles;
     }
@@ -986,6 +1096,7 @@ int launch_round_tiled_batched(int count, const TiledParams *pr, double *min_mar
         d.flagS = reinterpret_cast<unsigned *>(w + foff); foff += pad256(tiles * sizeof(unsigned));
         d.quad_done = reinterpret_cast<unsigned *>(w + foff); foff += pad256(tiles * sizeof(unsigned));
         d.qdep = reinterpret_cast<unsigned *>(w + foff); foff += pad256(4 * tiles * sizeof(unsigned));
+        d.qprog = reinterpret_cast<unsigned *>(w + foff); foff += pad256(4 * tiles * sizeof(unsigned));
         d.Ebuf = reinterpret_cast<double *>(w + boff); boff += mat;
         d.Cbuf = reinterpret_cast<double *>(w + boff); boff += mat;
         d.max_abs_e = reinterpret_cast<double *>(w + l.maxe_off) + b;
