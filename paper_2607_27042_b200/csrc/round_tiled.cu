@@ -10,22 +10,23 @@
 // so they run on the fp64 tensor path (dmma_gemm.cuh); tiles with equal I + J are independent.
 //
 // Scheduling.  Two kinds of work, one persistent cooperatively launched grid (one CTA per SM):
-//  * FAR parts.  Each tile's Cd and Rt contractions over every source tile EXCEPT the adjacent
-//    one.  Listed wave by wave (I + J ascending) and claimed in that order from one atomic
-//    counter.  A far part waits (bounded) only on tiles two or more waves back, parks its
+//  * FAR parts.  Each tile's Cd and Rt contractions over every source tile EXCEPT the two nearest
+//    ones.  Listed wave by wave (I + J ascending) and claimed in that order from one atomic
+//    counter.  A far part waits (bounded) only on tiles three or more waves back, parks its
 //    partial sum in the tile's own workspace region and then announces it to the tile's four
-//    quadrant tasks.  This is >90 % of the flops and runs on the fp64 tensor path.
+//    quadrant tasks; it is done long before they need it.  This is >90 % of the flops and runs on
+//    the fp64 tensor path.
 //  * QUADRANT tasks (64 x 64), the critical path.  In the grid of quadrants, (r, c) needs all
-//    quadrants above it in its column and to its left in its row.  What complete quadrants of the
-//    adjacent tiles (and of its own tile) contribute it pulls itself when it starts (up to four
-//    64^3 DMMA products).  The quadrant right above and the one right to the left are NOT waited
-//    for: every quadrant publishes its 8 x 8 leaves leaf-wave by leaf-wave (results to the
-//    workspace, a progress word per quadrant), and its two neighbours take them in as they come,
-//    running nine leaf-waves behind (block b of a neighbour is final after its leaf-wave 7 + b).
-//    A task counts arrivals from the two far parts of its tile, from (r-2, c) and (r, c-2) being
-//    complete, and from (r-1, c) and (r, c-1) having reached their third leaf-wave; the last arrival
-//    puts it on a global ready ring.  A running quadrant task waits -- bounded -- only on its two
-//    neighbours, which are running by then (or done).
+//    quadrants above it in its column and to its left in its row.  What the quadrants of the two
+//    nearest tiles contribute (rows 2 I - 4 .. r - 2 of the grid, columns likewise) it pulls itself
+//    when it starts: up to eight 64^3 DMMA products.  The quadrant right above and the one right to
+//    the left are NOT waited for: every quadrant publishes its 8 x 8 leaves leaf-wave by leaf-wave
+//    (results to the workspace, a progress word per quadrant), and its two neighbours take them in
+//    as they come, running nine leaf-waves behind (block b of a neighbour is final after its
+//    leaf-wave 7 + b).  A task counts arrivals from the two far parts of its tile and from
+//    (r-1, c) and (r, c-1) beginning to sweep; the last arrival puts it on a global ready ring.  A
+//    running quadrant task waits -- bounded -- only on quadrants above it / to its left, which are
+//    running by then (or done).
 // Every CTA serves the ready ring first: at the top of its loop, while a far part waits, and
 // every few chunks of a far part (it then parks its partial sum and un-parks it afterwards).
 // A far part only ever waits on tiles of earlier waves, whose far parts were claimed earlier and
@@ -213,7 +214,6 @@ __device__ __forceinline__ void leaf_pull(double *Ys, double *Cs, const double *
 constexpr int STG_E_LD = 12;                 // staged 64 x 8 column block of E, [k][n], 12 = 8 + 4 pad
 constexpr int STG_E = Q * STG_E_LD;          // doubles per staged E block
 constexpr int STG_C = 8 * QLD;               // staged 8 x 64 row block of C, [m][k]
-constexpr int GO_WAVE = 2;                   // a quadrant lets its two neighbours start at this leaf-wave
 
 struct Stream {
     const unsigned *prog_above, *prog_left;  // progress words of the two neighbours (NULL: none)
@@ -302,6 +302,15 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
         cp_async_commit();
         cp_async_wait<0>();
     };
+    if (tid == 7 * 32) {
+        // this quadrant is about to sweep: the one below it and the one to its right may start getting ready
+        const int qi = sm.q >> 1, qj = sm.q & 1;
+        if (qi == 0) quadrant_arrive(p, sm.I, sm.J, sm.q + 2);
+        else if (sm.I + 1 < p.ntm) quadrant_arrive(p, sm.I + 1, sm.J, sm.q - 2);
+        if (qj == 0) quadrant_arrive(p, sm.I, sm.J, sm.q + 1);
+        else if (sm.J + 1 < p.ntn) quadrant_arrive(p, sm.I, sm.J + 1, sm.q - 1);
+    }
+    __syncwarp();
     if (fresh && warp == 7) fetch_block(0);
 
     for (int lw = 0; lw < 15; ++lw) {
@@ -349,13 +358,6 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
             if (lane == 0 && lw > 0) {
                 __threadfence();
                 st_release_u32(sm.prog_self, (unsigned)lw);
-                if (lw == GO_WAVE) {
-                    const int qi = sm.q >> 1, qj = sm.q & 1;
-                    if (qi == 0) quadrant_arrive(p, sm.I, sm.J, sm.q + 2);
-                    else if (sm.I + 1 < p.ntm) quadrant_arrive(p, sm.I + 1, sm.J, sm.q - 2);
-                    if (qj == 0) quadrant_arrive(p, sm.I, sm.J, sm.q + 1);
-                    else if (sm.J + 1 < p.ntn) quadrant_arrive(p, sm.I, sm.J + 1, sm.q - 1);
-                }
             }
             __syncwarp();
             if (fresh && lw < 7) fetch_block(lw + 1);
@@ -470,9 +472,10 @@ __device__ __forceinline__ void load_lu_diag_async(double *dst, const TiledKerne
 // (r, c) = (2 I + q / 2, 2 J + q % 2).
 //
 // On entry the quadrant's part of the tile's Cbuf region holds the FAR part of Cd (all source
-// tiles above except the adjacent one) and its Ebuf part the FAR part of Rt.  The task
-//   1. pulls what the adjacent tiles and its own tile contribute from quadrants that are COMPLETE
-//      (rows r' <= r - 2, columns c' <= c - 2 of the quadrant grid): up to four 64^3 DMMA products;
+// tiles above except the two nearest) and its Ebuf part the FAR part of Rt.  The task
+//   1. pulls what the two nearest tiles and its own tile contribute from quadrants that are COMPLETE
+//      (rows 2 I - 4 .. r - 2, columns 2 J - 4 .. c - 2 of the quadrant grid): up to eight 64^3 DMMA
+//      products;
 //   2. forms Y = X + Rt + Cd, C = Cd and runs Algorithm 3 on the quadrant, taking the contributions
 //      of the quadrant right above it and of the one right to its left block by block as they
 //      finish (quadrant_sweep), and publishing its own leaves wave by wave.
@@ -487,38 +490,61 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
     double *eQ = p.Ebuf + (long)row0 * p.np + col0;
     double *cQ = p.Cbuf + (long)row0 * p.np + col0;
 
-    // ---- 1. pulls from complete quadrants.  Rows of the adjacent tile above that are not the 64 rows
-    // right above this quadrant: one block for a top quadrant, two for a bottom one; columns likewise.
+    // ---- 1. pulls from complete quadrants: rows r' = max(0, 2 I - 4) .. r - 2 of the quadrant grid (the
+    // two tiles above, without the quadrant right above this one), columns likewise.  The far parts of the
+    // tile cover everything further away.  Oldest sources first; the two newest, (r - 2, c) and
+    // (r, c - 2), may still be sweeping their last leaves when this task starts and are waited for
+    // right before their blocks are requested (they are running: the neighbour between them and this
+    // quadrant could not have started otherwise).
     QAcc accC, accR;
     accC.zero();
     accR.zero();
     {
-        const int nsa = I > 0 ? 1 + qi : 0, nsl = J > 0 ? 1 + qj : 0, ns = nsa + nsl;
+        const int r = 2 * I + qi, c = 2 * J + qj;
+        const int fa = max(0, 2 * I - 4), fl = max(0, 2 * J - 4);
+        const int nsa = max(0, r - 1 - fa), nsl = max(0, c - 1 - fl), ns = nsa + nsl;
+        auto prog_of = [&](int rr, int cc) {
+            return p.qprog + ((long)(rr >> 1) * p.ntn + (cc >> 1)) * 4 + (rr & 1) * 2 + (cc & 1);
+        };
+        // step i -> (direction, block): the older blocks of both directions first, then the newest of each
+        const int olda = max(0, nsa - 1), oldl = max(0, nsl - 1);
+        auto step_dir = [&](int i) {
+            return i < olda ? 0 : (i < olda + oldl ? 1 : ((i == olda + oldl && nsa > 0) ? 0 : 1));
+        };
+        auto step_blk = [&](int i) {
+            return i < olda ? fa + i : (i < olda + oldl ? fl + (i - olda) : (step_dir(i) == 0 ? r - 2 : c - 2));
+        };
         // three buffer pairs, so that up to three steps are in flight; all unused until the sweep proper
         auto bufA = [&](int j) { return j == 0 ? Lfa : (j == 1 ? LU : Ys); };
         auto bufB = [&](int j) { return j == 0 ? Ufl : (j == 1 ? Cs : tabL); };
         auto issue = [&](int i) {
             double *Ab = bufA(i % 3), *Bb = bufB(i % 3);
-            if (i < nsa) {
-                const int k0 = (I - 1) * T + i * Q;
+            const int dir = step_dir(i), blk = step_blk(i), k0 = blk * Q;
+            if (i >= olda + oldl) await_progress(p, dir == 0 ? prog_of(blk, c) : prog_of(r, blk), nullptr, 15u);
+            if (dir == 0) {
                 if (p.l_al16) load_full_block_async16(Ab, p.L, p.ldl, p.m, row0, k0);
                 else load_factor_block_async(Ab, p.L, p.ldl, p.m, row0, k0, 0);
                 load_quadrant_async(Bb, p.Ebuf + (long)k0 * p.np + col0, p.np);
             } else {
-                const int k0 = (J - 1) * T + (i - nsa) * Q;
                 load_quadrant_async(Ab, p.Cbuf + (long)row0 * p.np + k0, p.np);
                 if (p.u_al16) load_full_block_async16(Bb, p.U, p.ldu, p.n, k0, col0);
                 else load_factor_block_async(Bb, p.U, p.ldu, p.n, k0, col0, 0);
             }
             cp_async_commit();
         };
+        // the older sources: one warp each makes sure its quadrant is complete (it almost always is)
+        {
+            const int w = threadIdx.x >> 5;
+            if (w < olda) await_progress(p, prog_of(fa + w, c), nullptr, 15u);
+            else if (w < olda + oldl) await_progress(p, prog_of(r, fl + (w - olda)), nullptr, 15u);
+        }
         __syncthreads();
         for (int i = 0; i < ns && i < 3; ++i) issue(i);
         for (int i = 0; i < ns; ++i) {
             const int pending = min(ns, i + 3) - (i + 1);        // groups issued after step i's
             if (pending >= 2) cp_async_wait<2>(); else if (pending == 1) cp_async_wait<1>(); else cp_async_wait<0>();
             __syncthreads();
-            if (i < nsa) quad_mma(accC, bufA(i % 3), bufB(i % 3)); else quad_mma(accR, bufA(i % 3), bufB(i % 3));
+            if (step_dir(i) == 0) quad_mma(accC, bufA(i % 3), bufB(i % 3)); else quad_mma(accR, bufA(i % 3), bufB(i % 3));
             if (i + 3 < ns) {
                 __syncthreads();
                 issue(i + 3);
@@ -573,7 +599,7 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
 
 // ---------------------------------------------------------------------------------------------
 // Far parts in claim order: wave by wave (I + J ascending); inside a wave the longest contractions
-// first (the Cd part of tile (I, J) has I - 1 chunks, the Rt part J - 1), so that a wave's far parts
+// first (the Cd part of tile (I, J) has I - 2 chunks, the Rt part J - 2), so that a wave's far parts
 // finish close together instead of the long ones trailing.
 __device__ __forceinline__ void decode_task(int task, int ntm, int ntn, int &type, int &I, int &J) {
     int tt = task;
@@ -653,12 +679,11 @@ __device__ __forceinline__ unsigned ready_pop(const TiledKernelParams &p) {
     }
 }
 
-// Arrivals a quadrant task at (r, c) of the quadrant grid waits for: the two far parts of its tile,
-// the quadrants at (r - 2, c) and (r, c - 2) being complete (everything further up / left is then
-// complete as well), and the quadrants at (r - 1, c) and (r, c - 1) having reached GO_WAVE.
+// Arrivals a quadrant task at (r, c) of the quadrant grid waits for: the two far parts of its tile and
+// the quadrants at (r - 1, c) and (r, c - 1) having begun to sweep.
 __device__ __forceinline__ unsigned quadrant_needed(int I, int J, int q) {
     const int r = 2 * I + (q >> 1), c = 2 * J + (q & 1);
-    return 2u + (r >= 2 ? 1u : 0u) + (c >= 2 ? 1u : 0u) + (r >= 1 ? 1u : 0u) + (c >= 1 ? 1u : 0u);
+    return 2u + (r >= 1 ? 1u : 0u) + (c >= 1 ? 1u : 0u);
 }
 // A quadrant that lies wholly outside the matrix (ragged last tile row / column) is never a task:
 // arrivals at it are dropped here, its region of the workspace keeps the zeros the far parts parked
@@ -796,7 +821,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                         }
                         const TiledKernelParams &pk = VIEW(slot);
                         s_ctx[n][0] = ty; s_ctx[n][1] = fi; s_ctx[n][2] = fj; s_ctx[n][3] = 0;
-                        s_ctx[n][4] = max(0, (ty == 0 ? fi : fj) - 1); s_ctx[n][5] = task; s_ctx[n][6] = slot;
+                        s_ctx[n][4] = max(0, (ty == 0 ? fi : fj) - 2); s_ctx[n][5] = task; s_ctx[n][6] = slot;
                         s_nctx = n + 1;
                         const unsigned *fl = ty == 0 ? pk.flagS + fj : pk.flagS + (long)fi * pk.ntn;
                         if ((s_ctx[n][4] == 0 || ld_acquire_u32(fl) != 0u) && panels_arrived(((ty == 0 ? fi : fj) >> COPY_BLOCK_TILES_LOG2) + 1))
@@ -848,12 +873,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                 // atomic round trip); sweep_quadrant ended with a barrier, so each arriving thread's fence
                 // covers the whole CTA's results
                 if (tid < 8) {
-                    // completion: the quadrants two below / two to the right may pull from this one
-                    int aI = -1, aJ = 0;
-                    if (tid == 2 && I + 1 < pq.ntm) { aI = I + 1; aJ = J; }
-                    if (tid == 4 && J + 1 < pq.ntn) { aI = I; aJ = J + 1; }
                     __threadfence();
-                    if (aI >= 0) quadrant_arrive(pq, aI, aJ, q);
                     if (tid == 6) {
                         unsigned done = atomicAdd(pq.quad_done + (long)I * pq.ntn + J, 1u);
                         const unsigned nquad = (pq.m - I * T > Q ? 2u : 1u) * (pq.n - J * T > Q ? 2u : 1u);
@@ -876,7 +896,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             continue;
         }
 
-        // ================= B: far part s_pick (every source tile of the contraction except the adjacent one)
+        // ================= B: far part s_pick (every source tile of the contraction except the two nearest)
         const int k = s_pick;
         const TiledKernelParams &pk = VIEW(s_ctx[k][6]);
         if (k != cur) {
