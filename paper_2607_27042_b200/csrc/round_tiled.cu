@@ -791,7 +791,21 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
         if (tid == 0) {
             int state = 2, pick = -1;
             unsigned e = 0u;
+            // A far part of this CTA that is at most two chunks from done and can go on comes before
+            // everything else: the four quadrant tasks of its tile cannot start without it, and other
+            // CTAs can serve the ring.
+            for (int k = 0; k < s_nctx && pick < 0; ++k) {
+                const TiledKernelParams &pk = VIEW(s_ctx[k][6]);
+                const int ty = s_ctx[k][0], pos = s_ctx[k][3], left = s_ctx[k][4] - pos;
+                if (left < 1 || left > 2) continue;
+                const unsigned *fl = ty == 0 ? pk.flagS + (long)pos * pk.ntn + s_ctx[k][2]
+                                             : pk.flagS + (long)s_ctx[k][1] * pk.ntn + pos;
+                if (ld_acquire_u32(fl) != 0u &&
+                    panels_arrived(((ty == 0 ? s_ctx[k][1] : s_ctx[k][2]) >> COPY_BLOCK_TILES_LOG2) + 1))
+                    pick = k;
+            }
             if (ld_relaxed_u32(p.abort) != 0u) state = 4;
+            else if (pick >= 0) state = 0;
             else if ((e = await_panels(ready_pop(p))) != 0u) {
                 state = 1;
                 load_view(FAR_CTX, entry_matrix(e));
@@ -886,7 +900,8 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                 }
                 __syncthreads();
                 if (tid == 0) {
-                    const unsigned en = await_panels(ready_pop(p));
+                    // with far parts in hand, go back to the top of the loop after every task (see there)
+                    const unsigned en = s_nctx > 0 ? 0u : await_panels(ready_pop(p));
                     if (en != 0u) load_view(FAR_CTX, entry_matrix(en));
                     s_pop = en;
                 }
