@@ -352,15 +352,13 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
             }
             __syncthreads();
         }
-        if (warp == 7) {
-            // ---- publish what the previous leaf-waves stored (the barriers above order those stores before
-            // this thread's fence), then fetch the next block of the neighbours
-            if (lane == 0 && lw > 0) {
-                __threadfence();
-                st_release_u32(sm.prog_self, (unsigned)lw);
-            }
-            __syncwarp();
-            if (fresh && lw < 7) fetch_block(lw + 1);
+        // ---- warp 7 fetches the next block of the neighbours; warp 6 (a leaf of its own only in leaf-waves
+        // 6 to 8) publishes what the previous leaf-waves stored: the barriers above order those stores
+        // before this thread's fence
+        if (warp == 7 && fresh && lw < 7) fetch_block(lw + 1);
+        if (tid == 6 * 32 && lw > 0) {
+            __threadfence();
+            st_release_u32(sm.prog_self, (unsigned)lw);
         }
         const int a_lo = max(0, lw - 7), a_hi = min(7, lw);
         const int a = a_lo + warp, b = lw - a;
