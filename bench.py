@@ -222,8 +222,8 @@ def run_cuda(args):
         e2e = {"value": job_value(m, n, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": host_entry_h2d_bytes(m, n, args.fp32), "d2h_bytes_per_step": 4 * m * n + 16,
                "note": "fp64: inputs arrive in steps on a second stream while the sweep already runs; of L and U "
-                       "only the triangles (up to the edge of the 512 x 512 diagonal block) are sent; Z is written "
-                       "straight into the pinned host buffer by the kernel (d2h bytes cross the bus all the same)"}
+                       "only the triangles (up to the edge of the 512 x 512 diagonal block) are sent; Z is copied back "
+                       "row of tiles by row of tiles while the sweep runs (stream-ordered waits on the kernel's counters)"}
 
     if rank != 0:
         if dist:

@@ -110,9 +110,11 @@ int gptq2d_round(int m, int n,
  *   rectangle above and to its left only): step s = the blocks of X on block anti-diagonal s, block
  *   row s of L up to its diagonal block, block column s of U down to its diagonal block (the opposite
  *   triangles are never sent).  Each step is announced to the running kernel by a stream-ordered
- *   32-bit write; a task starts when its step has arrived.  If hZ is pinned, device-mapped memory the
- *   kernel writes Z straight into it, quadrant by quadrant, and no copy back follows.  Pinned buffers
- *   make all copies asynchronous and fast; pageable ones work.  If the driver lacks stream memory
+ *   32-bit write; a task starts when its step has arrived.  If hZ is pinned memory, Z goes back while
+ *   the sweep still runs: the kernel counts the swept tiles of every row of 128 x 128 tiles, and the
+ *   second stream copies the rows of a tile row as soon as a stream-ordered wait sees its count
+ *   complete.  Pinned buffers make all copies asynchronous and fast; pageable ones work (Z is then
+ *   copied at the end).  If the driver lacks stream memory
  *   operations the call falls back to copy-then-sweep.  Concurrent calls on one device take turns to
  *   enqueue (they share the copy stream).
  * Other precisions: X, L, U are copied first, the sweep runs, Z (and E, min_margin) are copied back.

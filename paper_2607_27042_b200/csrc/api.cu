@@ -34,10 +34,12 @@ static size_t pad256(size_t x) { return (x + 255) / 256 * 256; }
 // with a stream-ordered 32-bit write (driver entry point looked up through the runtime, so the
 // library has no link-time dependency on the driver library).
 typedef int (*StreamWriteValue32Fn)(cudaStream_t, unsigned long long, unsigned int, unsigned int);
+typedef int (*StreamWaitValue32Fn)(cudaStream_t, unsigned long long, unsigned int, unsigned int);
 struct HostPipe {
     cudaStream_t copy = nullptr;
     cudaEvent_t inputs_free = nullptr, copies_done = nullptr;
     StreamWriteValue32Fn write32 = nullptr;
+    StreamWaitValue32Fn wait32 = nullptr;    // stream-ordered wait until a device word is >= a value
     bool tried = false;
     std::mutex enqueue;         // one pipelined call at a time enqueues on the shared copy stream and events
 };
@@ -52,14 +54,16 @@ static HostPipe *host_pipe() {
     HostPipe &hp = g_pipe[dev];
     if (!hp.tried) {
         hp.tried = true;
-        void *fn = nullptr;
+        void *fn = nullptr, *fnw = nullptr;
         cudaDriverEntryPointQueryResult qr = cudaDriverEntryPointSymbolNotFound;
         bool ok = cudaGetDriverEntryPoint("cuStreamWriteValue32", &fn, cudaEnableDefault, &qr) == cudaSuccess &&
                   qr == cudaDriverEntryPointSuccess && fn != nullptr;
+        ok = ok && cudaGetDriverEntryPoint("cuStreamWaitValue32", &fnw, cudaEnableDefault, &qr) == cudaSuccess &&
+             qr == cudaDriverEntryPointSuccess && fnw != nullptr;
         ok = ok && cudaStreamCreateWithFlags(&hp.copy, cudaStreamNonBlocking) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&hp.inputs_free, cudaEventDisableTiming) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&hp.copies_done, cudaEventDisableTiming) == cudaSuccess;
-        if (ok) hp.write32 = reinterpret_cast<StreamWriteValue32Fn>(fn);
+        if (ok) { hp.write32 = reinterpret_cast<StreamWriteValue32Fn>(fn); hp.wait32 = reinterpret_cast<StreamWaitValue32Fn>(fnw); }
         (void)cudaGetLastError();
     }
     return hp.write32 ? &hp : nullptr;
@@ -259,6 +263,9 @@ int gptq2d_round_host(int m, int n, const double *hX, const double *hL, const do
         // triangles the sweep reads).  The kernel holds back each task until its step has arrived.
         unsigned *dpanels = reinterpret_cast<unsigned *>(p + 128);
         if (cudaMemsetAsync(dpanels, 0, sizeof(unsigned), stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+        const int ntm_rows = (m + 127) / 128, ntn_cols = (n + 127) / 128;
+        unsigned *rowdone = round_tiled_rowdone(w, m, n);
+        if (cudaMemsetAsync(rowdone, 0, (size_t)ntm_rows * sizeof(unsigned), stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;
         // the copies may overwrite dX, dL, dU only after everything queued on `stream` so far is done
         if (cudaEventRecord(hp->inputs_free, stream) != cudaSuccess ||
             cudaStreamWaitEvent(hp->copy, hp->inputs_free, 0) != cudaSuccess)
@@ -269,21 +276,17 @@ int gptq2d_round_host(int m, int n, const double *hX, const double *hL, const do
         tp.m = m; tp.n = n;
         tp.X = dX; tp.ldx = n; tp.L = dL; tp.ldl = m; tp.U = dU; tp.ldu = n;
         tp.Z = dZ; tp.ldz = n; tp.E = hE ? dE : nullptr; tp.lde = n; tp.info = dinfo;
-        // Z in pinned, device-mapped host memory is written by the kernel directly, quadrant by quadrant,
-        // as the sweep goes: no copy back at the end
+        // Z goes back row of tiles by row of tiles while the sweep still runs, if hZ is pinned: the copy stream
+        // waits (stream-ordered) until the kernel has counted every tile of a row as swept, then copies its rows.
         cudaPointerAttributes za{};
-        if (cudaPointerGetAttributes(&za, hZ) == cudaSuccess && za.type == cudaMemoryTypeHost && za.devicePointer) {
-            tp.Z = static_cast<int32_t *>(za.devicePointer);
-            z_direct = true;
-        }
+        const bool z_pinned = cudaPointerGetAttributes(&za, hZ) == cudaSuccess && za.type == cudaMemoryTypeHost;
         (void)cudaGetLastError();
         tp.panels_ready = dpanels;
         int st = launch_round_tiled(tp, w, inner, stream);
         if (st != GPTQ2D_OK) return st;
-        if (hmin_margin) {
-            margin_kernel<<<1, 1, 0, stream>>>(workspace_max_abs_e(w), dmargin);
-            if (cudaGetLastError() != cudaSuccess) return GPTQ2D_ERR_CUDA;
-        }
+        // From here until the copies are queued the kernel is waiting for this thread: nothing that could
+        // block on the device (a first launch of another kernel loads its module, which waits for running
+        // kernels) may come in between.
         // Step s sends the blocks of X on block anti-diagonal s, block row s of L and block column s of U
         // (COPY_BLOCK x COPY_BLOCK blocks): the order in which the wavefront of the sweep needs them.
         const int CB = COPY_BLOCK, nbm = (m + CB - 1) / CB, nbn = (n + CB - 1) / CB;
@@ -317,8 +320,25 @@ int gptq2d_round_host(int m, int n, const double *hX, const double *hL, const do
             (void)cudaStreamSynchronize(stream);
             return GPTQ2D_ERR_CUDA;
         }
+        // whatever happens in the kernel, no wait of the copy stream may outlast it
+        if (z_pinned && cudaMemsetAsync(rowdone, 0x7f, (size_t)ntm_rows * sizeof(unsigned), stream) != cudaSuccess)
+            return GPTQ2D_ERR_CUDA;
+        if (hmin_margin) {
+            margin_kernel<<<1, 1, 0, stream>>>(workspace_max_abs_e(w), dmargin);
+            if (cudaGetLastError() != cudaSuccess) return GPTQ2D_ERR_CUDA;
+        }
+        if (z_pinned) {
+            for (int I = 0; I < ntm_rows && ok; ++I) {
+                const int rows = m - I * 128 < 128 ? m - I * 128 : 128;
+                ok = hp->wait32(hp->copy, (unsigned long long)reinterpret_cast<uintptr_t>(rowdone + I),
+                                (unsigned)ntn_cols, 0u /* >= */) == 0;
+                ok = ok && cudaMemcpyAsync(hZ + (size_t)I * 128 * n, dZ + (size_t)I * 128 * n, (size_t)rows * n * 4,
+                                           cudaMemcpyDeviceToHost, hp->copy) == cudaSuccess;
+            }
+            z_direct = ok;       // (Z is on its way back: no copy at the end)
+        }
         if (cudaEventRecord(hp->copies_done, hp->copy) != cudaSuccess ||
-            cudaStreamWaitEvent(stream, hp->copies_done, 0) != cudaSuccess)
+            cudaStreamWaitEvent(stream, hp->copies_done, 0) != cudaSuccess || !ok)
             return GPTQ2D_ERR_CUDA;
         pipe_lock.unlock();
     } else

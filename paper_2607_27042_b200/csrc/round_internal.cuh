@@ -54,6 +54,8 @@ struct TiledParams {
 constexpr int COPY_BLOCK_TILES_LOG2 = 2;
 constexpr int COPY_BLOCK = 128 << COPY_BLOCK_TILES_LOG2;
 size_t round_tiled_workspace_bytes(int m, int n);
+// device array inside the workspace: for each row of 128 x 128 tiles, how many of its tiles are swept
+unsigned *round_tiled_rowdone(void *ws, int m, int n);
 int launch_round_tiled(const TiledParams &p, void *ws, size_t ws_bytes, cudaStream_t stream);
 // many matrices in one launch (fp64 tiled sweep); `info` is shared, `min_margin` (optional) gets one value per matrix
 constexpr int BATCH_MAX_COUNT = 8192;     // matrix index has 13 bits in a ready-ring entry

@@ -68,6 +68,7 @@ struct TiledKernelParams {
     unsigned *quad_done;         // [ntm*ntn] swept quadrants of the tile (4 -> tile flag)
     unsigned *qdep;              // [ntm*ntn][4] arrivals each quadrant task has received
     unsigned *qprog;             // [ntm*ntn][4] leaf-waves each quadrant has published (15: complete)
+    unsigned *rowdone;           // [ntm] tiles of each tile row that are swept (the host entry copies Z back row by row)
     double *max_abs_e;
     int *info;
     int l_al16, u_al16;
@@ -892,6 +893,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                         if (done + 1u == nquad) {   // tile swept: far parts that list it as a source may go on
                             __threadfence();
                             st_release_u32(pq.flagS + (long)I * pq.ntn + J, 1u);
+                            atomicAdd(pq.rowdone + I, 1u);
                             atomicAdd(p.tiles_done, 1u);
                         }
                     }
@@ -982,7 +984,7 @@ static size_t pad256(size_t x) { return (x + 255) / 256 * 256; }
 
 struct TiledLayout {
     int ntm, ntn;
-    size_t q_off, flags_off, quad_off, qdep_off, qprog_off, e_off, c_off, total;
+    size_t q_off, flags_off, quad_off, qdep_off, qprog_off, rowdone_off, e_off, c_off, total;
 };
 static TiledLayout tiled_layout(int m, int n) {
     TiledLayout l;
@@ -995,13 +997,17 @@ static TiledLayout tiled_layout(int m, int n) {
     l.quad_off = l.flags_off + pad256(tiles * sizeof(unsigned));
     l.qdep_off = l.quad_off + pad256(tiles * sizeof(unsigned));
     l.qprog_off = l.qdep_off + pad256(4 * tiles * sizeof(unsigned));
-    l.e_off = l.qprog_off + pad256(4 * tiles * sizeof(unsigned));
+    l.rowdone_off = l.qprog_off + pad256(4 * tiles * sizeof(unsigned));
+    l.e_off = l.rowdone_off + pad256((size_t)l.ntm * sizeof(unsigned));
     l.c_off = l.e_off + pad256(mat);
     l.total = l.c_off + pad256(mat);
     return l;
 }
 
 size_t round_tiled_workspace_bytes(int m, int n) { return tiled_layout(m, n).total; }
+unsigned *round_tiled_rowdone(void *ws, int m, int n) {
+    return reinterpret_cast<unsigned *>(static_cast<char *>(ws) + tiled_layout(m, n).rowdone_off);
+}
 
 int launch_round_tiled(const TiledParams &in, void *ws, size_t ws_bytes, cudaStream_t stream) {
     TiledLayout l = tiled_layout(in.m, in.n);
@@ -1027,6 +1033,7 @@ int launch_round_tiled(const TiledParams &in, void *ws, size_t ws_bytes, cudaStr
     p.quad_done = reinterpret_cast<unsigned *>(w + l.quad_off);
     p.qdep = reinterpret_cast<unsigned *>(w + l.qdep_off);
     p.qprog = reinterpret_cast<unsigned *>(w + l.qprog_off);
+    p.rowdone = reinterpret_cast<unsigned *>(w + l.rowdone_off);
     p.Ebuf = reinterpret_cast<double *>(w + l.e_off);
     p.Cbuf = reinterpret_cast<double *>(w + l.c_off);
     p.info = in.info;
@@ -1075,7 +1082,7 @@ static BatchedLayout batched_layout(int count, const TiledParams *pr) {
     for (int b = 0; b < count; ++b) {
         TiledLayout t = tiled_layout(pr[b].m, pr[b].n);
         size_t tiles = (size_t)t.ntm * t.ntn;
-        off += 2 * pad256(tiles * sizeof(unsigned)) + 2 * pad256(4 * tiles * sizeof(unsigned));
+        off += 2 * pad256(tiles * sizeof(unsigned)) + 2 * pad256(4 * tiles * sizeof(unsigned)) + pad256((size_t)t.ntm * sizeof(unsigned));
         bufs += 2 * pad256((size_t)t.ntm * T * (size_t)t.ntn * T * sizeof(double));
         l.ntiles += (long)tiles;
     }
@@ -1130,6 +1137,7 @@ int launch_round_tiled_batched(int count, const TiledParams *pr, double *min_mar
         d.quad_done = reinterpret_cast<unsigned *>(w + foff); foff += pad256(tiles * sizeof(unsigned));
         d.qdep = reinterpret_cast<unsigned *>(w + foff); foff += pad256(4 * tiles * sizeof(unsigned));
         d.qprog = reinterpret_cast<unsigned *>(w + foff); foff += pad256(4 * tiles * sizeof(unsigned));
+        d.rowdone = reinterpret_cast<unsigned *>(w + foff); foff += pad256((size_t)t.ntm * sizeof(unsigned));
         d.Ebuf = reinterpret_cast<double *>(w + boff); boff += mat;
         d.Cbuf = reinterpret_cast<double *>(w + boff); boff += mat;
         d.max_abs_e = reinterpret_cast<double *>(w + l.maxe_off) + b;
