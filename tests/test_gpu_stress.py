@@ -1,0 +1,66 @@
+"""Seeded random shapes through the tiled sweep: run-to-run bit-identity (a missing fence or a race in
+the streamed hand-over between quadrants would break it), agreement with the untiled Algorithm-3
+kernel (an independent implementation, itself checked against the oracle elsewhere), and the CPU
+oracle on a subset."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from oracle import cref
+
+pytestmark = pytest.mark.gpu
+
+MARGIN = 1e-9
+
+
+@pytest.fixture(scope="module")
+def g():
+    from paper_2607_27042_b200 import gptq2d
+    return gptq2d
+
+
+def make(rng, m, n):
+    X = rng.standard_normal((m, n)) * 4
+    L = np.tril(rng.standard_normal((m, m)) * (0.3 / np.sqrt(m)), -1) + np.eye(m)
+    U = np.triu(rng.standard_normal((n, n)) * (0.3 / np.sqrt(n)), 1) + np.eye(n)
+    return X, L, U
+
+
+def test_random_shapes_repeatable_and_equal_to_the_untiled_kernel(g):
+    rng = np.random.default_rng(2024)
+    shapes = [(int(rng.integers(1, 1100)), int(rng.integers(1, 1100))) for _ in range(24)]
+    shapes += [(128, 128), (129, 129), (64, 1300), (1300, 64), (127, 385), (1700, 1800)]
+    kept = []
+    for k, (m, n) in enumerate(shapes):
+        X, L, U = make(rng, m, n)
+        dX, dL, dU = (torch.from_numpy(a).cuda() for a in (X, L, U))
+        Z1, E1, m1, i1 = g.gptq2d_round(dX, dL, dU, want_E=True, want_margin=True)
+        Z2, E2, _, i2 = g.gptq2d_round(dX, dL, dU, want_E=True)
+        Zu, Eu, mu, iu = g.gptq2d_round(dX, dL, dU, precision=g.FP64_UNTILED, want_E=True, want_margin=True)
+        torch.cuda.synchronize()
+        for i in (i1, i2, iu):
+            g.check_info(i)
+        assert torch.equal(Z1, Z2) and torch.equal(E1, E2), (m, n)
+        margin = float(mu.cpu()[0])
+        assert abs(float(m1.cpu()[0]) - margin) < 1e-9
+        assert float((E1 - Eu).abs().max()) < 1e-9, (m, n)
+        if margin >= MARGIN:
+            assert torch.equal(Z1, Zu), (m, n)
+            if k % 6 == 0 and m * n <= 600 * 600:
+                ref = cref.nested(X, L, U)
+                assert np.array_equal(Z1.cpu().numpy().astype(np.int64), ref["Z"]), (m, n)
+        kept.append((dX, dL, dU, Z1))
+    # the same matrices again, a dozen at a time, in batched launches and through the host entry
+    for trial in range(3):
+        idx = rng.permutation(len(kept))[:12]
+        Zs, _, _, info = g.gptq2d_round_batched([kept[i][0] for i in idx], [kept[i][1] for i in idx],
+                                                [kept[i][2] for i in idx])
+        torch.cuda.synchronize()
+        g.check_info(info)
+        for k, i in enumerate(idx):
+            assert torch.equal(Zs[k], kept[i][3]), (trial, tuple(kept[i][0].shape))
+    for i in rng.permutation(len(kept))[:6]:
+        dX, dL, dU, Z1 = kept[i]
+        hZ, _ = g.gptq2d_round_host(dX.cpu().pin_memory(), dL.cpu().pin_memory(), dU.cpu().pin_memory())
+        assert torch.equal(hZ, Z1.cpu()), tuple(dX.shape)
