@@ -28,7 +28,7 @@
 //    running quadrant task waits -- bounded -- only on quadrants above it / to its left, which are
 //    running by then (or done).
 // Every CTA serves the ready ring first: at the top of its loop, while a far part waits, and
-// every few chunks of a far part (it then parks its partial sum and un-parks it afterwards).
+// every 64 chunks of a far part (its accumulator stays in registers meanwhile).
 // A far part only ever waits on tiles of earlier waves, whose far parts were claimed earlier and
 // whose quadrant tasks wait on running tasks only, so the earliest unfinished work can always
 // progress.
@@ -649,7 +649,7 @@ __device__ __forceinline__ void load_acc(Acc &acc, const double *srcT, long np, 
 // needs at most 512 slots (ntm, ntn <= 256 tiles would be 32768 rows); a batched launch sizes its
 // ring from the sum over its matrices.
 constexpr unsigned QCAP = 4096;
-constexpr int FAR_RUN_CHUNKS = 16;
+constexpr int FAR_RUN_CHUNKS = 64;
 constexpr unsigned IDLE_SLEEP_NS = 400; // a far part looks at the ready queue every this many K = 128 chunks
 
 // multi-producer / multi-consumer ring in global memory; slot value 0 = empty.
@@ -864,12 +864,8 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
         spins = 0;
 
         if (state == 1) {
-            // ================= A: quadrant tasks from the ready ring.  Never waits.  The live far part,
-            // if any, is parked first (the quadrant task needs the shared memory and the registers).
-            if (cur >= 0) {
-                if (s_ctx[cur][3] > 0) store_acc(acc, tile_region(cur), VIEW(s_ctx[cur][6]).np, wm, wn, g, t);
-                cur = -1;
-            }
+            // ================= A: quadrant tasks from the ready ring.  The accumulator of the live far part,
+            // if any, stays in its registers meanwhile: the quadrant task takes the shared memory only.
             unsigned e = s_pop;
             while (e != 0u) {
                 const TiledKernelParams &pq = VIEW(FAR_CTX);
