@@ -42,7 +42,10 @@ typedef enum {
     GPTQ2D_ERR_CUDA = 4,               /* a CUDA runtime call failed (launch, attribute query, copy)    */
     GPTQ2D_ERR_NOT_SPD = 5,            /* device: Gram pivot <= 0 or non-finite; info[1] = pivot index,
                                           info[2] = 0 for A^T A, 1 for B B^T                            */
-    GPTQ2D_ERR_NONFINITE = 6,          /* device: NaN/Inf met while rounding; info[1] = row, info[2] = col */
+    GPTQ2D_ERR_NONFINITE = 6,          /* device: NaN/Inf met while rounding; info[1] = row, info[2] = col of an
+                                          entry on the first anti-diagonal where one was met (inside an 8 x 8
+                                          block of the sweep a NaN also reaches neighbours that exact arithmetic
+                                          would spare, so this may be a neighbour of the offending input)    */
     GPTQ2D_ERR_INT_OVERFLOW = 7,       /* device: |corrected value| >= 2^31; info[1] = row, info[2] = col  */
     GPTQ2D_ERR_DEVICE_TIMEOUT = 8,     /* device: a bounded wait gave up; info[1] = where it waited     */
     GPTQ2D_ERR_TOO_LARGE = 9           /* gptq2d_round_static: m or n beyond GPTQ2D_STATIC_MAX_DIM;

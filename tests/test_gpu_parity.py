@@ -263,6 +263,26 @@ def test_host_entry_streams_inputs_while_sweeping(g, m, n, seed, pinned):
     assert np.array_equal(Ed, hE.numpy())
 
 
+def test_host_entry_reports_data_errors_and_stays_usable(g):
+    """A NaN in X through the streamed host entry: the status words come back, nothing hangs (the copy
+    stream's waits are released when the kernel ends), and the next call is fine."""
+    m, n = 700, 900
+    X, A, B = W.general_bases(m, n, 77)
+    L, U, _, _ = O.feedback_factors(A, B)
+    hX, hL, hU = (torch.from_numpy(np.ascontiguousarray(a)).pin_memory() for a in (X, L, U))
+    hZ = torch.zeros((m, n), dtype=torch.int32).pin_memory()
+    bad = hX.clone().pin_memory()
+    bad[300, 500] = float("nan")
+    with pytest.raises(g.Gptq2dError) as ei:
+        g.gptq2d_round_host(bad, hL, hU, hZ=hZ)
+    # the entry reported lies on the anti-diagonal of the first non-finite value, within one 8 x 8 leaf of it
+    assert ei.value.status == 6
+    assert ei.value.info[1] + ei.value.info[2] == 800 and abs(ei.value.info[1] - 300) < 8
+    g.gptq2d_round_host(hX, hL, hU, hZ=hZ)
+    Zd, _, _ = gpu_round(g, X, L, U, want_E=False)
+    assert np.array_equal(Zd, hZ.numpy())
+
+
 def test_two_streams_two_workspaces(g):
     """Calls on different streams with their own workspaces may be in flight together (the persistent
     launches take turns on the device); neither disturbs the other's result."""
