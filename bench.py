@@ -278,6 +278,22 @@ def run_cuda(args):
                             "objective_fp32": o32, "objective_fp64": o64, "relative_objective_gap": (o32 - o64) / o64}
         out["roofline"]["kernel"] = "round_untiled_kernel<float>"
         out["roofline"]["bound"] = "hbm"
+    if args.f32in:
+        # inputs kept in fp32, arithmetic in fp64: how far is the result from the one on the fp64 inputs?
+        Zf, _, _, infof = g.gptq2d_round_f32in(dX.float(), L.float(), U.float())
+        torch.cuda.synchronize()
+        g.check_info(infof)
+        o32 = float(g.gptq2d_objective(dX, Zf, dA, dB).cpu()[0])
+        o64 = float(g.gptq2d_objective(dX, Z, dA, dB).cpu()[0])
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        X32, L32, U32 = dX.float(), L.float(), U.float()
+        wsf = torch.empty(g.gptq2d_round_f32in_workspace_bytes(m, n), dtype=torch.uint8, device="cuda")
+        t0.record(stream)
+        g.gptq2d_round_f32in(X32, L32, U32, Z=Zf, workspace=wsf, info=infof, stream=stream)
+        t1.record(stream)
+        torch.cuda.synchronize()
+        out["f32_inputs"] = {"ms_per_sweep": t0.elapsed_time(t1), "z_mismatch_fraction": float((Zf != Z).double().mean().item()),
+                             "objective_f32_inputs": o32, "objective_fp64": o64, "relative_objective_gap": (o32 - o64) / o64}
     if args.pull:
         # every entry streams 2 (i + j) words: 8 m n (m + n) bytes in all
         pull_bytes = 8.0 * m * n * (m + n)
@@ -491,6 +507,8 @@ def main():
     ap.add_argument("--config", type=int, default=4, help="configuration index 0..4 (4 = 8192 x 8192 headline)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--fp32", action="store_true", help="time the fp32 mode instead")
+    ap.add_argument("--f32in", action="store_true",
+                    help="also run the sweep on fp32-stored inputs (fp64 arithmetic) and report the objective gap")
     ap.add_argument("--pull", action="store_true",
                     help="time the untiled pull-form kernel (Algorithm 6) instead: the memory-bound comparison point")
     ap.add_argument("--no-e2e", action="store_true")

@@ -213,6 +213,22 @@ int gptq2d_round_reverse(int m, int n,
                          double *E, long lde, double *min_margin,
                          void *workspace, size_t workspace_bytes, int *info, void *stream);
 
+/* ---- inputs stored in fp32, arithmetic in fp64 (the paper works in exact arithmetic and fixes no
+ * storage format; this is a packaging variant for callers that keep X and the factors in fp32) ----
+ * X, L, U are float arrays; they are widened to fp64 (exactly) into the workspace and the fp64 tiled
+ * sweep of gptq2d_round runs on them, so Z is exactly the trajectory of Algorithm 3 for the fp32-
+ * rounded data: against the sweep on the fp64 originals only the inputs' rounding differs (unlike
+ * GPTQ2D_FP32, which also computes in fp32).  Outputs, status words and stream behaviour as
+ * gptq2d_round.
+ */
+size_t gptq2d_round_f32in_workspace_bytes(int m, int n);
+int gptq2d_round_f32in(int m, int n,
+                       const float *X, long ldx,
+                       const float *L, long ldl, const float *U, long ldu,
+                       int32_t *Z, long ldz,
+                       double *E, long lde, double *min_margin,
+                       void *workspace, size_t workspace_bytes, int *info, void *stream);
+
 /* ---- the objective (Eq. 7): obj = || A (Z - X) B ||_F^2 ----
  * obj: device scalar.  A or B may be NULL (identity).
  */

@@ -1,3 +1,5 @@
+// Thin compositions around the forward kernels: reverse-order rounding and fp32-stored inputs.
+//
 // Reverse-order rounding (paper Section 2, "Two-sided and Kronecker-factored rounding": the same
 // greedy rounding taken from the last row and column towards the first).
 //
@@ -35,6 +37,18 @@ static bool flip(T *dst, long ldd, const T *src, long lds, int rows, int cols, i
         if (cudaGetLastError() != cudaSuccess) return false;
     }
     return true;
+}
+
+// dst (double, leading dimension ldd) = src (float, leading dimension lds)
+__global__ void widen_kernel(double *dst, long ldd, const float *src, long lds, int rows, int cols) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= cols) return;
+    for (int i = blockIdx.y; i < rows; i += gridDim.y) dst[(long)i * ldd + j] = (double)src[(long)i * lds + j];
+}
+static bool widen(double *dst, long ldd, const float *src, long lds, int rows, int cols, cudaStream_t stream) {
+    dim3 grid((cols + 255) / 256, rows < 65535 ? rows : 65535);
+    widen_kernel<<<grid, 256, 0, stream>>>(dst, ldd, src, lds, rows, cols);
+    return cudaGetLastError() == cudaSuccess;
 }
 
 static size_t pad256(size_t x) { return (x + 255) / 256 * 256; }
@@ -115,6 +129,34 @@ int gptq2d_round_reverse(int m, int n, const double *X, long ldx, const double *
     if (!flip(Z, ldz, Zp, (long)n, m, n, 1, 1, stream)) return GPTQ2D_ERR_CUDA;
     if (E && !flip(E, lde, Ep, (long)n, m, n, 1, 1, stream)) return GPTQ2D_ERR_CUDA;
     return GPTQ2D_OK;
+}
+
+size_t gptq2d_round_f32in_workspace_bytes(int m, int n) {
+    if (m < 1 || n < 1) return 0;
+    return pad256((size_t)m * n * 8) + pad256((size_t)m * m * 8) + pad256((size_t)n * n * 8) +
+           gptq2d_round_workspace_bytes(m, n, GPTQ2D_FP64);
+}
+
+int gptq2d_round_f32in(int m, int n, const float *X, long ldx, const float *L, long ldl, const float *U, long ldu,
+                       int32_t *Z, long ldz, double *E, long lde, double *min_margin, void *workspace,
+                       size_t workspace_bytes, int *info, void *stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (m < 1 || n < 1 || !X || !L || !U || !Z) return GPTQ2D_ERR_INVALID_ARG;
+    if (ldx < n || ldl < m || ldu < n || ldz < n || (E && lde < n)) return GPTQ2D_ERR_INVALID_ARG;
+    if (!aligned(X, 4) || !aligned(L, 4) || !aligned(U, 4) || !aligned(Z, 4) || !aligned(E, 8) ||
+        !aligned(min_margin, 8))
+        return GPTQ2D_ERR_INVALID_ARG;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gptq2d_round_f32in_workspace_bytes(m, n))
+        return GPTQ2D_ERR_WORKSPACE;
+    char *w = static_cast<char *>(workspace);
+    double *Xd = reinterpret_cast<double *>(w); w += pad256((size_t)m * n * 8);
+    double *Ld = reinterpret_cast<double *>(w); w += pad256((size_t)m * m * 8);
+    double *Ud = reinterpret_cast<double *>(w); w += pad256((size_t)n * n * 8);
+    if (!widen(Xd, (long)n, X, ldx, m, n, stream) || !widen(Ld, (long)m, L, ldl, m, m, stream) ||
+        !widen(Ud, (long)n, U, ldu, n, n, stream))
+        return GPTQ2D_ERR_CUDA;
+    return gptq2d_round(m, n, Xd, n, Ld, m, Ud, n, Z, ldz, E, lde, min_margin, GPTQ2D_FP64, w,
+                        gptq2d_round_workspace_bytes(m, n, GPTQ2D_FP64), info, stream_);
 }
 
 }  // extern "C"

@@ -33,6 +33,7 @@ EXPORTS = (
     "gptq2d_round_batched_workspace_bytes", "gptq2d_round_batched",
     "gptq2d_factor_reverse_workspace_bytes", "gptq2d_factor_reverse",
     "gptq2d_round_reverse_workspace_bytes", "gptq2d_round_reverse",
+    "gptq2d_round_f32in_workspace_bytes", "gptq2d_round_f32in",
 )
 
 BATCH_MAX_COUNT, BATCH_MAX_DIM = 8192, 32768
@@ -84,7 +85,10 @@ def _load():
     lib.gptq2d_round_static.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, vp]
     lib.gptq2d_round_static_max_dim.restype = sz
     lib.gptq2d_round_static_max_dim.argtypes = []
-    for name in ("gptq2d_factor_reverse_workspace_bytes", "gptq2d_round_reverse_workspace_bytes"):
+    lib.gptq2d_round_f32in.restype = i32
+    lib.gptq2d_round_f32in.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, sz, vp, vp]
+    for name in ("gptq2d_factor_reverse_workspace_bytes", "gptq2d_round_reverse_workspace_bytes",
+                 "gptq2d_round_f32in_workspace_bytes"):
         getattr(lib, name).restype = sz
         getattr(lib, name).argtypes = [i32, i32]
     lib.gptq2d_factor_reverse.restype = i32
@@ -255,6 +259,34 @@ def gptq2d_round_reverse(X, Lr, Ur, Z=None, E=None, min_margin=None, workspace=N
     pE, lde = _mat(E, torch.float64, "E")
     st = _lib.gptq2d_round_reverse(m, n, pX, ldx, pL, ldl, pU, ldu, pZ, ldz, pE, lde, _ptr(min_margin),
                                    _ptr(workspace), workspace.numel(), _ptr(info), _stream_ptr(stream))
+    if st != OK:
+        raise Gptq2dError(st)
+    return Z, E, min_margin, info
+
+
+def gptq2d_round_f32in_workspace_bytes(m, n):
+    return int(_lib.gptq2d_round_f32in_workspace_bytes(m, n))
+
+
+def gptq2d_round_f32in(X, L, U, Z=None, E=None, min_margin=None, workspace=None, info=None, stream=None,
+                       want_E=False, want_margin=False):
+    """The fp64 sweep on inputs stored in fp32 (float32 CUDA tensors).  Returns (Z, E, min_margin, info)."""
+    m, n = X.shape
+    dev = X.device
+    Z = torch.empty((m, n), dtype=torch.int32, device=dev) if Z is None else Z
+    if E is None and want_E:
+        E = torch.empty((m, n), dtype=torch.float64, device=dev)
+    if min_margin is None and want_margin:
+        min_margin = torch.empty(1, dtype=torch.float64, device=dev)
+    info = torch.zeros(4, dtype=torch.int32, device=dev) if info is None else info
+    workspace = _workspace(gptq2d_round_f32in_workspace_bytes(m, n), dev) if workspace is None else workspace
+    pX, ldx = _mat(X, torch.float32, "X")
+    pL, ldl = _mat(L, torch.float32, "L")
+    pU, ldu = _mat(U, torch.float32, "U")
+    pZ, ldz = _mat(Z, torch.int32, "Z")
+    pE, lde = _mat(E, torch.float64, "E")
+    st = _lib.gptq2d_round_f32in(m, n, pX, ldx, pL, ldl, pU, ldu, pZ, ldz, pE, lde, _ptr(min_margin),
+                                 _ptr(workspace), workspace.numel(), _ptr(info), _stream_ptr(stream))
     if st != OK:
         raise Gptq2dError(st)
     return Z, E, min_margin, info

@@ -95,3 +95,24 @@ def test_strided_outputs_and_identity_bases(g):
     g.check_info(info)
     assert np.array_equal(Zbig[:, :n].cpu().numpy(), np.rint(X).astype(np.int32))
     assert bool((Zbig[:, n:] == -3).all())
+
+
+@pytest.mark.parametrize("m,n,seed", [(17, 5, 0), (200, 330, 1), (515, 300, 2)])
+def test_fp32_stored_inputs_give_the_exact_trajectory_of_the_rounded_data(g, m, n, seed):
+    """gptq2d_round_f32in: inputs kept in fp32, arithmetic in fp64.  The oracle is the fp64 oracle on the
+    fp32-rounded data (exactly representable in fp64), so Z must be bit-exact against it."""
+    X, A, B = W.general_bases(m, n, seed)
+    L, U, _, _ = O.feedback_factors(A, B)
+    X32, L32, U32 = (a.astype(np.float32) for a in (X, L, U))
+    Xw, Lw, Uw = (a.astype(np.float64) for a in (X32, L32, U32))
+    ref = cref.nested(Xw, Lw, Uw)
+    margin, Eref = O.certificate_margin(Xw, ref["Z"], Lw, Uw)
+    if margin < MARGIN:
+        pytest.skip("seed not certified")
+    Z, E, mm, info = g.gptq2d_round_f32in(torch.from_numpy(X32).cuda(), torch.from_numpy(L32).cuda(),
+                                          torch.from_numpy(U32).cuda(), want_E=True, want_margin=True)
+    torch.cuda.synchronize()
+    g.check_info(info)
+    assert np.array_equal(Z.cpu().numpy().astype(np.int64), ref["Z"])
+    assert np.max(np.abs(E.cpu().numpy() - Eref)) < 1e-9
+    assert abs(float(mm.cpu()[0]) - margin) < 1e-9
