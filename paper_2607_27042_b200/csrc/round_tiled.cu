@@ -513,7 +513,7 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
         auto step_blk = [&](int i) {
             return i < olda ? fa + i : (i < olda + oldl ? fl + (i - olda) : (step_dir(i) == 0 ? r - 2 : c - 2));
         };
-        // three buffer pairs, so that up to three steps are in flight; all unused until the sweep proper
+        // three buffer pairs: one being multiplied, two being filled; all unused until the sweep proper
         auto bufA = [&](int j) { return j == 0 ? Lfa : (j == 1 ? LU : Ys); };
         auto bufB = [&](int j) { return j == 0 ? Ufl : (j == 1 ? Cs : tabL); };
         auto issue = [&](int i) {
@@ -538,16 +538,13 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
             else if (w < olda + oldl) await_progress(p, prog_of(r, fl + (w - olda)), nullptr, 15u);
         }
         __syncthreads();
-        for (int i = 0; i < ns && i < 3; ++i) issue(i);
+        for (int i = 0; i < ns && i < 2; ++i) issue(i);
         for (int i = 0; i < ns; ++i) {
-            const int pending = min(ns, i + 3) - (i + 1);        // groups issued after step i's
-            if (pending >= 2) cp_async_wait<2>(); else if (pending == 1) cp_async_wait<1>(); else cp_async_wait<0>();
+            if (i + 1 < ns) cp_async_wait<1>(); else cp_async_wait<0>();     // step i's operands have landed
             __syncthreads();
+            // every warp is past product i - 1 now, so its buffer pair, (i + 2) % 3, can take step i + 2
+            if (i + 2 < ns) issue(i + 2);
             if (step_dir(i) == 0) quad_mma(accC, bufA(i % 3), bufB(i % 3)); else quad_mma(accR, bufA(i % 3), bufB(i % 3));
-            if (i + 3 < ns) {
-                __syncthreads();
-                issue(i + 3);
-            }
         }
         __syncthreads();
     }
