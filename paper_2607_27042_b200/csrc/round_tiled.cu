@@ -257,9 +257,9 @@ __device__ __forceinline__ void quadrant_arrive(const TiledKernelParams &p, int 
 // row0/col0: global coordinates of the quadrant.
 //
 // Leaf-wave lw (leaves (a, lw - a), one per warp).  For lw <= 7, all warps first add what block lw
-// of the neighbours feeds into this quadrant (pull phase), and request block lw + 1.  Then every
-// leaf pulls the feedback of the leaves swept before it (leaf_pull), runs the 15 anti-diagonal
-// steps on its 8 x 8 entries and stores its results.
+// of the neighbours feeds into this quadrant (pull phase).  Then every leaf pulls the feedback of
+// the leaves swept before it (leaf_pull), runs the 15 anti-diagonal steps on its 8 x 8 entries and
+// stores its results, while warp 7 fetches block lw + 1 and warp 6 publishes the previous waves.
 __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const double *LU, const double *Lfa,
                                                const double *Ufl, double *stg, double *tabL, double *tabU, int row0,
                                                int col0, const Stream &sm, const TiledKernelParams &p,
@@ -646,8 +646,8 @@ __device__ __forceinline__ void load_acc(Acc &acc, const double *srcT, long np, 
 // needs at most 512 slots (ntm, ntn <= 256 tiles would be 32768 rows); a batched launch sizes its
 // ring from the sum over its matrices.
 constexpr unsigned QCAP = 4096;
-constexpr int FAR_RUN_CHUNKS = 64;
-constexpr unsigned IDLE_SLEEP_NS = 400; // a far part looks at the ready queue every this many K = 128 chunks
+constexpr int FAR_RUN_CHUNKS = 64;      // a far part looks at the ready ring every this many K = 128 chunks
+constexpr unsigned IDLE_SLEEP_NS = 400; // pause of a CTA that found nothing to do
 
 // multi-producer / multi-consumer ring in global memory; slot value 0 = empty.
 __device__ __forceinline__ void ready_push(const TiledKernelParams &p, unsigned entry) {
