@@ -16,7 +16,8 @@ Pins (see tests/test_oracle_pins.py): brute-force conditional minimiser that use
 A and B only; closed forms for 1x1 / 2x2; F == U^T (x) L; B = I column
 independence and an elimination-form GPTQ; A = B = I round-to-nearest; the
 Kronecker-vec identity; transpose symmetry; mutual agreement of Algorithms
-1, 2, 3, 5, 6; the integer-matrix certificate.  The reverse-order functions at the
+1, 2, 3, 4, 5, 6 (Algorithm 4 for block widths from 1 to one block that holds the
+whole sweep); the integer-matrix certificate.  The reverse-order functions at the
 end (Section 2, "Two-sided and Kronecker-factored rounding": the same rounding
 taken from the last row and column) are pinned by their own brute force, by
 F~ == U~^T (x) L~ and by the index-reversal identity with the forward functions.
@@ -31,7 +32,7 @@ __all__ = [
     "gram_pair", "kron_gram", "unit_lower_ldl_of_inverse_literal",
     "unit_lower_ldl_of_inverse", "feedback_factors", "adaptive_round_1d",
     "vec_sweep_explicit", "vec_sweep_implicit", "anti_diagonal",
-    "sweep_dense_antidiagonal", "sweep_gptq2d", "sweep_nested", "sweep_implicit_y",
+    "sweep_dense_antidiagonal", "sweep_gptq2d", "sweep_blocked", "sweep_nested", "sweep_implicit_y",
     "brute_force_trajectory", "local_errors_from_Z", "certificate_margin",
     "objective", "objective_kron", "objective_from_errors", "gptq_one_sided_elimination",
     "unit_upper_udu_of_inverse", "feedback_factors_reverse", "adaptive_round_1d_reverse",
@@ -218,6 +219,60 @@ def sweep_gptq2d(X, L, U):
             Y[i + 1:, j] += M[1:]
         for (i, j) in idx:
             Y[i, j + 1:] += C[i, j] * U[j, j + 1:]
+    out = _pack(Z, E)
+    out["C"] = C
+    return out
+
+
+def sweep_blocked(X, L, U, w):
+    """Algorithm 4 (blocked GPTQ-2D): the sweep in blocks of w anti-diagonals with ONE buffer
+    C = L E kept across blocks.  Inside a block Algorithm 3 runs with the fold and both pushes cut
+    off at the block's last anti-diagonal s1; after the block, every later entry receives the
+    rest at once: the down flush (the block's band of E in its column through L, added to Y and
+    to C) and the right flush (the block's band of C in its row through U, added to Y).
+
+    0-based: blocks start at s0 = 0, w, 2w, ... <= m+n-2 (the paper's 2, 2+w, ... in 1-based
+    index sums); index ranges are clipped to the matrix, so the last block may hold a single
+    anti-diagonal."""
+    Y = np.array(X, dtype=np.float64)
+    m, n = Y.shape
+    w = int(w)
+    if w < 1:
+        raise ValueError("block width must be positive")
+    Z = np.zeros((m, n))
+    E = np.zeros((m, n))
+    C = np.zeros((m, n))
+    last = m + n - 2
+    for s0 in range(0, last + 1, w):
+        s1 = min(s0 + w - 1, last)
+        for s in range(s0, s1 + 1):
+            idx = anti_diagonal(s, m, n)
+            for (i, j) in idx:
+                Z[i, j] = np.rint(Y[i, j])
+                E[i, j] = Z[i, j] - Y[i, j]
+                end = min(s1 - j, m - 1) + 1              # rows of column j still inside the block
+                M = L[i:end, i] * E[i, j]
+                C[i:end, j] += M
+                Y[i + 1:end, j] += M[1:]
+            for (i, j) in idx:
+                end = min(s1 - i, n - 1) + 1              # columns of row i still inside the block
+                Y[i, j + 1:end] += C[i, j] * U[j, j + 1:end]
+        # down flush: column j's part of the block is rows s0-j .. s1-j; everything below s1-j is later
+        for j in range(n):
+            lo, hi = max(s0 - j, 0), min(s1 - j, m - 1)
+            first = max(s1 - j + 1, 0)
+            if lo > hi or first >= m:
+                continue
+            M = L[first:, lo:hi + 1] @ E[lo:hi + 1, j]
+            C[first:, j] += M
+            Y[first:, j] += M
+        # right flush: row i's part of the block is columns s0-i .. s1-i
+        for i in range(m):
+            lo, hi = max(s0 - i, 0), min(s1 - i, n - 1)
+            first = max(s1 - i + 1, 0)
+            if lo > hi or first >= n:
+                continue
+            Y[i, first:] += C[i, lo:hi + 1] @ U[lo:hi + 1, first:]
     out = _pack(Z, E)
     out["C"] = C
     return out

@@ -176,6 +176,27 @@ def test_all_forms_share_the_trajectory(m, n, seed):
     assert np.allclose(g["Z"], X + L @ g["E"] @ U, atol=1e-10)
 
 
+@pytest.mark.parametrize("m,n,seed", [(6, 9, 0), (9, 6, 1), (12, 12, 2), (1, 7, 3), (7, 1, 4), (1, 1, 5), (23, 17, 6)])
+def test_blocked_form_shares_the_trajectory_for_every_block_width(m, n, seed):
+    """Algorithm 4 against the explicit vectorised sweep (Algorithm 1 under the Kronecker Gram), which
+    shares none of its steps: width 1 (no in-block push at all, every contribution arrives by a flush),
+    widths that leave a ragged last block or a last block of a single anti-diagonal, and one block that
+    holds the whole sweep (no flush at all)."""
+    X, A, B = _rand_general(m, n, seed)
+    L, U, _, _ = O.feedback_factors(A, B)
+    ref = O.vec_sweep_explicit(X, A, B)
+    assert ref["margin"] > 1e-7
+    widths = sorted({1, 2, 3, 5, 8, max(1, (m + n - 2) // 2), max(1, m + n - 2), m + n - 1, m + n + 5})
+    for w in widths:
+        o = O.sweep_blocked(X, L, U, w)
+        assert np.array_equal(o["Z"], ref["Z"]), w
+        assert np.allclose(o["E"], ref["E"], atol=1e-10), w
+        # the single buffer is complete at the end, whichever mix of folds and flushes filled it
+        assert np.allclose(o["C"], L @ o["E"], atol=1e-11), w
+    with pytest.raises(ValueError):
+        O.sweep_blocked(X, L, U, 0)
+
+
 def test_transpose_symmetry():
     X, A, B = _rand_general(5, 8, 17)
     Z = O.vec_sweep_explicit(X, A, B)["Z"]
