@@ -108,6 +108,12 @@ def job_value(m, n, world, ms_per_step):
     return world * m * n / (ms_per_step * 1e-3)
 
 
+def _entries_up_to(m, n, s):
+    """Number of entries (i, j) of an m x n matrix with i + j <= s."""
+    i = np.arange(m, dtype=np.int64)
+    return int(np.clip(s - i + 1, 0, n).sum())
+
+
 def host_entry_h2d_bytes(m, n, fp32):
     """Bytes gptq2d_round_host copies to the device: all of X, L, U in the fp32 mode; in the fp64 mode X
     plus the rows of L up to the end of each 512 x 512 diagonal block and the columns of U down to it."""
@@ -294,6 +300,29 @@ def run_cuda(args):
         torch.cuda.synchronize()
         out["f32_inputs"] = {"ms_per_sweep": t0.elapsed_time(t1), "z_mismatch_fraction": float((Zf != Z).double().mean().item()),
                              "objective_f32_inputs": o32, "objective_fp64": o64, "relative_objective_gap": (o32 - o64) / o64}
+    if args.blocked:
+        # Algorithm 4 with block width w on the same inputs: the paper's own blocked formulation as a comparison point
+        wb = args.blocked
+        wsb = torch.empty(g.gptq2d_round_blocked_workspace_bytes(m, n, wb), dtype=torch.uint8, device="cuda")
+        Zb = torch.empty((m, n), dtype=torch.int32, device="cuda")
+        infob = torch.zeros(4, dtype=torch.int32, device="cuda")
+        tb = []
+        for _ in range(2 + 3):
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0.record(stream)
+            g.gptq2d_round_blocked(dX, L, U, wb, Z=Zb, workspace=wsb, info=infob, stream=stream)
+            t1.record(stream)
+            torch.cuda.synchronize()
+            tb.append(t0.elapsed_time(t1))
+        g.check_info(infob)
+        bms = float(np.median(tb[2:]))
+        nblocks = (m + n - 2) // wb + 1
+        out["blocked"] = {"w": wb, "ms_per_sweep": bms, "z_equal_to_tiled": bool(torch.equal(Zb, Z)),
+                          "tflops": flops / (bms * 1e-3) / 1e12, "frac": flops / (bms * 1e-3) / 1e12 / FP64_NOMINAL_TFLOPS,
+                          "kernel_launches": 2 * nblocks, "times_slower_than_tiled": bms / kernel_ms,
+                          "flush_rw_bytes": 32.0 * sum(max(0, m * n - _entries_up_to(m, n, min(b * wb + wb - 1, m + n - 2)))
+                                                       for b in range(nblocks - 1))}
+        del wsb
     if args.pull:
         # every entry streams 2 (i + j) words: 8 m n (m + n) bytes in all
         pull_bytes = 8.0 * m * n * (m + n)
@@ -509,6 +538,8 @@ def main():
     ap.add_argument("--fp32", action="store_true", help="time the fp32 mode instead")
     ap.add_argument("--f32in", action="store_true",
                     help="also run the sweep on fp32-stored inputs (fp64 arithmetic) and report the objective gap")
+    ap.add_argument("--blocked", type=int, default=0, metavar="W",
+                    help="also time the blocked sweep (Algorithm 4) with block width W on the same inputs")
     ap.add_argument("--pull", action="store_true",
                     help="time the untiled pull-form kernel (Algorithm 6) instead: the memory-bound comparison point")
     ap.add_argument("--no-e2e", action="store_true")

@@ -229,6 +229,28 @@ int gptq2d_round_f32in(int m, int n,
                        double *E, long lde, double *min_margin,
                        void *workspace, size_t workspace_bytes, int *info, void *stream);
 
+/* ---- blocked GPTQ-2D (Algorithm 4, Section 4 "Blocked GPTQ-2D") as an alternative kernel ----
+ * The same rounding in blocks of w consecutive anti-diagonals, 1 <= w <= GPTQ2D_BLOCKED_MAX_WIDTH:
+ * inside a block the feedback stops at the block's last anti-diagonal; after it, a down flush (the
+ * block's band of E through L, added to Y and to the buffer C = L E) and a right flush (the block's
+ * band of C through U, added to Y) reach every later entry.  By the paper's correctness argument Z
+ * equals that of gptq2d_round for every w.  X, L, U, Z, E, min_margin, info, stream: as gptq2d_round
+ * (all device memory; only the strictly lower part of L and the strictly upper part of U are read).
+ * Two kernel launches per block, (m + n - 2) / w + 1 blocks.  The workspace holds Y, C and E.
+ * Returns GPTQ2D_ERR_INVALID_ARG for a width outside the range (the workspace size is then 0).
+ * This is the paper's own GPU formulation kept as a comparison point: it re-reads every later entry
+ * once per block and is slower than the tiled sweep at every size.
+ */
+#define GPTQ2D_BLOCKED_MAX_WIDTH 64
+size_t gptq2d_round_blocked_workspace_bytes(int m, int n, int w);
+int gptq2d_round_blocked(int m, int n,
+                         const double *X, long ldx,
+                         const double *L, long ldl, const double *U, long ldu,
+                         int w,
+                         int32_t *Z, long ldz,
+                         double *E, long lde, double *min_margin,
+                         void *workspace, size_t workspace_bytes, int *info, void *stream);
+
 /* ---- the objective (Eq. 7): obj = || A (Z - X) B ||_F^2 ----
  * obj: device scalar.  A or B may be NULL (identity).
  */

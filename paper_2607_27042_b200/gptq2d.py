@@ -34,7 +34,10 @@ EXPORTS = (
     "gptq2d_factor_reverse_workspace_bytes", "gptq2d_factor_reverse",
     "gptq2d_round_reverse_workspace_bytes", "gptq2d_round_reverse",
     "gptq2d_round_f32in_workspace_bytes", "gptq2d_round_f32in",
+    "gptq2d_round_blocked_workspace_bytes", "gptq2d_round_blocked",
 )
+
+BLOCKED_MAX_WIDTH = 64
 
 BATCH_MAX_COUNT, BATCH_MAX_DIM = 8192, 32768
 
@@ -87,6 +90,10 @@ def _load():
     lib.gptq2d_round_static_max_dim.argtypes = []
     lib.gptq2d_round_f32in.restype = i32
     lib.gptq2d_round_f32in.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, sz, vp, vp]
+    lib.gptq2d_round_blocked_workspace_bytes.restype = sz
+    lib.gptq2d_round_blocked_workspace_bytes.argtypes = [i32, i32, i32]
+    lib.gptq2d_round_blocked.restype = i32
+    lib.gptq2d_round_blocked.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, i32, vp, lng, vp, lng, vp, vp, sz, vp, vp]
     for name in ("gptq2d_factor_reverse_workspace_bytes", "gptq2d_round_reverse_workspace_bytes",
                  "gptq2d_round_f32in_workspace_bytes"):
         getattr(lib, name).restype = sz
@@ -287,6 +294,35 @@ def gptq2d_round_f32in(X, L, U, Z=None, E=None, min_margin=None, workspace=None,
     pE, lde = _mat(E, torch.float64, "E")
     st = _lib.gptq2d_round_f32in(m, n, pX, ldx, pL, ldl, pU, ldu, pZ, ldz, pE, lde, _ptr(min_margin),
                                  _ptr(workspace), workspace.numel(), _ptr(info), _stream_ptr(stream))
+    if st != OK:
+        raise Gptq2dError(st)
+    return Z, E, min_margin, info
+
+
+def gptq2d_round_blocked_workspace_bytes(m, n, w):
+    return int(_lib.gptq2d_round_blocked_workspace_bytes(m, n, w))
+
+
+def gptq2d_round_blocked(X, L, U, w, Z=None, E=None, min_margin=None, workspace=None, info=None, stream=None,
+                         want_E=False, want_margin=False):
+    """Blocked GPTQ-2D (Algorithm 4) with block width w.  Returns (Z, E, min_margin, info)."""
+    m, n = X.shape
+    dev = X.device
+    Z = torch.empty((m, n), dtype=torch.int32, device=dev) if Z is None else Z
+    if E is None and want_E:
+        E = torch.empty((m, n), dtype=torch.float64, device=dev)
+    if min_margin is None and want_margin:
+        min_margin = torch.empty(1, dtype=torch.float64, device=dev)
+    info = torch.zeros(4, dtype=torch.int32, device=dev) if info is None else info
+    if workspace is None:
+        workspace = _workspace(gptq2d_round_blocked_workspace_bytes(m, n, w), dev)
+    pX, ldx = _mat(X, torch.float64, "X")
+    pL, ldl = _mat(L, torch.float64, "L")
+    pU, ldu = _mat(U, torch.float64, "U")
+    pZ, ldz = _mat(Z, torch.int32, "Z")
+    pE, lde = _mat(E, torch.float64, "E")
+    st = _lib.gptq2d_round_blocked(m, n, pX, ldx, pL, ldl, pU, ldu, int(w), pZ, ldz, pE, lde, _ptr(min_margin),
+                                   _ptr(workspace), workspace.numel(), _ptr(info), _stream_ptr(stream))
     if st != OK:
         raise Gptq2dError(st)
     return Z, E, min_margin, info
