@@ -51,6 +51,13 @@ def test_full_config_certificate(index):
         i, j = int(rng.integers(m)), int(rng.integers(n))
         y = X[i, j] + L[i, :i + 1] @ Ecert[:i + 1, :j + 1] @ U[:j + 1, j] - Ecert[i, j]
         assert Zh[i, j] == int(np.rint(y))
+    # the blocked sweep (Algorithm 4) must land on the same certified Z
+    Zb, _, mb, infob = g.gptq2d_round_blocked(dX, Ld, Ud, 64, want_margin=True)
+    torch.cuda.synchronize()
+    g.check_info(infob)
+    assert np.array_equal(Zb.cpu().numpy().astype(np.int64), Zh)
+    assert abs(float(mb.cpu()[0]) - margin) < 1e-8
+    del Zb
     obj = float(g.gptq2d_objective(dX, Z, dA, dB).cpu()[0])
     want = O.objective(X, Zh, A, B)
     assert abs(obj - want) <= 1e-10 * want
