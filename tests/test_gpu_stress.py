@@ -64,3 +64,30 @@ def test_random_shapes_repeatable_and_equal_to_the_untiled_kernel(g):
         dX, dL, dU, Z1 = kept[i]
         hZ, _ = g.gptq2d_round_host(dX.cpu().pin_memory(), dL.cpu().pin_memory(), dU.cpu().pin_memory())
         assert torch.equal(hZ, Z1.cpu()), tuple(dX.shape)
+
+
+def test_random_shapes_and_widths_through_the_blocked_sweep(g):
+    """Algorithm 4 on seeded random shapes and block widths against the oracle's plain-C nested sweep
+    (Z bit-exact where the certificate's margin allows it, E and the margin always), and run-to-run
+    bit-identity (the CTAs of a block recompute each other's rows: the copies must agree bit for bit)."""
+    rng = np.random.default_rng(4)
+    cases = [(int(rng.integers(1, 500)), int(rng.integers(1, 500)), int(rng.integers(1, 65))) for _ in range(16)]
+    cases += [(64, 64, 64), (65, 63, 63), (128, 129, 17), (1, 300, 64), (300, 1, 5), (257, 511, 64)]
+    checked = 0
+    for (m, n, w) in cases:
+        X, L, U = make(rng, m, n)
+        ref = cref.nested(X, L, U)
+        margin, Eref = O.certificate_margin(X, ref["Z"], L, U)
+        dX, dL, dU = (torch.from_numpy(a).cuda() for a in (X, L, U))
+        Z1, E1, m1, i1 = g.gptq2d_round_blocked(dX, dL, dU, w, want_E=True, want_margin=True)
+        Z2, E2, _, i2 = g.gptq2d_round_blocked(dX, dL, dU, w, want_E=True)
+        torch.cuda.synchronize()
+        g.check_info(i1)
+        g.check_info(i2)
+        assert torch.equal(Z1, Z2) and torch.equal(E1, E2), (m, n, w)
+        if margin >= MARGIN:
+            assert np.array_equal(Z1.cpu().numpy().astype(np.int64), ref["Z"]), (m, n, w)
+            assert np.max(np.abs(E1.cpu().numpy() - Eref)) < 1e-9, (m, n, w)
+            assert abs(float(m1.cpu()[0]) - margin) < 1e-9, (m, n, w)
+            checked += 1
+    assert checked >= len(cases) // 2
