@@ -273,7 +273,7 @@ def run_cuda(args):
         "per_step_ms": per_step,
     }
     if args.fp32:
-        # the optional fp32 mode is judged against the fp64 sweep of the same inputs
+        # the optional fp32 mode is compared with the fp64 sweep of the same inputs
         ws64 = torch.empty(g.gptq2d_round_workspace_bytes(m, n, g.FP64), dtype=torch.uint8, device="cuda")
         Z64, _, _, info64 = g.gptq2d_round(dX, L, U, precision=g.FP64, workspace=ws64)
         torch.cuda.synchronize()
