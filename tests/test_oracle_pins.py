@@ -197,6 +197,35 @@ def test_blocked_form_shares_the_trajectory_for_every_block_width(m, n, seed):
         O.sweep_blocked(X, L, U, 0)
 
 
+def test_blocked_form_random_shapes_and_widths_and_its_block_invariant():
+    """Seeded random (m, n, w): Algorithm 4 against the nested column sweep (Algorithm 5), plus the state
+    the correctness argument of Section 4 rests on: once every block is flushed, a later entry's Y is
+    X + (L E U) over the entries rounded so far -- checked by stopping after the first block through a
+    width that holds exactly that block and comparing with Eq. 11 on the partial E."""
+    rng = np.random.default_rng(77)
+    for _ in range(24):
+        m, n = int(rng.integers(1, 20)), int(rng.integers(1, 20))
+        w = int(rng.integers(1, m + n + 2))
+        X, A, B = _rand_general(m, n, int(rng.integers(1 << 30)))
+        L, U, _, _ = O.feedback_factors(A, B)
+        ref = O.sweep_nested(X, L, U)
+        if ref["margin"] < 1e-7:
+            continue
+        o = O.sweep_blocked(X, L, U, w)
+        assert np.array_equal(o["Z"], ref["Z"]), (m, n, w)
+        assert np.allclose(o["E"], ref["E"], atol=1e-10), (m, n, w)
+        # partial state: zero the errors of everything after the first block; Eq. 11 then gives the
+        # corrected value every later entry must have been handed by the flushes, and rounding the
+        # first entry of the second block from it must reproduce Z there
+        s1 = min(w - 1, m + n - 2)
+        if s1 < m + n - 2:
+            idx = np.add.outer(np.arange(m), np.arange(n))
+            Epart = np.where(idx <= s1, o["E"], 0.0)
+            Ypart = X + L @ Epart @ U
+            for (i, j) in O.anti_diagonal(s1 + 1, m, n):
+                assert np.rint(Ypart[i, j]) == o["Z"][i, j], (m, n, w, i, j)
+
+
 def test_transpose_symmetry():
     X, A, B = _rand_general(5, 8, 17)
     Z = O.vec_sweep_explicit(X, A, B)["Z"]
