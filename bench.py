@@ -269,7 +269,8 @@ def run_cuda(args):
                    "timed": "gptq2d_round (init + sweep); factorisation timed separately"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps,
         "roofline": roofline, "factor_ms": factor_ms,
-        "factor_tflops": (2.0 * (m ** 3 + n ** 3) * (1.0 / 2 + 1.0 / 3 + 2.0 / 3)) / (factor_ms * 1e-3) / 1e12,
+        # set-up flops per side of order k: Gram (lower tiles) k^3, reverse Cholesky k^3 / 3, triangular inverse k^3 / 3
+        "factor_tflops": ((m ** 3 + n ** 3) * (1.0 + 1.0 / 3 + 1.0 / 3)) / (factor_ms * 1e-3) / 1e12,
         "per_step_ms": per_step,
     }
     if args.fp32:

@@ -230,6 +230,7 @@ int factor_one_side(int k, const double *M, long ldm, int side, double *out, lon
             g1.B = X + off11; g1.ldb = ld; g1.strideB = stride;
             g1.C = T + off21; g1.ldc = ld; g1.strideC = stride;
             g1.batch = (int)cnt;
+            g1.b_lower = 1;  // X11 is lower triangular
             CK(launch_gemm(g1, stream));
             GemmArgs g2{};   // X21 = -X22 T21
             g2.opA = OP_N; g2.opB = OP_N;
@@ -239,6 +240,7 @@ int factor_one_side(int k, const double *M, long ldm, int side, double *out, lon
             g2.B = T + off21; g2.ldb = ld; g2.strideB = stride;
             g2.C = X + off21; g2.ldc = ld; g2.strideC = stride;
             g2.batch = (int)cnt;
+            g2.a_lower = 1;  // X22 is lower triangular
             CK(launch_gemm(g2, stream));
         }
     }

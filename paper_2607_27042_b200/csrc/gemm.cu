@@ -27,9 +27,15 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(GemmArgs p) {
     B.mn_valid = min(BN, p.N - n0);
     B.aligned16 = ((((uintptr_t)B.ptr) & 15) == 0) && ((p.ldb & 1) == 0);
 
+    // k-range of this tile (whole range unless an operand is triangular); both ends are multiples of 128
+    const int k_lo = p.b_lower ? min(p.K, n0) : 0;
+    const int k_hi = p.a_lower ? min(p.K, m0 + BM) : p.K;
+    A.ptr += A_KCONTIG ? (long)k_lo : (long)k_lo * p.lda;
+    B.ptr += B_KCONTIG ? (long)k_lo : (long)k_lo * p.ldb;
+
     Acc acc;
     acc.zero();
-    gemm_tile<A_KCONTIG, B_KCONTIG, GEMM_NSTAGE>(acc, smem, A, B, p.K);
+    if (k_hi > k_lo) gemm_tile<A_KCONTIG, B_KCONTIG, GEMM_NSTAGE>(acc, smem, A, B, k_hi - k_lo);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int wm = warp >> 2, wn = warp & 3, g = lane >> 2, t = lane & 3;

@@ -18,6 +18,9 @@ struct GemmArgs {
     double *C; long ldc; long strideC;
     int batch;
     int lower_tiles_only;   // skip 128 x 128 output tiles strictly above the block diagonal
+    // Triangular operands: the part of the contraction that only meets structural zeros is skipped.
+    int a_lower;            // op(A) is lower triangular (M x K, zero for k > m): tile row tm stops at k = 128 (tm + 1)
+    int b_lower;            // op(B) is lower triangular (K x N, zero for k < n): tile column tn starts at k = 128 tn
     double *sumsq_partials; // if non-null: do not store C; write sum(C^2) of each CTA tile
                             // to sumsq_partials[tile index] (tiles_m * tiles_n * batch entries)
 };
