@@ -50,10 +50,35 @@ __global__ void __launch_bounds__(256) factor_diag_kernel(double *S, long lds, i
         if (tid == 0) a[k * 129 + k] = pk;
         for (int i = tid; i < k; i += blockDim.x) a[k * 129 + i] *= rk;     // P[k][i], i < k
         __syncthreads();
-        // Schur complement of the leading k x k part (lower triangle)
-        for (int i = ty; i < k; i += 16) {
-            const double pi = a[k * 129 + i];
-            for (int j = tx; j <= i; j += 16) a[i * 129 + j] = fma(-pi, a[k * 129 + j], a[i * 129 + j]);
+        // Schur complement of the leading k x k part (lower triangle).  The row of P and each thread's
+        // eight entries of a row of the complement are read into registers before anything is stored, so
+        // that the loads are in flight together (loads and stores of the same array cannot be reordered
+        // by the compiler).
+        {
+            // every index below is < 128, so all loads are unconditional; only the stores are masked
+            double pj[8];
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) pj[jj] = a[k * 129 + tx + 16 * jj];
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                double pi[4], v[4][8];
+#pragma unroll
+                for (int ii = 0; ii < 4; ++ii) {
+                    const int i = ty + 16 * (4 * half + ii);
+                    pi[ii] = a[k * 129 + i];
+#pragma unroll
+                    for (int jj = 0; jj < 8; ++jj) v[ii][jj] = a[i * 129 + tx + 16 * jj];
+                }
+#pragma unroll
+                for (int ii = 0; ii < 4; ++ii) {
+                    const int i = ty + 16 * (4 * half + ii);
+#pragma unroll
+                    for (int jj = 0; jj < 8; ++jj) {
+                        const int j = tx + 16 * jj;
+                        if (i < k && j <= i) a[i * 129 + j] = fma(-pi[ii], pj[jj], v[ii][jj]);
+                    }
+                }
+            }
         }
         __syncthreads();
     }
