@@ -76,6 +76,11 @@ const char *gptq2d_status_string(int status);
  * A or B may be NULL, meaning the identity (L or U is then the identity).
  * Device error: GPTQ2D_ERR_NOT_SPD when a Gram is numerically not positive definite
  * (A or B singular); L and U are then undefined.
+ * Streams: everything is ordered after the work already on `stream`, and `stream` waits for all of it
+ * before the call's outputs are used by later work on it.  With both bases given, part of the work runs
+ * on streams of the library's own (per device, created on first use: the B side next to the A side, and
+ * each side's chain of diagonal blocks ahead of its large updates); concurrent calls on one device are
+ * serialised while they enqueue.
  */
 size_t gptq2d_factor_workspace_bytes(int m, int n);
 int gptq2d_factor(int m, int n,

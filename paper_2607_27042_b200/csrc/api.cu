@@ -2,14 +2,11 @@
 #include <cuda_runtime.h>
 #include "common.cuh"
 #include "round_internal.cuh"
+#include "factor.cuh"
 #include <mutex>
 #include <vector>
 
 namespace gptq2d {
-size_t factor_workspace_bytes(int m, int n);
-size_t factor_side_workspace_bytes(int k);
-int factor_one_side(int k, const double *M, long ldm, int side, double *out, long ldo, double *dinv, void *ws,
-                    int *info, cudaStream_t stream);
 size_t objective_workspace_bytes(int m, int n);
 int launch_objective(int m, int n, const double *X, long ldx, const int *Z, long ldz, const double *A, long lda,
                      const double *B, long ldb, double *obj, void *ws, cudaStream_t stream);
@@ -38,6 +35,7 @@ typedef int (*StreamWaitValue32Fn)(cudaStream_t, unsigned long long, unsigned in
 struct HostPipe {
     cudaStream_t copy = nullptr;
     cudaEvent_t inputs_free = nullptr, copies_done = nullptr;
+    FactorLookahead look[2] = {};            // per side of the set-up: spine stream and its events (spine == NULL: none)
     StreamWriteValue32Fn write32 = nullptr;
     StreamWaitValue32Fn wait32 = nullptr;    // stream-ordered wait until a device word is >= a value
     bool tried = false;
@@ -63,6 +61,17 @@ static HostPipe *host_pipe() {
         ok = ok && cudaStreamCreateWithFlags(&hp.copy, cudaStreamNonBlocking) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&hp.inputs_free, cudaEventDisableTiming) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&hp.copies_done, cudaEventDisableTiming) == cudaSuccess;
+        for (int sd = 0; ok && sd < 2; ++sd) {
+            FactorLookahead &lk = hp.look[sd];
+            cudaEvent_t *ev[5] = {&lk.fork, &lk.join, &lk.panel, &lk.t2[0], &lk.t2[1]};
+            // highest priority: the one-CTA spine kernels must get an SM as soon as one is free, ahead of the
+            // queued CTAs of the large updates
+            int prio_lo = 0, prio_hi = 0;
+            bool lok = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) == cudaSuccess &&
+                       cudaStreamCreateWithPriority(&lk.spine, cudaStreamNonBlocking, prio_hi) == cudaSuccess;
+            for (int e = 0; lok && e < 5; ++e) lok = cudaEventCreateWithFlags(ev[e], cudaEventDisableTiming) == cudaSuccess;
+            if (!lok) lk.spine = nullptr;        // the set-up then runs that side on one stream
+        }
         if (ok) { hp.write32 = reinterpret_cast<StreamWriteValue32Fn>(fn); hp.wait32 = reinterpret_cast<StreamWaitValue32Fn>(fnw); }
         (void)cudaGetLastError();
     }
@@ -134,16 +143,16 @@ int gptq2d_factor(int m, int n, const double *A, long lda, const double *B, long
     char *wsB = static_cast<char *>(workspace) + factor_side_workspace_bytes(m);
     HostPipe *hp = (A && B) ? host_pipe() : nullptr;
     if (!hp) {
-        st = factor_one_side(m, A, lda, 0, L, ldl, dL, workspace, info, stream);
+        st = factor_one_side(m, A, lda, 0, L, ldl, dL, workspace, info, stream, nullptr);
         if (st != GPTQ2D_OK) return st;
-        return factor_one_side(n, B, ldb, 1, U, ldu, dU, wsB, info, stream);
+        return factor_one_side(n, B, ldb, 1, U, ldu, dU, wsB, info, stream, nullptr);
     }
     std::unique_lock<std::mutex> lock(hp->enqueue);
     if (cudaEventRecord(hp->inputs_free, stream) != cudaSuccess ||
         cudaStreamWaitEvent(hp->copy, hp->inputs_free, 0) != cudaSuccess)
         return GPTQ2D_ERR_CUDA;
-    st = factor_one_side(m, A, lda, 0, L, ldl, dL, workspace, info, stream);
-    int st2 = factor_one_side(n, B, ldb, 1, U, ldu, dU, wsB, info, hp->copy);
+    st = factor_one_side(m, A, lda, 0, L, ldl, dL, workspace, info, stream, hp->look[0].spine ? &hp->look[0] : nullptr);
+    int st2 = factor_one_side(n, B, ldb, 1, U, ldu, dU, wsB, info, hp->copy, hp->look[1].spine ? &hp->look[1] : nullptr);
     // join even if an enqueue failed, so that nothing of this call is left running behind the caller's stream
     if (cudaEventRecord(hp->copies_done, hp->copy) != cudaSuccess ||
         cudaStreamWaitEvent(stream, hp->copies_done, 0) != cudaSuccess)

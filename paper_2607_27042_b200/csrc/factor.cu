@@ -15,6 +15,7 @@
 // and a final column scaling (transposed on the way out for U).
 #include "common.cuh"
 #include "gemm.cuh"
+#include "factor.cuh"
 
 namespace gptq2d {
 
@@ -185,7 +186,7 @@ size_t factor_workspace_bytes(int m, int n) { return factor_side_workspace_bytes
 
 // side 0: S = M^T M -> out = F (unit lower).  side 1: S = M M^T -> out = F^T (unit upper).
 int factor_one_side(int k, const double *M, long ldm, int side, double *out, long ldo, double *dinv, void *ws,
-                    int *info, cudaStream_t stream) {
+                    int *info, cudaStream_t stream, const FactorLookahead *look) {
     if (!M) {
         long tot = (long)k * k;
         identity_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, stream>>>(out, ldo, k, dinv);
@@ -213,28 +214,75 @@ int factor_one_side(int k, const double *M, long ldm, int side, double *out, lon
     }
     const size_t diag_smem = (128 * 129 + 128 * 129 / 2) * sizeof(double);
     CK(cudaFuncSetAttribute(factor_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)diag_smem));
-    for (int K = nblk - 1; K >= 0; --K) {
+    auto diag = [&](int K, cudaStream_t s) -> int {
         const long k0 = (long)K * FB;
         const int bs = (int)((k - k0) < FB ? (k - k0) : FB);
-        double *Gkk = G + k0 * ld + k0;
-        double *Wkk = X + k0 * ld + k0;
-        factor_diag_kernel<<<1, 256, diag_smem, stream>>>(Gkk, ld, bs, Wkk, ld, p + k0, info, side, (int)k0);
+        factor_diag_kernel<<<1, 256, diag_smem, s>>>(G + k0 * ld + k0, ld, bs, X + k0 * ld + k0, ld, p + k0, info, side,
+                                                     (int)k0);
         CK(cudaGetLastError());
-        if (K == 0) break;
-        GemmArgs g{};   // panel, in place: P_K,0:k0 = W^T G_K,0:k0
+        return GPTQ2D_OK;
+    };
+    auto panel = [&](int K, cudaStream_t s) -> int {       // in place: P_K,0:k0 = W^T G_K,0:k0
+        const long k0 = (long)K * FB;
+        const int bs = (int)((k - k0) < FB ? (k - k0) : FB);
+        GemmArgs g{};
         g.opA = OP_T; g.opB = OP_N;
         g.M = bs; g.N = (int)k0; g.K = bs;
         g.alpha = 1.0; g.beta = 0.0;
-        g.A = Wkk; g.lda = ld; g.B = G + k0 * ld; g.ldb = ld;
+        g.A = X + k0 * ld + k0; g.lda = ld; g.B = G + k0 * ld; g.ldb = ld;
         g.C = G + k0 * ld; g.ldc = ld; g.batch = 1;
-        CK(launch_gemm(g, stream));
-        GemmArgs t{};   // trailing: G_0:k0,0:k0 -= panel^T panel
+        CK(launch_gemm(g, s));
+        return GPTQ2D_OK;
+    };
+    // trailing update with the panel of block row K: rows [r0, r1) of the leading part,
+    // G[r0:r1, 0:r1] -= P_K,r0:r1^T P_K,0:r1 (lower tiles only when the rows start at 0)
+    auto trailing = [&](int K, long r0, long r1, cudaStream_t s) -> int {
+        const long k0 = (long)K * FB;
+        const int bs = (int)((k - k0) < FB ? (k - k0) : FB);
+        if (r1 <= r0) return GPTQ2D_OK;
+        GemmArgs t{};
         t.opA = OP_T; t.opB = OP_N;
-        t.M = t.N = (int)k0; t.K = bs;
+        t.M = (int)(r1 - r0); t.N = (int)r1; t.K = bs;
         t.alpha = -1.0; t.beta = 1.0;
-        t.A = G + k0 * ld; t.lda = ld; t.B = G + k0 * ld; t.ldb = ld;
-        t.C = G; t.ldc = ld; t.batch = 1; t.lower_tiles_only = 1;
-        CK(launch_gemm(t, stream));
+        t.A = G + k0 * ld + r0; t.lda = ld; t.B = G + k0 * ld; t.ldb = ld;
+        t.C = G + r0 * ld; t.ldc = ld; t.batch = 1; t.lower_tiles_only = r0 == 0 ? 1 : 0;
+        CK(launch_gemm(t, s));
+        return GPTQ2D_OK;
+    };
+    if (!look || nblk < 4) {
+        for (int K = nblk - 1; K >= 0; --K) {
+            int st = diag(K, stream);
+            if (st != GPTQ2D_OK) return st;
+            if (K == 0) break;
+            if ((st = panel(K, stream)) != GPTQ2D_OK || (st = trailing(K, 0, (long)K * FB, stream)) != GPTQ2D_OK) return st;
+        }
+    } else {
+        // Spine (diag K, panel K, then the update of block row K-1, which the next diagonal block needs) on
+        // look->spine; the update of rows 0 .. K-2 with panel K on `stream`.  What diag K reads has been
+        // updated by the row update of K+1 (same stream, before it) and by the large updates of K+2 and
+        // earlier; the row update of K and the large update of K+1 both write block row K-1, so the former
+        // waits for the latter.  An event waited on takes its latest record at the time of the call, so two
+        // alternating events tell the large updates of K+2 and K+1 apart.
+        cudaStream_t sp = look->spine;
+        CK(cudaEventRecord(look->fork, stream));
+        CK(cudaStreamWaitEvent(sp, look->fork, 0));
+        for (int K = nblk - 1; K >= 0; --K) {
+            if (K + 2 <= nblk - 1) CK(cudaStreamWaitEvent(sp, look->t2[(K + 2) & 1], 0));
+            int st = diag(K, sp);
+            if (st != GPTQ2D_OK) return st;
+            if (K == 0) break;
+            if ((st = panel(K, sp)) != GPTQ2D_OK) return st;
+            CK(cudaEventRecord(look->panel, sp));
+            if (K + 1 <= nblk - 1 && K + 1 >= 2) CK(cudaStreamWaitEvent(sp, look->t2[(K + 1) & 1], 0));
+            if ((st = trailing(K, (long)(K - 1) * FB, (long)K * FB, sp)) != GPTQ2D_OK) return st;
+            if (K >= 2) {
+                CK(cudaStreamWaitEvent(stream, look->panel, 0));
+                if ((st = trailing(K, 0, (long)(K - 1) * FB, stream)) != GPTQ2D_OK) return st;
+                CK(cudaEventRecord(look->t2[K & 1], stream));
+            }
+        }
+        CK(cudaEventRecord(look->join, sp));
+        CK(cudaStreamWaitEvent(stream, look->join, 0));
     }
     // X = P^{-1}: diagonal blocks are in place; double the block size level by level
     for (long b = FB; b < k; b *= 2) {
