@@ -35,9 +35,19 @@ __global__ void __launch_bounds__(256) factor_diag_kernel(double *S, long lds, i
     double *a = sm;               // [128][129]: P in the lower triangle, scratch above it
     double *w = sm + 128 * 129;   // packed lower triangle of W
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-    for (int idx = tid; idx < 128 * 128; idx += blockDim.x) {
-        int i = idx >> 7, j = idx & 127;
-        if (j <= i) a[i * 129 + j] = (i < bs) ? S[(long)i * lds + j] : (i == j ? 1.0 : 0.0);
+    // the block, padded with the identity: eight loads in flight per thread
+    for (int base = 0; base < 128 * 128; base += 8 * 256) {
+        double v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int idx = base + u * 256 + tid, i = idx >> 7, j = idx & 127;
+            v[u] = (j <= i && i < bs) ? S[(long)i * lds + j] : (i == j ? 1.0 : 0.0);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int idx = base + u * 256 + tid, i = idx >> 7, j = idx & 127;
+            if (j <= i) a[i * 129 + j] = v[u];
+        }
     }
     __syncthreads();
     for (int k = bs - 1; k >= 0; --k) {
@@ -214,6 +224,8 @@ int factor_one_side(int k, const double *M, long ldm, int side, double *out, lon
     }
     const size_t diag_smem = (128 * 129 + 128 * 129 / 2) * sizeof(double);
     CK(cudaFuncSetAttribute(factor_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)diag_smem));
+    CK(cudaFuncSetAttribute(factor_diag_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                            cudaSharedmemCarveoutMaxShared));
     auto diag = [&](int K, cudaStream_t s) -> int {
         const long k0 = (long)K * FB;
         const int bs = (int)((k - k0) < FB ? (k - k0) : FB);

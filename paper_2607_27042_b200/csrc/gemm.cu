@@ -103,6 +103,11 @@ static cudaError_t launch_t(const GemmArgs &g, cudaStream_t stream) {
     if (!configured) {
         e = cudaFuncSetAttribute(gemm_kernel<AK, BKc>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
+        // same shared-memory carve-out as the single-CTA kernels of the set-up that run between the GEMMs, so
+        // that the SMs are not reconfigured from launch to launch
+        e = cudaFuncSetAttribute(gemm_kernel<AK, BKc>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared);
+        if (e != cudaSuccess) return e;
         configured = true;
     }
     dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.batch);
