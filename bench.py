@@ -273,6 +273,24 @@ def run_cuda(args):
         "factor_tflops": ((m ** 3 + n ** 3) * (1.0 + 1.0 / 3 + 1.0 / 3)) / (factor_ms * 1e-3) / 1e12,
         "per_step_ms": per_step,
     }
+    if not args.fp32:
+        # the objective of Eq. 7, timed on its own, with plain round-to-nearest of the same X beside it
+        ows = torch.empty(g.gptq2d_objective_workspace_bytes(m, n), dtype=torch.uint8, device="cuda")
+        oval = torch.empty(1, dtype=torch.float64, device="cuda")
+        g.gptq2d_objective(dX, Z, dA, dB, obj=oval, workspace=ows, stream=stream)
+        torch.cuda.synchronize()
+        o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        o0.record(stream)
+        g.gptq2d_objective(dX, Z, dA, dB, obj=oval, workspace=ows, stream=stream)
+        o1.record(stream)
+        torch.cuda.synchronize()
+        out["objective_ms"] = o0.elapsed_time(o1)
+        out["objective"] = float(oval.cpu()[0])
+        Zrtn = torch.round(dX).to(torch.int32)
+        g.gptq2d_objective(dX, Zrtn, dA, dB, obj=oval, workspace=ows, stream=stream)
+        torch.cuda.synchronize()
+        out["objective_round_to_nearest"] = float(oval.cpu()[0])
+        del ows, Zrtn
     if args.fp32:
         # the optional fp32 mode is compared with the fp64 sweep of the same inputs
         ws64 = torch.empty(g.gptq2d_round_workspace_bytes(m, n, g.FP64), dtype=torch.uint8, device="cuda")
