@@ -14,6 +14,7 @@
 //   X21 = -X22 (P21 X11)      (strided-batched GEMMs, one batch entry per block pair)
 // and a final column scaling (transposed on the way out for U).
 #include "common.cuh"
+#include "dmma_gemm.cuh"
 #include "gemm.cuh"
 #include "factor.cuh"
 
@@ -26,7 +27,8 @@ constexpr int FB = 128;
 // The block is padded to 128 x 128 with the identity in shared memory.  Cholesky runs from the last
 // index to the first (one column scaling + one rank-one update of the leading part per step, 16 x 16
 // thread tiling); the inverse is built from 32 x 32 diagonal blocks by doubling,
-// W21 = -W22 (P21 W11), with the temporary product kept in the unused upper triangle of the P array.
+// W21 = -W22 (P21 W11), both products as m8n8k4 DMMA fragments, with the temporary product kept in
+// the unused upper triangle of the P array.
 __device__ __forceinline__ int tri(int i, int j) { return i * (i + 1) / 2 + j; }   // packed lower triangle
 
 __global__ void __launch_bounds__(256) factor_diag_kernel(double *S, long lds, int bs, double *W, long ldw,
@@ -50,35 +52,44 @@ __global__ void __launch_bounds__(256) factor_diag_kernel(double *S, long lds, i
         }
     }
     __syncthreads();
+    // Two barriers per step: the scaled row k goes to `prow` (the packed W array is free until the inverse),
+    // so the update below never reads what the scaling writes in place.
+    double *prow = w;
     for (int k = bs - 1; k >= 0; --k) {
         double d = a[k * 129 + k];
-        __syncthreads();
         if (!(d > 0.0) || !isfinite(d)) {
             if (tid == 0) report(info, GPTQ2D_ERR_NOT_SPD, k0 + k, side, 0);
             d = 1.0;
         }
-        const double pk = sqrt(d), rk = 1.0 / pk;
-        if (tid == 0) a[k * 129 + k] = pk;
-        for (int i = tid; i < k; i += blockDim.x) a[k * 129 + i] *= rk;     // P[k][i], i < k
-        __syncthreads();
-        // Schur complement of the leading k x k part (lower triangle).  The row of P and each thread's
-        // eight entries of a row of the complement are read into registers before anything is stored, so
-        // that the loads are in flight together (loads and stores of the same array cannot be reordered
-        // by the compiler).
+        double rk = rsqrt(d);
+        rk = rk * fma(-0.5 * d, rk * rk, 1.5);                 // one Newton step: 1 / sqrt(d) to the last bit or two
+        if (tid < k) {
+            const double val = a[k * 129 + tid] * rk;          // P[k][tid]
+            a[k * 129 + tid] = val;
+            prow[tid] = val;
+        }
+        __syncthreads();                                       // everyone has read d; prow is complete
+        if (tid == 0) a[k * 129 + k] = d * rk;
+        // Schur complement of the leading k x k part (lower triangle).  Each thread's entries of four rows
+        // are read into registers before anything is stored, so that the loads are in flight together
+        // (loads and stores of the same array cannot be reordered by the compiler).  Every index is < 128,
+        // so the loads are unconditional; only the stores are masked.
         {
-            // every index below is < 128, so all loads are unconditional; only the stores are masked
             double pj[8];
 #pragma unroll
-            for (int jj = 0; jj < 8; ++jj) pj[jj] = a[k * 129 + tx + 16 * jj];
+            for (int jj = 0; jj < 8; ++jj) pj[jj] = prow[tx + 16 * jj];
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
+                if (64 * half >= k) break;                     // rows 64 .. 127 are done once k <= 64
                 double pi[4], v[4][8];
 #pragma unroll
                 for (int ii = 0; ii < 4; ++ii) {
-                    const int i = ty + 16 * (4 * half + ii);
-                    pi[ii] = a[k * 129 + i];
+                    const int R = 4 * half + ii, i = ty + 16 * R;
+                    pi[ii] = prow[i];
+                    // only the 16 x 16 tiles that meet the lower triangle of the leading k x k part
+                    // (the same for the whole warp): the loop is bound by shared-memory bandwidth
 #pragma unroll
-                    for (int jj = 0; jj < 8; ++jj) v[ii][jj] = a[i * 129 + tx + 16 * jj];
+                    for (int jj = 0; jj < 8; ++jj) v[ii][jj] = (jj <= R && 16 * R < k) ? a[i * 129 + tx + 16 * jj] : 0.0;
                 }
 #pragma unroll
                 for (int ii = 0; ii < 4; ++ii) {
@@ -109,25 +120,44 @@ __global__ void __launch_bounds__(256) factor_diag_kernel(double *S, long lds, i
         }
     }
     __syncthreads();
-    // ---- doubling: blocks of b = 32, then 64
-    for (int b = 32; b < 128; b *= 2) {
-        const int npair = 128 / (2 * b), per = b * b;
-        // T = P21 W11, stored above the diagonal at rows s.., columns s + b ..
-        for (int idx = tid; idx < npair * per; idx += blockDim.x) {
-            const int pr = idx / per, rem = idx - pr * per, r = rem / b, c = rem - r * b, s0 = pr * 2 * b;
-            double acc = 0.0;
-            for (int k = c; k < b; ++k) acc = fma(a[(s0 + b + r) * 129 + s0 + k], w[tri(s0 + k, s0 + c)], acc);
-            a[(s0 + r) * 129 + s0 + b + c] = acc;
+    // ---- doubling: blocks of b = 32, then 64, on the fp64 tensor path.  The 128 / (2 b) pairs have b / 8
+    // rows of 8 x 8 fragments each, eight rows in all: one per warp, which takes every fragment of its row.
+    // The triangular operands come from the packed array, zeros where the packed array has no entry.
+    {
+        const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+        for (int b = 32; b < 128; b *= 2) {
+            const int nf = b >> 3, pr = warp / nf, fr = warp - pr * nf, s0 = pr * 2 * b;
+            // T = P21 W11, stored above the diagonal at rows s0 .., columns s0 + b ..
+            for (int fc = 0; fc < nf; ++fc) {
+                double c0 = 0.0, c1 = 0.0;
+                const int cc = 8 * fc + g;
+                for (int kk = 8 * fc; kk < b; kk += 4) {       // W11[k][c] = 0 for k < c
+                    const int k = kk + t;
+                    const double af = a[(s0 + b + 8 * fr + g) * 129 + s0 + k];
+                    const double bf = k >= cc ? w[tri(s0 + k, s0 + min(cc, k))] : 0.0;     // index clamped: stays inside the array
+                    dmma_m8n8k4(c0, c1, af, bf);
+                }
+                double *dst = a + (s0 + 8 * fr + g) * 129 + s0 + b + 8 * fc + 2 * t;
+                dst[0] = c0;
+                dst[1] = c1;
+            }
+            __syncthreads();
+            // W21 = -W22 T
+            for (int fc = 0; fc < nf; ++fc) {
+                double c0 = 0.0, c1 = 0.0;
+                const int rr = 8 * fr + g;
+                for (int kk = 0; kk < 8 * fr + 8; kk += 4) {   // W22[r][k] = 0 for k > r
+                    const int k = kk + t;
+                    const double af = k <= rr ? w[tri(s0 + b + rr, s0 + b + min(k, rr))] : 0.0;
+                    const double bf = a[(s0 + k) * 129 + s0 + b + 8 * fc + g];
+                    dmma_m8n8k4(c0, c1, af, bf);
+                }
+                double *dst = w + tri(s0 + b + rr, s0 + 8 * fc + 2 * t);
+                dst[0] = -c0;
+                dst[1] = -c1;
+            }
+            __syncthreads();
         }
-        __syncthreads();
-        // W21 = -W22 T
-        for (int idx = tid; idx < npair * per; idx += blockDim.x) {
-            const int pr = idx / per, rem = idx - pr * per, r = rem / b, c = rem - r * b, s0 = pr * 2 * b;
-            double acc = 0.0;
-            for (int k = 0; k <= r; ++k) acc = fma(w[tri(s0 + b + r, s0 + b + k)], a[(s0 + k) * 129 + s0 + b + c], acc);
-            w[tri(s0 + b + r, s0 + c)] = -acc;
-        }
-        __syncthreads();
     }
     for (int idx = tid; idx < bs * bs; idx += blockDim.x) {
         int i = idx / bs, j = idx - i * bs;
