@@ -463,6 +463,34 @@ def run_batched(args):
                      "kernel_ms": ms_per_step, "flops_per_launch": flops},
         "per_step_ms": per_step,
     }
+    # the set-up of the same K layers: one gptq2d_factor_batched call against K gptq2d_factor calls
+    # (every layer gets its own bases here, perturbed copies of the configuration's)
+    Kf = min(K, 64) if max(m, n) > 128 else K
+    frng = np.random.default_rng(args.seed + 13)
+    fAs = [torch.from_numpy(np.ascontiguousarray(A * (1.0 + 0.01 * frng.standard_normal(A.shape)))).cuda() for _ in range(Kf)]
+    fBs = [torch.from_numpy(np.ascontiguousarray(B * (1.0 + 0.01 * frng.standard_normal(B.shape)))).cuda() for _ in range(Kf)]
+    fLs = [torch.empty((m, m), dtype=torch.float64, device="cuda") for _ in range(Kf)]
+    fUs = [torch.empty((n, n), dtype=torch.float64, device="cuda") for _ in range(Kf)]
+    fws1 = torch.empty(g.gptq2d_factor_workspace_bytes(m, n), dtype=torch.uint8, device="cuda")
+
+    fprobs = g.make_factor_problems(fAs, fBs, fLs, fUs)
+    fwsb = torch.empty(max(256, g.gptq2d_factor_batched_workspace_bytes(fprobs)), dtype=torch.uint8, device="cuda")
+
+    def factor_batched():
+        g.gptq2d_factor_batched(problems=fprobs, workspace=fwsb, info=info, stream=stream)
+
+    def factor_one_by_one():
+        for b in range(Kf):
+            g.gptq2d_factor(fAs[b], fBs[b], L=fLs[b], U=fUs[b], workspace=fws1, info=info, stream=stream)
+
+    factor_batched()
+    factor_one_by_one()
+    torch.cuda.synchronize()
+    fb = float(np.mean(timed(factor_batched, 3)))
+    f1 = float(np.mean(timed(factor_one_by_one, 3)))
+    g.check_info(info)
+    out["factor"] = {"layers": Kf, "batched_ms": fb, "one_by_one_ms": f1, "speedup": f1 / fb,
+                     "note": "problems whose bases both have order <= 128 are factorised one CTA per side in one launch; the others take the blocked route of gptq2d_factor one after the other"}
     print(json.dumps(out))
     if dist:
         dist.destroy_process_group()

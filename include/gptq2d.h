@@ -165,6 +165,31 @@ int gptq2d_round_batched(int count, const gptq2d_problem_t *problems,
                          double *min_margin,
                          void *workspace, size_t workspace_bytes, int *info, void *stream);
 
+/* ---- the set-up of many matrices in one call (the factors that gptq2d_round_batched consumes) ----
+ * For every problem the same L, U, dL, dU as gptq2d_factor (Section 3.1; Algorithm 3 lines 1-2).  The
+ * problems whose bases both have order <= GPTQ2D_FACTOR_SMALL_MAX are factorised one CTA per side, all
+ * in ONE launch, entirely in shared memory (Gram, Cholesky from the last index to the first, triangular
+ * inverse, scaling); a problem with a larger basis takes the blocked route of gptq2d_factor, one problem
+ * after the other.
+ *   problems: HOST array of `count` descriptors (device pointers inside, rules as gptq2d_factor: A or B
+ *             may be NULL for the identity, dL / dU optional); read before the call returns.
+ *   info:     device int[4] shared by all problems; for GPTQ2D_ERR_NOT_SPD from a small side info[3] is
+ *             the index of the problem (first error wins; the other problems are still factorised).
+ *   workspace: device, 256-byte aligned, gptq2d_factor_batched_workspace_bytes(count, problems) bytes.
+ */
+#define GPTQ2D_FACTOR_SMALL_MAX 128
+typedef struct gptq2d_factor_problem {
+    int m, n;
+    const double *A; long lda;   /* m x m or NULL */
+    const double *B; long ldb;   /* n x n or NULL */
+    double *L; long ldl;
+    double *U; long ldu;
+    double *dL, *dU;             /* optional (NULL ok) */
+} gptq2d_factor_problem_t;
+size_t gptq2d_factor_batched_workspace_bytes(int count, const gptq2d_factor_problem_t *problems);
+int gptq2d_factor_batched(int count, const gptq2d_factor_problem_t *problems,
+                          void *workspace, size_t workspace_bytes, int *info, void *stream);
+
 /* ---- the sweep without any allocation (the paper has no counterpart: this is a packaging variant
  * of gptq2d_round, not a different method) ----
  * For callers that must not allocate device memory -- a step that will be replayed from a CUDA

@@ -3,6 +3,7 @@
 #include "common.cuh"
 #include "round_internal.cuh"
 #include "factor.cuh"
+#include <algorithm>
 #include <mutex>
 #include <vector>
 
@@ -125,6 +126,32 @@ size_t gptq2d_factor_workspace_bytes(int m, int n) {
     return factor_workspace_bytes(m, n);
 }
 
+// Both sides of one problem, arguments already checked, `info` already cleared.
+static int factor_pair(int m, int n, const double *A, long lda, const double *B, long ldb, double *L, long ldl, double *U,
+                       long ldu, double *dL, double *dU, void *workspace, int *info, cudaStream_t stream) {
+    // The two sides are independent.  Each has a serial spine (one small diagonal-block kernel per 128
+    // rows, between the panel and trailing updates) that leaves most SMs idle, so the B side runs on a
+    // second stream and its GEMMs fill the gaps of the A side and vice versa.
+    char *wsB = static_cast<char *>(workspace) + factor_side_workspace_bytes(m);
+    HostPipe *hp = (A && B) ? host_pipe() : nullptr;
+    if (!hp) {
+        int st = factor_one_side(m, A, lda, 0, L, ldl, dL, workspace, info, stream, nullptr);
+        if (st != GPTQ2D_OK) return st;
+        return factor_one_side(n, B, ldb, 1, U, ldu, dU, wsB, info, stream, nullptr);
+    }
+    std::unique_lock<std::mutex> lock(hp->enqueue);
+    if (cudaEventRecord(hp->inputs_free, stream) != cudaSuccess ||
+        cudaStreamWaitEvent(hp->copy, hp->inputs_free, 0) != cudaSuccess)
+        return GPTQ2D_ERR_CUDA;
+    int st = factor_one_side(m, A, lda, 0, L, ldl, dL, workspace, info, stream, hp->look[0].spine ? &hp->look[0] : nullptr);
+    int st2 = factor_one_side(n, B, ldb, 1, U, ldu, dU, wsB, info, hp->copy, hp->look[1].spine ? &hp->look[1] : nullptr);
+    // join even if an enqueue failed, so that nothing of this call is left running behind the caller's stream
+    if (cudaEventRecord(hp->copies_done, hp->copy) != cudaSuccess ||
+        cudaStreamWaitEvent(stream, hp->copies_done, 0) != cudaSuccess)
+        return GPTQ2D_ERR_CUDA;
+    return st != GPTQ2D_OK ? st : st2;
+}
+
 int gptq2d_factor(int m, int n, const double *A, long lda, const double *B, long ldb, double *L, long ldl, double *U,
                   long ldu, double *dL, double *dU, void *workspace, size_t workspace_bytes, int *info,
                   void *stream_) {
@@ -137,27 +164,68 @@ int gptq2d_factor(int m, int n, const double *A, long lda, const double *B, long
     int st = check_device();
     if (st != GPTQ2D_OK) return st;
     if (info && cudaMemsetAsync(info, 0, 4 * sizeof(int), stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;
-    // The two sides are independent.  Each has a serial spine (one small diagonal-block kernel per 128
-    // rows, between the panel and trailing updates) that leaves most SMs idle, so the B side runs on a
-    // second stream and its GEMMs fill the gaps of the A side and vice versa.
-    char *wsB = static_cast<char *>(workspace) + factor_side_workspace_bytes(m);
-    HostPipe *hp = (A && B) ? host_pipe() : nullptr;
-    if (!hp) {
-        st = factor_one_side(m, A, lda, 0, L, ldl, dL, workspace, info, stream, nullptr);
-        if (st != GPTQ2D_OK) return st;
-        return factor_one_side(n, B, ldb, 1, U, ldu, dU, wsB, info, stream, nullptr);
+    return factor_pair(m, n, A, lda, B, ldb, L, ldl, U, ldu, dL, dU, workspace, info, stream);
+}
+
+static size_t factor_batched_table_bytes(int count) { return pad256((size_t)2 * count * sizeof(FactorSmallSide)); }
+// a problem with a basis of order > FACTOR_SMALL_MAX takes the blocked route of gptq2d_factor, both sides
+static bool factor_problem_is_large(const gptq2d_factor_problem_t &q) {
+    return (q.A && q.m > FACTOR_SMALL_MAX) || (q.B && q.n > FACTOR_SMALL_MAX);
+}
+
+size_t gptq2d_factor_batched_workspace_bytes(int count, const gptq2d_factor_problem_t *pr) {
+    if (count < 1 || !pr) return 0;
+    size_t large = 0;
+    for (int b = 0; b < count; ++b) {
+        if (pr[b].m < 1 || pr[b].n < 1) return 0;
+        if (factor_problem_is_large(pr[b])) large = std::max(large, factor_workspace_bytes(pr[b].m, pr[b].n));
     }
-    std::unique_lock<std::mutex> lock(hp->enqueue);
-    if (cudaEventRecord(hp->inputs_free, stream) != cudaSuccess ||
-        cudaStreamWaitEvent(hp->copy, hp->inputs_free, 0) != cudaSuccess)
-        return GPTQ2D_ERR_CUDA;
-    st = factor_one_side(m, A, lda, 0, L, ldl, dL, workspace, info, stream, hp->look[0].spine ? &hp->look[0] : nullptr);
-    int st2 = factor_one_side(n, B, ldb, 1, U, ldu, dU, wsB, info, hp->copy, hp->look[1].spine ? &hp->look[1] : nullptr);
-    // join even if an enqueue failed, so that nothing of this call is left running behind the caller's stream
-    if (cudaEventRecord(hp->copies_done, hp->copy) != cudaSuccess ||
-        cudaStreamWaitEvent(stream, hp->copies_done, 0) != cudaSuccess)
-        return GPTQ2D_ERR_CUDA;
-    return st != GPTQ2D_OK ? st : st2;
+    return factor_batched_table_bytes(count) + large;
+}
+
+int gptq2d_factor_batched(int count, const gptq2d_factor_problem_t *pr, void *workspace, size_t workspace_bytes,
+                          int *info, void *stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (count < 1 || !pr) return GPTQ2D_ERR_INVALID_ARG;
+    for (int b = 0; b < count; ++b) {
+        const gptq2d_factor_problem_t &q = pr[b];
+        if (q.m < 1 || q.n < 1 || !q.L || !q.U || q.ldl < q.m || q.ldu < q.n) return GPTQ2D_ERR_INVALID_ARG;
+        if ((q.A && q.lda < q.m) || (q.B && q.ldb < q.n)) return GPTQ2D_ERR_INVALID_ARG;
+        if (!aligned(q.A, 8) || !aligned(q.B, 8) || !aligned(q.L, 8) || !aligned(q.U, 8) || !aligned(q.dL, 8) ||
+            !aligned(q.dU, 8))
+            return GPTQ2D_ERR_INVALID_ARG;
+    }
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gptq2d_factor_batched_workspace_bytes(count, pr))
+        return GPTQ2D_ERR_WORKSPACE;
+    int st = check_device();
+    if (st != GPTQ2D_OK) return st;
+    if (info && cudaMemsetAsync(info, 0, 4 * sizeof(int), stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+    // problems whose bases both have order <= FACTOR_SMALL_MAX (or are absent): one CTA per side, one launch
+    std::vector<FactorSmallSide> small;
+    small.reserve((size_t)2 * count);
+    for (int b = 0; b < count; ++b) {
+        const gptq2d_factor_problem_t &q = pr[b];
+        if (factor_problem_is_large(q)) continue;
+        small.push_back(FactorSmallSide{q.m, 0, b, q.A, q.lda, q.L, q.ldl, q.dL});
+        small.push_back(FactorSmallSide{q.n, 1, b, q.B, q.ldb, q.U, q.ldu, q.dU});
+    }
+    char *w = static_cast<char *>(workspace);
+    if (!small.empty()) {
+        // pageable source: the copy is staged before the call returns, so the vector may go out of scope
+        if (cudaMemcpyAsync(w, small.data(), small.size() * sizeof(FactorSmallSide), cudaMemcpyHostToDevice, stream) !=
+            cudaSuccess)
+            return GPTQ2D_ERR_CUDA;
+        st = launch_factor_small((int)small.size(), reinterpret_cast<const FactorSmallSide *>(w), info, stream);
+        if (st != GPTQ2D_OK) return st;
+    }
+    char *wl = w + factor_batched_table_bytes(count);
+    for (int b = 0; b < count; ++b) {
+        const gptq2d_factor_problem_t &q = pr[b];
+        if (!factor_problem_is_large(q)) continue;
+        st = factor_pair(q.m, q.n, q.A, q.lda, q.B, q.ldb, q.L, q.ldl, q.U, q.ldu, q.dL, q.dU, wl, info, stream);
+        if (st != GPTQ2D_OK) return st;
+    }
+    return GPTQ2D_OK;
 }
 
 size_t gptq2d_round_workspace_bytes(int m, int n, int precision) {

@@ -31,34 +31,19 @@ constexpr int FB = 128;
 // the unused upper triangle of the P array.
 __device__ __forceinline__ int tri(int i, int j) { return i * (i + 1) / 2 + j; }   // packed lower triangle
 
-__global__ void __launch_bounds__(256) factor_diag_kernel(double *S, long lds, int bs, double *W, long ldw,
-                                                          double *pdiag, int *info, int side, int k0) {
-    extern __shared__ double sm[];
-    double *a = sm;               // [128][129]: P in the lower triangle, scratch above it
-    double *w = sm + 128 * 129;   // packed lower triangle of W
+// In place, in shared memory, by one CTA of 256 threads: a [128][129] holds the lower triangle of a Schur
+// complement padded to 128 x 128 with the identity (bs rows are real); on return its lower triangle is P
+// (S = P^T P, Cholesky from the last index to the first) and w is the packed lower triangle of W = P^{-1}.
+// Ends with a barrier.  err_c: what a non-positive pivot reports in info[3], beside its index and the side.
+__device__ __forceinline__ void chol_inverse_128(double *a, double *w, int bs, int *info, int side, int k0, int err_c) {
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-    // the block, padded with the identity: eight loads in flight per thread
-    for (int base = 0; base < 128 * 128; base += 8 * 256) {
-        double v[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int idx = base + u * 256 + tid, i = idx >> 7, j = idx & 127;
-            v[u] = (j <= i && i < bs) ? S[(long)i * lds + j] : (i == j ? 1.0 : 0.0);
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int idx = base + u * 256 + tid, i = idx >> 7, j = idx & 127;
-            if (j <= i) a[i * 129 + j] = v[u];
-        }
-    }
-    __syncthreads();
     // Two barriers per step: the scaled row k goes to `prow` (the packed W array is free until the inverse),
     // so the update below never reads what the scaling writes in place.
     double *prow = w;
     for (int k = bs - 1; k >= 0; --k) {
         double d = a[k * 129 + k];
         if (!(d > 0.0) || !isfinite(d)) {
-            if (tid == 0) report(info, GPTQ2D_ERR_NOT_SPD, k0 + k, side, 0);
+            if (tid == 0) report(info, GPTQ2D_ERR_NOT_SPD, k0 + k, side, err_c);
             d = 1.0;
         }
         double rk = rsqrt(d);
@@ -159,6 +144,30 @@ __global__ void __launch_bounds__(256) factor_diag_kernel(double *S, long lds, i
             __syncthreads();
         }
     }
+}
+
+__global__ void __launch_bounds__(256) factor_diag_kernel(double *S, long lds, int bs, double *W, long ldw,
+                                                          double *pdiag, int *info, int side, int k0) {
+    extern __shared__ double sm[];
+    double *a = sm;               // [128][129]: P in the lower triangle, scratch above it
+    double *w = sm + 128 * 129;   // packed lower triangle of W
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    // the block, padded with the identity: eight loads in flight per thread
+    for (int base = 0; base < 128 * 128; base += 8 * 256) {
+        double v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int idx = base + u * 256 + tid, i = idx >> 7, j = idx & 127;
+            v[u] = (j <= i && i < bs) ? S[(long)i * lds + j] : (i == j ? 1.0 : 0.0);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int idx = base + u * 256 + tid, i = idx >> 7, j = idx & 127;
+            if (j <= i) a[i * 129 + j] = v[u];
+        }
+    }
+    __syncthreads();
+    chol_inverse_128(a, w, bs, info, side, k0, 0);
     for (int idx = tid; idx < bs * bs; idx += blockDim.x) {
         int i = idx / bs, j = idx - i * bs;
         if (j <= i) S[(long)i * lds + j] = a[i * 129 + j];
@@ -205,6 +214,89 @@ __global__ void identity_kernel(double *out, long ldo, int k, double *dinv) {
         out[(long)i * ldo + j] = (i == j) ? 1.0 : 0.0;
     }
     if (dinv && idx < k) dinv[idx] = 1.0;
+}
+
+// One side of one small problem (order k <= 128) per CTA, everything in shared memory: the Gram of the
+// basis, its Cholesky factorisation and inverse (chol_inverse_128), the unit triangular factor and 1/Lambda.
+// For the set-up of many small matrices at once, where one launch sequence per matrix would cost far more
+// than the arithmetic.
+__global__ void __launch_bounds__(256) factor_small_kernel(const FactorSmallSide *sides, int *info) {
+    extern __shared__ double sm[];
+    double *a = sm;               // [128][129]
+    double *w = sm + 128 * 129;   // packed lower triangle of W
+    const FactorSmallSide q = sides[blockIdx.x];
+    const int k = q.k, tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    if (!q.M) {                                           // identity basis
+        for (int idx = tid; idx < k * k; idx += blockDim.x) {
+            const int i = idx / k, j = idx - i * k;
+            q.out[(long)i * q.ldo + j] = i == j ? 1.0 : 0.0;
+        }
+        if (q.dinv)
+            for (int j = tid; j < k; j += blockDim.x) q.dinv[j] = 1.0;
+        return;
+    }
+    // a[r][i] = M[r][i] (side 0, S = M^T M) or M[i][r] (side 1, S = M M^T), zero outside k x k
+    for (int base = 0; base < 128 * 128; base += 8 * 256) {
+        double v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int idx = base + u * 256 + tid, r = idx >> 7, i = idx & 127;
+            v[u] = (r < k && i < k) ? (q.side == 0 ? q.M[(long)r * q.ldm + i] : q.M[(long)i * q.ldm + r]) : 0.0;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int idx = base + u * 256 + tid;
+            a[(idx >> 7) * 129 + (idx & 127)] = v[u];
+        }
+    }
+    __syncthreads();
+    // S[i][j] = sum_r a[r][i] a[r][j]; thread (tx, ty) owns i = ty + 16 ii, j = tx + 16 jj
+    double acc[8][8];
+#pragma unroll
+    for (int ii = 0; ii < 8; ++ii)
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) acc[ii][jj] = 0.0;
+    for (int r = 0; r < k; ++r) {
+        double ai[8], aj[8];
+#pragma unroll
+        for (int x = 0; x < 8; ++x) {
+            ai[x] = a[r * 129 + ty + 16 * x];
+            aj[x] = a[r * 129 + tx + 16 * x];
+        }
+#pragma unroll
+        for (int ii = 0; ii < 8; ++ii)
+#pragma unroll
+            for (int jj = 0; jj < 8; ++jj) acc[ii][jj] = fma(ai[ii], aj[jj], acc[ii][jj]);
+    }
+    __syncthreads();
+    // the Gram, padded with the identity, replaces the basis
+#pragma unroll
+    for (int ii = 0; ii < 8; ++ii)
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+            const int i = ty + 16 * ii, j = tx + 16 * jj;
+            if (j <= i) a[i * 129 + j] = i < k ? acc[ii][jj] : (i == j ? 1.0 : 0.0);
+        }
+    __syncthreads();
+    chol_inverse_128(a, w, k, info, q.side, 0, q.index);
+    // F = W diag(P): unit lower (side 0) or, transposed on the way out, unit upper (side 1)
+    for (int idx = tid; idx < k * k; idx += blockDim.x) {
+        const int i = idx / k, j = idx - i * k;
+        const double v = i > j ? w[tri(i, j)] * a[j * 129 + j] : (i == j ? 1.0 : 0.0);
+        if (q.side == 0) q.out[(long)i * q.ldo + j] = v;
+        else q.out[(long)j * q.ldo + i] = v;
+    }
+    if (q.dinv)
+        for (int j = tid; j < k; j += blockDim.x) q.dinv[j] = a[j * 129 + j] * a[j * 129 + j];
+}
+
+int launch_factor_small(int nsides, const FactorSmallSide *dev_sides, int *info, cudaStream_t stream) {
+    if (nsides <= 0) return GPTQ2D_OK;
+    const size_t smem = (128 * 129 + 128 * 129 / 2) * sizeof(double);
+    if (cudaFuncSetAttribute(factor_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return GPTQ2D_ERR_CUDA;
+    factor_small_kernel<<<nsides, 256, smem, stream>>>(dev_sides, info);
+    return cudaGetLastError() == cudaSuccess ? GPTQ2D_OK : GPTQ2D_ERR_CUDA;
 }
 
 static inline long round_up(long x, long a) { return (x + a - 1) / a * a; }

@@ -35,7 +35,9 @@ EXPORTS = (
     "gptq2d_round_reverse_workspace_bytes", "gptq2d_round_reverse",
     "gptq2d_round_f32in_workspace_bytes", "gptq2d_round_f32in",
     "gptq2d_round_blocked_workspace_bytes", "gptq2d_round_blocked",
+    "gptq2d_factor_batched_workspace_bytes", "gptq2d_factor_batched",
 )
+FACTOR_SMALL_MAX = 128
 
 BLOCKED_MAX_WIDTH = 64
 
@@ -50,6 +52,16 @@ class Problem(ctypes.Structure):
                 ("U", ctypes.c_void_p), ("ldu", ctypes.c_long),
                 ("Z", ctypes.c_void_p), ("ldz", ctypes.c_long),
                 ("E", ctypes.c_void_p), ("lde", ctypes.c_long)]
+
+
+class FactorProblem(ctypes.Structure):
+    """gptq2d_factor_problem_t: one (A, B) pair of a batched set-up (device pointers; A or B may be NULL)."""
+    _fields_ = [("m", ctypes.c_int), ("n", ctypes.c_int),
+                ("A", ctypes.c_void_p), ("lda", ctypes.c_long),
+                ("B", ctypes.c_void_p), ("ldb", ctypes.c_long),
+                ("L", ctypes.c_void_p), ("ldl", ctypes.c_long),
+                ("U", ctypes.c_void_p), ("ldu", ctypes.c_long),
+                ("dL", ctypes.c_void_p), ("dU", ctypes.c_void_p)]
 
 
 class Gptq2dError(RuntimeError):
@@ -90,6 +102,10 @@ def _load():
     lib.gptq2d_round_static_max_dim.argtypes = []
     lib.gptq2d_round_f32in.restype = i32
     lib.gptq2d_round_f32in.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, sz, vp, vp]
+    lib.gptq2d_factor_batched_workspace_bytes.restype = sz
+    lib.gptq2d_factor_batched_workspace_bytes.argtypes = [i32, vp]
+    lib.gptq2d_factor_batched.restype = i32
+    lib.gptq2d_factor_batched.argtypes = [i32, vp, vp, sz, vp, vp]
     lib.gptq2d_round_blocked_workspace_bytes.restype = sz
     lib.gptq2d_round_blocked_workspace_bytes.argtypes = [i32, i32, i32]
     lib.gptq2d_round_blocked.restype = i32
@@ -297,6 +313,65 @@ def gptq2d_round_f32in(X, L, U, Z=None, E=None, min_margin=None, workspace=None,
     if st != OK:
         raise Gptq2dError(st)
     return Z, E, min_margin, info
+
+
+def _factor_problems(As, Bs, Ls, Us, dLs, dUs, shapes):
+    count = len(shapes)
+    arr = (FactorProblem * count)()
+    for b, (m, n) in enumerate(shapes):
+        pA, lda = _mat(As[b], torch.float64, "A")
+        pB, ldb = _mat(Bs[b], torch.float64, "B")
+        pL, ldl = _mat(Ls[b], torch.float64, "L")
+        pU, ldu = _mat(Us[b], torch.float64, "U")
+        arr[b] = FactorProblem(m, n, pA, lda, pB, ldb, pL, ldl, pU, ldu,
+                               _ptr(dLs[b]) if dLs is not None else None, _ptr(dUs[b]) if dUs is not None else None)
+    return arr
+
+
+def make_factor_problems(As, Bs, Ls, Us, dLs=None, dUs=None, shapes=None):
+    """The host descriptor array (gptq2d_factor_problem_t[count]) of a batched set-up; reusable across calls
+    as long as the tensors it points to stay alive and in place."""
+    if shapes is None:
+        shapes = [(Ls[b].shape[0], Us[b].shape[0]) for b in range(len(Ls))]
+    return _factor_problems(As, Bs, Ls, Us, dLs, dUs, shapes)
+
+
+def gptq2d_factor_batched_workspace_bytes(problems):
+    return int(_lib.gptq2d_factor_batched_workspace_bytes(len(problems), ctypes.cast(problems, ctypes.c_void_p)))
+
+
+def gptq2d_factor_batched(As=None, Bs=None, shapes=None, Ls=None, Us=None, dLs=None, dUs=None, workspace=None,
+                          info=None, stream=None, device=None, problems=None):
+    """The set-up of many (A, B) pairs in one call.  As, Bs: sequences of CUDA tensors or None (identity;
+    `shapes` = [(m, n), ...] is then needed for those), or `problems` = an array from make_factor_problems
+    (the outputs are then whatever that array points to).  Returns (Ls, Us, dLs, dUs, info)."""
+    dev = device
+    if problems is None:
+        count = len(As)
+        if shapes is None:
+            shapes = [(As[b].shape[0], Bs[b].shape[0]) for b in range(count)]
+        if dev is None:
+            dev = next((t.device for t in list(As) + list(Bs) if t is not None),
+                       torch.device("cuda", torch.cuda.current_device()))
+        if Ls is None:
+            Ls = [torch.empty((m, m), dtype=torch.float64, device=dev) for (m, n) in shapes]
+        if Us is None:
+            Us = [torch.empty((n, n), dtype=torch.float64, device=dev) for (m, n) in shapes]
+        if dLs is None:
+            dLs = [torch.empty(m, dtype=torch.float64, device=dev) for (m, n) in shapes]
+        if dUs is None:
+            dUs = [torch.empty(n, dtype=torch.float64, device=dev) for (m, n) in shapes]
+        problems = _factor_problems(As, Bs, Ls, Us, dLs, dUs, shapes)
+    elif dev is None:
+        dev = torch.device("cuda", torch.cuda.current_device())
+    info = torch.zeros(4, dtype=torch.int32, device=dev) if info is None else info
+    if workspace is None:
+        workspace = _workspace(gptq2d_factor_batched_workspace_bytes(problems), dev)
+    st = _lib.gptq2d_factor_batched(len(problems), ctypes.cast(problems, ctypes.c_void_p), _ptr(workspace),
+                                    workspace.numel(), _ptr(info), _stream_ptr(stream))
+    if st != OK:
+        raise Gptq2dError(st)
+    return Ls, Us, dLs, dUs, info
 
 
 def gptq2d_round_blocked_workspace_bytes(m, n, w):

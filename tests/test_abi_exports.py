@@ -87,3 +87,29 @@ def test_batched_entry_argument_checks_need_no_gpu():
     # workspace too small / missing
     assert lib.gptq2d_round_batched(3, c.cast(arr, c.c_void_p), None, ws, total - 1, None, None) == 2
     assert lib.gptq2d_round_batched(3, c.cast(arr, c.c_void_p), None, None, total, None, None) == 2
+
+
+def test_batched_setup_argument_checks_need_no_gpu():
+    """Host-side validation of gptq2d_factor_batched: made-up (never dereferenced) device addresses."""
+    import ctypes as c
+    from paper_2607_27042_b200 import gptq2d as g
+    lib = g._lib
+
+    def probs(shapes, a=0x1000):
+        arr = (g.FactorProblem * len(shapes))()
+        for b, (m, n) in enumerate(shapes):
+            arr[b] = g.FactorProblem(m, n, a, m, 0x2000, n, 0x3000, m, 0x4000, n, None, None)
+        return arr
+
+    small = probs([(64, 64), (1, 128), (100, 7)])
+    table = lib.gptq2d_factor_batched_workspace_bytes(3, c.cast(small, c.c_void_p))
+    assert 0 < table <= 4096                                    # descriptors only: no blocked route needed
+    mixed = probs([(64, 64), (300, 90)])
+    total = lib.gptq2d_factor_batched_workspace_bytes(2, c.cast(mixed, c.c_void_p))
+    assert total >= g.gptq2d_factor_workspace_bytes(300, 90)    # the blocked route's own workspace on top
+    assert lib.gptq2d_factor_batched_workspace_bytes(0, c.cast(small, c.c_void_p)) == 0
+    assert lib.gptq2d_factor_batched(0, c.cast(small, c.c_void_p), None, 0, None, None) == 1      # INVALID_ARG
+    bad = probs([(64, 64)])
+    bad[0].ldl = 10                                             # leading dimension below m
+    assert lib.gptq2d_factor_batched(1, c.cast(bad, c.c_void_p), None, 0, None, None) == 1
+    assert lib.gptq2d_factor_batched(3, c.cast(small, c.c_void_p), None, 0, None, None) == 2      # WORKSPACE
