@@ -169,8 +169,9 @@ int gptq2d_round_batched(int count, const gptq2d_problem_t *problems,
  * For every problem the same L, U, dL, dU as gptq2d_factor (Section 3.1; Algorithm 3 lines 1-2).  The
  * problems whose bases both have order <= GPTQ2D_FACTOR_SMALL_MAX are factorised one CTA per side, all
  * in ONE launch, entirely in shared memory (Gram, Cholesky from the last index to the first, triangular
- * inverse, scaling); a problem with a larger basis takes the blocked route of gptq2d_factor, one problem
- * after the other.
+ * inverse, scaling); problems with a larger basis take the blocked route of gptq2d_factor, several of
+ * them side by side on streams of the library's own (everything is ordered after the work already on
+ * `stream`, and `stream` waits for all of it).
  *   problems: HOST array of `count` descriptors (device pointers inside, rules as gptq2d_factor: A or B
  *             may be NULL for the identity, dL / dU optional); read before the call returns.
  *   info:     device int[4] shared by all problems; for GPTQ2D_ERR_NOT_SPD from a small side info[3] is

@@ -37,6 +37,10 @@ struct HostPipe {
     cudaStream_t copy = nullptr;
     cudaEvent_t inputs_free = nullptr, copies_done = nullptr;
     FactorLookahead look[2] = {};            // per side of the set-up: spine stream and its events (spine == NULL: none)
+    static constexpr int POOL = 8;           // streams that carry independent problems of a batched set-up
+    cudaStream_t pool[POOL] = {};
+    cudaEvent_t pool_done[POOL] = {};
+    bool pool_ok = false;
     StreamWriteValue32Fn write32 = nullptr;
     StreamWaitValue32Fn wait32 = nullptr;    // stream-ordered wait until a device word is >= a value
     bool tried = false;
@@ -73,6 +77,10 @@ static HostPipe *host_pipe() {
             for (int e = 0; lok && e < 5; ++e) lok = cudaEventCreateWithFlags(ev[e], cudaEventDisableTiming) == cudaSuccess;
             if (!lok) lk.spine = nullptr;        // the set-up then runs that side on one stream
         }
+        hp.pool_ok = ok;
+        for (int k = 0; hp.pool_ok && k < HostPipe::POOL; ++k)
+            hp.pool_ok = cudaStreamCreateWithFlags(&hp.pool[k], cudaStreamNonBlocking) == cudaSuccess &&
+                         cudaEventCreateWithFlags(&hp.pool_done[k], cudaEventDisableTiming) == cudaSuccess;
         if (ok) { hp.write32 = reinterpret_cast<StreamWriteValue32Fn>(fn); hp.wait32 = reinterpret_cast<StreamWaitValue32Fn>(fnw); }
         (void)cudaGetLastError();
     }
@@ -176,10 +184,16 @@ static bool factor_problem_is_large(const gptq2d_factor_problem_t &q) {
 size_t gptq2d_factor_batched_workspace_bytes(int count, const gptq2d_factor_problem_t *pr) {
     if (count < 1 || !pr) return 0;
     size_t large = 0;
+    int nlarge = 0;
     for (int b = 0; b < count; ++b) {
         if (pr[b].m < 1 || pr[b].n < 1) return 0;
-        if (factor_problem_is_large(pr[b])) large = std::max(large, factor_workspace_bytes(pr[b].m, pr[b].n));
+        if (factor_problem_is_large(pr[b])) {
+            large = std::max(large, factor_workspace_bytes(pr[b].m, pr[b].n));
+            ++nlarge;
+        }
     }
+    // several problems of the blocked route run side by side, each in a slot of its own
+    large *= (size_t)std::min(nlarge, (int)HostPipe::POOL);
     return factor_batched_table_bytes(count) + large;
 }
 
@@ -219,12 +233,48 @@ int gptq2d_factor_batched(int count, const gptq2d_factor_problem_t *pr, void *wo
         if (st != GPTQ2D_OK) return st;
     }
     char *wl = w + factor_batched_table_bytes(count);
+    size_t slot_bytes = 0;
+    int nlarge = 0;
+    for (int b = 0; b < count; ++b)
+        if (factor_problem_is_large(pr[b])) {
+            slot_bytes = std::max(slot_bytes, factor_workspace_bytes(pr[b].m, pr[b].n));
+            ++nlarge;
+        }
+    HostPipe *hp = nlarge > 1 ? host_pipe() : nullptr;
+    if (!hp || !hp->pool_ok) {
+        // one problem (or no second stream): the two-stream route of gptq2d_factor, problem after problem
+        for (int b = 0; b < count; ++b) {
+            const gptq2d_factor_problem_t &q = pr[b];
+            if (!factor_problem_is_large(q)) continue;
+            st = factor_pair(q.m, q.n, q.A, q.lda, q.B, q.ldb, q.L, q.ldl, q.U, q.ldu, q.dL, q.dU, wl, info, stream);
+            if (st != GPTQ2D_OK) return st;
+        }
+        return GPTQ2D_OK;
+    }
+    // Several problems: each is a chain of many small launches, so independent problems go to different
+    // streams (round robin; a stream and its workspace slot are shared by every POOL-th problem, in order).
+    std::unique_lock<std::mutex> lock(hp->enqueue);
+    const int nslots = std::min(nlarge, (int)HostPipe::POOL);
+    if (cudaEventRecord(hp->inputs_free, stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+    for (int k = 0; k < nslots; ++k)
+        if (cudaStreamWaitEvent(hp->pool[k], hp->inputs_free, 0) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+    int idx = 0, first_err = GPTQ2D_OK;
     for (int b = 0; b < count; ++b) {
         const gptq2d_factor_problem_t &q = pr[b];
         if (!factor_problem_is_large(q)) continue;
-        st = factor_pair(q.m, q.n, q.A, q.lda, q.B, q.ldb, q.L, q.ldl, q.U, q.ldu, q.dL, q.dU, wl, info, stream);
-        if (st != GPTQ2D_OK) return st;
+        const int k = idx++ % nslots;
+        char *wk = wl + (size_t)k * slot_bytes;
+        int s1 = factor_one_side(q.m, q.A, q.lda, 0, q.L, q.ldl, q.dL, wk, info, hp->pool[k], nullptr);
+        int s2 = factor_one_side(q.n, q.B, q.ldb, 1, q.U, q.ldu, q.dU, wk + factor_side_workspace_bytes(q.m), info,
+                                 hp->pool[k], nullptr);
+        if (first_err == GPTQ2D_OK) first_err = s1 != GPTQ2D_OK ? s1 : s2;
     }
+    // join even if an enqueue failed, so that nothing of this call is left running behind the caller's stream
+    for (int k = 0; k < nslots; ++k)
+        if (cudaEventRecord(hp->pool_done[k], hp->pool[k]) != cudaSuccess ||
+            cudaStreamWaitEvent(stream, hp->pool_done[k], 0) != cudaSuccess)
+            return GPTQ2D_ERR_CUDA;
+    if (first_err != GPTQ2D_OK) return first_err;
     return GPTQ2D_OK;
 }
 

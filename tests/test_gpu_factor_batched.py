@@ -61,6 +61,14 @@ def test_mixed_small_and_large_sides_and_agreement_with_the_single_call(g):
         assert float((U1 - Us[b]).abs().max()) < 1e-10 * max(1.0, float(U1.abs().max()))
 
 
+def test_one_large_problem_among_small_ones_and_many_large_ones(g):
+    """One problem of the blocked route takes gptq2d_factor's two-stream path; several of them are spread
+    over a pool of streams (more problems than streams here, so slots are reused in order)."""
+    check(g, [(64, 64), (300, 200), (5, 7)], seeds=[20, 21, 22])
+    shapes = [(130 + 7 * b, 129 + 5 * b) for b in range(11)] + [(33, 33)]
+    check(g, shapes, seeds=range(30, 30 + len(shapes)))
+
+
 def test_two_hundred_config_c0_like_pairs_feed_the_batched_sweep(g):
     """The use the entry point exists for: factors of many 64 x 64 layers in one launch, then one batched sweep;
     every Z against the oracle's plain-C nested sweep where the certificate allows it."""
