@@ -114,3 +114,24 @@ def test_a_singular_basis_names_its_problem_and_the_others_are_still_factorised(
         L, U, _, _ = O.feedback_factors(A, B)
         assert np.max(np.abs(Ls[b].cpu().numpy() - L)) < 1e-9 * max(1.0, np.max(np.abs(L)))
         assert np.max(np.abs(Us[b].cpu().numpy() - U)) < 1e-9 * max(1.0, np.max(np.abs(U)))
+
+
+def test_the_multi_stream_set_up_is_bit_identical_to_the_one_stream_set_up(g):
+    """With both bases given, gptq2d_factor runs the two sides on two streams and each side's chain of
+    diagonal blocks ahead of its large updates on a third and fourth; with one basis it runs on the
+    caller's stream alone.  Same kernels, same operands, so the outputs must agree bit for bit, run after
+    run (a missing dependency between the streams would show up here)."""
+    torch.manual_seed(3)
+    for k, kb, reps in [(300, 337, 20), (640, 513, 10), (1500, 1200, 4)]:
+        A = torch.randn(k, k, dtype=torch.float64, device="cuda") / k ** 0.5 + torch.eye(k, dtype=torch.float64, device="cuda")
+        B = torch.randn(kb, kb, dtype=torch.float64, device="cuda") / kb ** 0.5 + torch.eye(kb, dtype=torch.float64, device="cuda")
+        L0, _, dL0, _, i0 = g.gptq2d_factor(A, None, n=1)
+        _, U0, _, dU0, i1 = g.gptq2d_factor(None, B, m=1)
+        torch.cuda.synchronize()
+        g.check_info(i0)
+        g.check_info(i1)
+        for _ in range(reps):
+            L, U, dL, dU, info = g.gptq2d_factor(A, B)
+            torch.cuda.synchronize()
+            g.check_info(info)
+            assert torch.equal(L, L0) and torch.equal(U, U0) and torch.equal(dL, dL0) and torch.equal(dU, dU0), k
