@@ -292,6 +292,20 @@ int gptq2d_objective(int m, int n,
                      double *obj,
                      void *workspace, size_t workspace_bytes, int *info, void *stream);
 
+/* ---- test hook for the library's failure handling (the paper has no counterpart; not for production use) ----
+ * Every device-side wait of the sweep kernels is bounded: after a number of polls it gives up, records
+ * where in `info` (GPTQ2D_ERR_DEVICE_TIMEOUT, info[1] = the wait's code, negative), raises an abort word
+ * that all other waits watch, and the kernel returns normally.  This hook lets a test make one such wait
+ * run out WITHOUT faulting or hanging the GPU; the failure is made on the host.
+ *   key 1, value != 0: the next pipelined gptq2d_round_host call (GPTQ2D_FP64) does not announce its last
+ *          copy step to the running kernel (one-shot; cleared by that call).  The tasks that need the step
+ *          wait for it (wait code -6) until their limit.
+ *   key 2, value = polls (about 0.2 us each) after which the wait for a copy step gives up; 0 restores the
+ *          default (about a second).  All other waits keep the default.
+ * Returns GPTQ2D_OK, or GPTQ2D_ERR_INVALID_ARG for an unknown key.
+ */
+int gptq2d_internal_test_hook(int key, long value);
+
 #ifdef __cplusplus
 }
 #endif

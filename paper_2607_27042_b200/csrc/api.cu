@@ -4,6 +4,7 @@
 #include "round_internal.cuh"
 #include "factor.cuh"
 #include <algorithm>
+#include <atomic>
 #include <mutex>
 #include <vector>
 
@@ -13,6 +14,10 @@ int launch_objective(int m, int n, const double *X, long ldx, const int *Z, long
                      const double *B, long ldb, double *obj, void *ws, cudaStream_t stream);
 
 __global__ void margin_kernel(const double *max_abs_e, double *min_margin) { *min_margin = 0.5 - *max_abs_e; }
+
+// Test hooks (gptq2d_internal_test_hook): host-made failures only.
+static std::atomic<long> g_hook_withhold_last_step{0};   // one-shot: the next pipelined host call does not announce its last copy step
+static std::atomic<long> g_hook_panel_spin_limit{0};      // polls a task waits for its copy step (0: default)
 
 static bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -409,8 +414,21 @@ int gptq2d_round_host(int m, int n, const double *hX, const double *hL, const do
         const bool z_pinned = cudaPointerGetAttributes(&za, hZ) == cudaSuccess && za.type == cudaMemoryTypeHost;
         (void)cudaGetLastError();
         tp.panels_ready = dpanels;
+        tp.panel_spin_limit = (unsigned long long)g_hook_panel_spin_limit.load();
+        const bool withhold_last = g_hook_withhold_last_step.exchange(0) != 0;
         int st = launch_round_tiled(tp, w, inner, stream);
         if (st != GPTQ2D_OK) return st;
+        // Every failure from here on leaves through this exit: the kernel and the copy stream's waits are
+        // released (all copy steps "announced", every tile row "swept"), both streams are drained, and
+        // only then does the call return, so nothing of it runs on behind the caller's back.
+        auto fail_out = [&]() {
+            (void)hp->write32(hp->copy, (unsigned long long)reinterpret_cast<uintptr_t>(dpanels), 0x7fffffffu, 0u);
+            (void)cudaMemsetAsync(rowdone, 0x7f, (size_t)ntm_rows * sizeof(unsigned), stream);
+            (void)cudaStreamSynchronize(stream);
+            (void)cudaStreamSynchronize(hp->copy);
+            (void)cudaGetLastError();
+            return (int)GPTQ2D_ERR_CUDA;
+        };
         // From here until the copies are queued the kernel is waiting for this thread: nothing that could
         // block on the device (a first launch of another kernel loads its module, which waits for running
         // kernels) may come in between.
@@ -437,22 +455,19 @@ int gptq2d_round_host(int m, int n, const double *hX, const double *hL, const do
             if (step < nbn)       // columns of block column `step`, rows down to the end of the diagonal block
                 ok = ok && copy2d(dU + (size_t)step * CB, hU + (size_t)step * CB, n,
                                   (step + 1) * CB < n ? (step + 1) * CB : n, extent(step, n));
-            ok = ok && hp->write32(hp->copy, (unsigned long long)reinterpret_cast<uintptr_t>(dpanels),
-                                   (unsigned)(step + 1), 0u) == 0;
+            // (a test may withhold the announcement of the last step: the tasks that need it then run into
+            // their bounded wait and the call reports GPTQ2D_ERR_DEVICE_TIMEOUT)
+            if (!(withhold_last && step == nbm + nbn - 2))
+                ok = ok && hp->write32(hp->copy, (unsigned long long)reinterpret_cast<uintptr_t>(dpanels),
+                                       (unsigned)(step + 1), 0u) == 0;
         }
-        if (!ok) {
-            // the kernel may be waiting for panels that will never come: let it through (its result is
-            // discarded) rather than have it run into its time limit
-            (void)hp->write32(hp->copy, (unsigned long long)reinterpret_cast<uintptr_t>(dpanels), 0x7fffffffu, 0u);
-            (void)cudaStreamSynchronize(stream);
-            return GPTQ2D_ERR_CUDA;
-        }
+        if (!ok) return fail_out();
         // whatever happens in the kernel, no wait of the copy stream may outlast it
         if (z_pinned && cudaMemsetAsync(rowdone, 0x7f, (size_t)ntm_rows * sizeof(unsigned), stream) != cudaSuccess)
-            return GPTQ2D_ERR_CUDA;
+            return fail_out();
         if (hmin_margin) {
             margin_kernel<<<1, 1, 0, stream>>>(workspace_max_abs_e(w), dmargin);
-            if (cudaGetLastError() != cudaSuccess) return GPTQ2D_ERR_CUDA;
+            if (cudaGetLastError() != cudaSuccess) return fail_out();
         }
         if (z_pinned) {
             for (int I = 0; I < ntm_rows && ok; ++I) {
@@ -466,7 +481,7 @@ int gptq2d_round_host(int m, int n, const double *hX, const double *hL, const do
         }
         if (cudaEventRecord(hp->copies_done, hp->copy) != cudaSuccess ||
             cudaStreamWaitEvent(stream, hp->copies_done, 0) != cudaSuccess || !ok)
-            return GPTQ2D_ERR_CUDA;
+            return fail_out();
         pipe_lock.unlock();
     } else
     if (cudaMemcpyAsync(dX, hX, (size_t)m * n * 8, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
@@ -509,6 +524,12 @@ int gptq2d_objective(int m, int n, const double *X, long ldx, const int32_t *Z, 
     if (st != GPTQ2D_OK) return st;
     if (info && cudaMemsetAsync(info, 0, 4 * sizeof(int), stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;
     return launch_objective(m, n, X, ldx, Z, ldz, A, lda, B, ldb, obj, workspace, stream);
+}
+
+int gptq2d_internal_test_hook(int key, long value) {
+    if (key == 1) { g_hook_withhold_last_step.store(value != 0); return GPTQ2D_OK; }
+    if (key == 2) { g_hook_panel_spin_limit.store(value > 0 ? value : 0); return GPTQ2D_OK; }
+    return GPTQ2D_ERR_INVALID_ARG;
 }
 
 }  // extern "C"

@@ -98,18 +98,15 @@ template <bool AK, bool BKc>
 static cudaError_t launch_t(const GemmArgs &g, cudaStream_t stream) {
     using SL = SlabLayout<AK, BKc>;
     size_t smem = (size_t)SL::STAGE_DOUBLES * GEMM_NSTAGE * sizeof(double);
-    static bool configured = false;   // per instantiation; attribute is per device function
-    cudaError_t e;
-    if (!configured) {
-        e = cudaFuncSetAttribute(gemm_kernel<AK, BKc>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        // same shared-memory carve-out as the single-CTA kernels of the set-up that run between the GEMMs, so
-        // that the SMs are not reconfigured from launch to launch
-        e = cudaFuncSetAttribute(gemm_kernel<AK, BKc>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                 cudaSharedmemCarveoutMaxShared);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    // Function attributes are kept per device: set them on every call (two cheap host-side calls), so that
+    // a process that uses several GPUs gets the opt-in on each of them.  Same shared-memory carve-out as the
+    // single-CTA kernels of the set-up that run between the GEMMs, so that the SMs are not reconfigured
+    // from launch to launch.
+    cudaError_t e = cudaFuncSetAttribute(gemm_kernel<AK, BKc>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(gemm_kernel<AK, BKc>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
     dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.batch);
     gemm_kernel<AK, BKc><<<grid, GEMM_THREADS, smem, stream>>>(g);
     return cudaGetLastError();

@@ -47,6 +47,8 @@ struct TiledParams {
     // optional: device word that counts the copy steps of X, L and U that have arrived (the sweep then
     // starts while the rest is still on its way, see COPY_BLOCK_TILES); NULL = everything is resident
     const unsigned *panels_ready;
+    // polls after which the wait for an announced copy step gives up; 0 = the library's default
+    unsigned long long panel_spin_limit;
 };
 // Inputs that arrive while the sweep runs come in blocks of COPY_BLOCK_TILES x COPY_BLOCK_TILES tiles of
 // 128 x 128: step s = the blocks of X on block anti-diagonal s, block row s of L (up to the end of its

@@ -80,6 +80,9 @@ struct TiledKernelParams {
     const unsigned *far_tasks;   // far parts of all matrices in claim order: b << 17 | type << 16 | I << 8 | J
     // pipelined host entry only: number of 128-row panels of X, L and U that have reached the device
     const unsigned *panels_ready;
+    // polls after which a device-side wait gives up (host-set; SPIN_LIMIT unless a test shortens it):
+    // every wait of the kernel, and the wait for an announced copy step of the host entry on its own
+    unsigned long long spin_limit, panel_spin_limit;
 };
 static_assert(sizeof(TiledKernelParams) % 8 == 0, "descriptors are copied as 8-byte words");
 
@@ -233,7 +236,7 @@ __device__ __forceinline__ void await_progress(const TiledKernelParams &p, const
         for (;;) {
             const unsigned va = wa ? ld_acquire_u32(wa) : need, vl = wl ? ld_acquire_u32(wl) : need;
             if (va >= need && vl >= need) break;
-            if (++it > SPIN_LIMIT || ld_relaxed_u32(p.abort) != 0u) {
+            if (++it > p.spin_limit || ld_relaxed_u32(p.abort) != 0u) {
                 report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -8, (int)need, (int)blockIdx.x);
                 atomicExch(p.abort, 1u);
                 break;
@@ -664,7 +667,7 @@ __device__ __forceinline__ unsigned ready_pop(const TiledKernelParams &p) {
         unsigned long long spins = 0;
         unsigned e;
         while ((e = ld_acquire_u32(slot)) == 0u) {          // producer has the ticket but has not written yet
-            if (++spins > SPIN_LIMIT || ld_relaxed_u32(p.abort) != 0u) {
+            if (++spins > p.spin_limit || ld_relaxed_u32(p.abort) != 0u) {
                 report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -3, (int)h, (int)blockIdx.x);
                 atomicExch(p.abort, 1u);
                 return 0u;
@@ -764,7 +767,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                              ((int)(e & 0x7fffu) >> COPY_BLOCK_TILES_LOG2) + 1;
             unsigned long long it = 0;
             while (!panels_arrived(need)) {
-                if (++it > SPIN_LIMIT || ld_relaxed_u32(p.abort) != 0u) {
+                if (++it > p.panel_spin_limit || ld_relaxed_u32(p.abort) != 0u) {
                     report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -6, need, (int)blockIdx.x);
                     atomicExch(p.abort, 1u);
                     return 0u;
@@ -848,7 +851,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
         const int state = s_state;
         if (state >= 3) break;
         if (state == 2) {
-            if (++spins > SPIN_LIMIT) {
+            if (++spins > p.spin_limit) {
                 if (tid == 0) {
                     report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -4, (int)blockIdx.x, s_nctx);
                     atomicExch(p.abort, 1u);
@@ -1038,6 +1041,8 @@ int launch_round_tiled(const TiledParams &in, void *ws, size_t ws_bytes, cudaStr
     if (cudaGetDevice(&dev) != cudaSuccess) return GPTQ2D_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GPTQ2D_ERR_CUDA;
     p.panels_ready = in.panels_ready;
+    p.spin_limit = SPIN_LIMIT;
+    p.panel_spin_limit = in.panel_spin_limit ? in.panel_spin_limit : SPIN_LIMIT;
     const void *kernel = in.panels_ready ? (const void *)round_tiled_kernel<false, true>
                                          : (const void *)round_tiled_kernel<false, false>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TILED_SMEM) != cudaSuccess)
@@ -1138,6 +1143,7 @@ int launch_round_tiled_batched(int count, const TiledParams *pr, double *min_mar
         d.l_al16 = ((reinterpret_cast<uintptr_t>(in.L) & 15) == 0) && ((in.ldl & 1) == 0);
         d.u_al16 = ((reinterpret_cast<uintptr_t>(in.U) & 15) == 0) && ((in.ldu & 1) == 0);
         d.batch_index = b;
+        d.spin_limit = d.panel_spin_limit = SPIN_LIMIT;
         d.ntiles_total = (int)tiles;
         desc[b] = d;
         if (t.ntm + t.ntn - 1 > max_waves) max_waves = t.ntm + t.ntn - 1;
@@ -1167,6 +1173,7 @@ int launch_round_tiled_batched(int count, const TiledParams *pr, double *min_mar
     p.info = info;
     p.probs = reinterpret_cast<const TiledKernelParams *>(w + l.desc_off);
     p.far_tasks = reinterpret_cast<const unsigned *>(w + l.table_off);
+    p.spin_limit = p.panel_spin_limit = SPIN_LIMIT;
 
     if (cudaMemsetAsync(w, 0, l.zero_end, stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;
     // pageable source: the call returns once the bytes have left `stage`

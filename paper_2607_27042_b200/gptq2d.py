@@ -36,6 +36,7 @@ EXPORTS = (
     "gptq2d_round_f32in_workspace_bytes", "gptq2d_round_f32in",
     "gptq2d_round_blocked_workspace_bytes", "gptq2d_round_blocked",
     "gptq2d_factor_batched_workspace_bytes", "gptq2d_factor_batched",
+    "gptq2d_internal_test_hook",
 )
 FACTOR_SMALL_MAX = 128
 
@@ -98,6 +99,8 @@ def _load():
     lib.gptq2d_objective.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, sz, vp, vp]
     lib.gptq2d_round_static.restype = i32
     lib.gptq2d_round_static.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, vp]
+    lib.gptq2d_internal_test_hook.restype = i32
+    lib.gptq2d_internal_test_hook.argtypes = [i32, lng]
     lib.gptq2d_round_static_max_dim.restype = sz
     lib.gptq2d_round_static_max_dim.argtypes = []
     lib.gptq2d_round_f32in.restype = i32
@@ -401,6 +404,14 @@ def gptq2d_round_blocked(X, L, U, w, Z=None, E=None, min_margin=None, workspace=
     if st != OK:
         raise Gptq2dError(st)
     return Z, E, min_margin, info
+
+
+def gptq2d_internal_test_hook(key, value):
+    """Host-made failure for tests (see the header): 1 = withhold the last copy step of the next pipelined
+    host call, 2 = polls after which the wait for a copy step gives up (0: default)."""
+    st = _lib.gptq2d_internal_test_hook(int(key), int(value))
+    if st != OK:
+        raise Gptq2dError(st)
 
 
 def gptq2d_round_static_max_dim():
