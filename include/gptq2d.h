@@ -54,9 +54,12 @@ typedef enum {
 
 typedef enum {
     GPTQ2D_FP64 = 0,   /* all sweep arithmetic in fp64 (tiled wavefront kernel)                       */
-    GPTQ2D_FP32 = 1,   /* X, L, U rounded to fp32 and all sweep arithmetic in fp32 (Algorithm 3 as
-                          written, one grid-wide barrier per anti-diagonal); Z may differ from FP64  */
+    GPTQ2D_FP32 = 1,   /* X, L, U rounded to fp32 and all sweep arithmetic in fp32, on 64 x 64 tiles (the
+                          tile restatement of Algorithm 3; far feedback as an FFMA contraction); Z may
+                          differ from FP64 wherever a pre-rounding value lies within fp32 error of a tie */
     GPTQ2D_FP64_UNTILED = 2, /* fp64 with the untiled Algorithm-3 kernel; a cross-check, not fast     */
+    GPTQ2D_FP32_UNTILED = 4, /* fp32 with the untiled Algorithm-3 kernel (one grid-wide barrier per
+                               anti-diagonal): the literal order of operations in fp32; a cross-check, not fast */
     GPTQ2D_FP64_PULL = 3    /* fp64, implicit-Y form (Algorithm 6, Eq. 19-20) with C pulled as well: every
                                entry reconstructs its corrected value from L, E, C, U at rounding time;
                                untiled and bound by memory bandwidth: the comparison point, not fast   */
@@ -302,9 +305,21 @@ int gptq2d_objective(int m, int n,
  *          wait for it (wait code -6) until their limit.
  *   key 2, value = polls (about 0.2 us each) after which the wait for a copy step gives up; 0 restores the
  *          default (about a second).  All other waits keep the default.
+ *   key 3, value 0 / 1: route the library's fp64 products (set-up, objective) through the cp.async kernel
+ *          only / through the TMA-fed kernel where the operands allow it (default 1).  Comparison runs.
  * Returns GPTQ2D_OK, or GPTQ2D_ERR_INVALID_ARG for an unknown key.
  */
 int gptq2d_internal_test_hook(int key, long value);
+
+/* The library's own fp64 product, exposed for tests and for measuring the fp64 tensor rate it reaches
+ * (the denominator the sweep's roofline is quoted against): C = alpha op(A) op(B) + beta C, row-major,
+ * op(A) M x K (stored K x M if transa), op(B) K x N (stored N x K if transb).  Device pointers, 8-byte
+ * aligned; enqueues on `stream`.  This is the dense contraction that the set-up (Section 3.1) and the
+ * objective (Eq. 7) are made of, and the same tile loop that carries the far parts of the sweep.
+ */
+int gptq2d_internal_gemm(int transa, int transb, int M, int N, int K, double alpha,
+                         const double *A, long lda, const double *B, long ldb,
+                         double beta, double *C, long ldc, void *stream);
 
 #ifdef __cplusplus
 }

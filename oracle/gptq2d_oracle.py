@@ -37,7 +37,7 @@ __all__ = [
     "objective", "objective_kron", "objective_from_errors", "gptq_one_sided_elimination",
     "unit_upper_udu_of_inverse", "feedback_factors_reverse", "adaptive_round_1d_reverse",
     "vec_sweep_reverse", "sweep_gptq2d_reverse", "brute_force_trajectory_reverse",
-    "certificate_margin_reverse",
+    "certificate_margin_reverse", "sweep_gptq2d_fp32",
 ]
 
 
@@ -492,3 +492,40 @@ def certificate_margin_reverse(X, Z, Lr, Ur):
     Et = sla.solve_triangular(Ur.T, T.T, lower=False, unit_diagonal=True)
     E = Et.T.copy()
     return float(0.5 - np.max(np.abs(E))), E
+
+
+def sweep_gptq2d_fp32(X, L, U):
+    """Algorithm 3 with every value held and every operation rounded in IEEE single precision.
+
+    TEST INFRASTRUCTURE (reduced-precision mode).  X, L, U are rounded to float32 first; the steps are those of
+    Algorithm 3 in the paper's order (round, error, scale by the column of L, fold into C, push down; then push
+    right from the folded C), with numpy float32 arithmetic: products and sums are rounded separately (no fused
+    multiply-add).  Z is returned as int64, E and C as float32.  A tiled fp32 kernel sums in another order, so it
+    agrees with this only up to fp32 rounding: entries whose pre-rounding value lies within that error of a
+    half-integer may differ, and every such flip moves the entries below and to the right of it.
+    """
+    X = np.asarray(X, dtype=np.float32)
+    L = np.asarray(L, dtype=np.float32)
+    U = np.asarray(U, dtype=np.float32)
+    m, n = X.shape
+    Y = X.copy()
+    C = np.zeros((m, n), dtype=np.float32)
+    E = np.zeros((m, n), dtype=np.float32)
+    Z = np.zeros((m, n), dtype=np.int64)
+    for s in range(m + n - 1):
+        lo, hi = max(0, s - n + 1), min(m - 1, s)
+        rows = np.arange(lo, hi + 1)
+        cols = s - rows
+        y = Y[rows, cols]
+        z = np.rint(y)
+        e = (z - y).astype(np.float32)
+        Z[rows, cols] = z.astype(np.int64)
+        E[rows, cols] = e
+        for i, j, eij in zip(rows, cols, e):            # fold and push down, column by column
+            M = (L[i:, i] * eij).astype(np.float32)
+            M[0] = eij                                    # L_ii = 1
+            C[i:, j] = (C[i:, j] + M).astype(np.float32)
+            Y[i + 1:, j] = (Y[i + 1:, j] + M[1:]).astype(np.float32)
+        for i, j in zip(rows, cols):                     # push right from the folded C
+            Y[i, j + 1:] = (Y[i, j + 1:] + (C[i, j] * U[j, j + 1:]).astype(np.float32)).astype(np.float32)
+    return {"Z": Z, "E": E, "C": C, "margin": float(0.5 - np.max(np.abs(E))) if E.size else 0.5}

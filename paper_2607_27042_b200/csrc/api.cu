@@ -3,6 +3,7 @@
 #include "common.cuh"
 #include "round_internal.cuh"
 #include "factor.cuh"
+#include "gemm.cuh"
 #include <algorithm>
 #include <atomic>
 #include <mutex>
@@ -286,7 +287,8 @@ int gptq2d_factor_batched(int count, const gptq2d_factor_problem_t *pr, void *wo
 size_t gptq2d_round_workspace_bytes(int m, int n, int precision) {
     if (m < 1 || n < 1) return 0;
     if (precision == GPTQ2D_FP64) return round_tiled_workspace_bytes(m, n);
-    if (precision == GPTQ2D_FP32) return round_untiled_workspace_bytes(m, n, true);
+    if (precision == GPTQ2D_FP32) return round_tiled_f32_workspace_bytes(m, n);
+    if (precision == GPTQ2D_FP32_UNTILED) return round_untiled_workspace_bytes(m, n, true);
     if (precision == GPTQ2D_FP64_UNTILED) return round_untiled_workspace_bytes(m, n, false);
     if (precision == GPTQ2D_FP64_PULL) return round_pull_workspace_bytes(m, n);
     return 0;
@@ -302,7 +304,7 @@ int gptq2d_round(int m, int n, const double *X, long ldx, const double *L, long 
         !aligned(min_margin, 8))
         return GPTQ2D_ERR_INVALID_ARG;
     if (precision != GPTQ2D_FP64 && precision != GPTQ2D_FP32 && precision != GPTQ2D_FP64_UNTILED &&
-        precision != GPTQ2D_FP64_PULL)
+        precision != GPTQ2D_FP64_PULL && precision != GPTQ2D_FP32_UNTILED)
         return GPTQ2D_ERR_INVALID_ARG;
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < gptq2d_round_workspace_bytes(m, n, precision))
         return GPTQ2D_ERR_WORKSPACE;
@@ -316,6 +318,12 @@ int gptq2d_round(int m, int n, const double *X, long ldx, const double *L, long 
         p.X = X; p.ldx = ldx; p.L = L; p.ldl = ldl; p.U = U; p.ldu = ldu;
         p.Z = Z; p.ldz = ldz; p.E = E; p.lde = lde; p.info = info;
         st = launch_round_tiled(p, workspace, workspace_bytes, stream);
+    } else if (precision == GPTQ2D_FP32) {
+        TiledParams p{};
+        p.m = m; p.n = n;
+        p.X = X; p.ldx = ldx; p.L = L; p.ldl = ldl; p.U = U; p.ldu = ldu;
+        p.Z = Z; p.ldz = ldz; p.E = E; p.lde = lde; p.info = info;
+        st = launch_round_tiled_f32(p, workspace, workspace_bytes, stream);
     } else if (precision == GPTQ2D_FP64_PULL) {
         PullParams p{};
         p.m = m; p.n = n;
@@ -327,7 +335,7 @@ int gptq2d_round(int m, int n, const double *X, long ldx, const double *L, long 
         p.m = m; p.n = n;
         p.X = X; p.ldx = ldx; p.L = L; p.ldl = ldl; p.U = U; p.ldu = ldu;
         p.Z = Z; p.ldz = ldz; p.E = E; p.lde = lde; p.info = info;
-        st = launch_round_untiled(p, precision == GPTQ2D_FP32, workspace, stream);
+        st = launch_round_untiled(p, precision == GPTQ2D_FP32_UNTILED, workspace, stream);
     }
     if (st != GPTQ2D_OK) return st;
     if (min_margin) {
@@ -529,7 +537,22 @@ int gptq2d_objective(int m, int n, const double *X, long ldx, const int32_t *Z, 
 int gptq2d_internal_test_hook(int key, long value) {
     if (key == 1) { g_hook_withhold_last_step.store(value != 0); return GPTQ2D_OK; }
     if (key == 2) { g_hook_panel_spin_limit.store(value > 0 ? value : 0); return GPTQ2D_OK; }
+    if (key == 3) { gemm_set_tma_mode((int)value); return GPTQ2D_OK; }
+    if (key == 4) { round_fused_set_mode((int)value); return GPTQ2D_OK; }
     return GPTQ2D_ERR_INVALID_ARG;
+}
+
+int gptq2d_internal_gemm(int transa, int transb, int M, int N, int K, double alpha, const double *A, long lda,
+                         const double *B, long ldb, double beta, double *C, long ldc, void *stream_) {
+    if (M < 1 || N < 1 || K < 1 || !A || !B || !C) return GPTQ2D_ERR_INVALID_ARG;
+    if (lda < (transa ? M : K) || ldb < (transb ? K : N) || ldc < N) return GPTQ2D_ERR_INVALID_ARG;
+    int st = check_device();
+    if (st != GPTQ2D_OK) return st;
+    GemmArgs g{};
+    g.opA = transa ? OP_T : OP_N; g.opB = transb ? OP_T : OP_N;
+    g.M = M; g.N = N; g.K = K; g.alpha = alpha; g.beta = beta;
+    g.A = A; g.lda = lda; g.B = B; g.ldb = ldb; g.C = C; g.ldc = ldc; g.batch = 1;
+    return launch_gemm(g, static_cast<cudaStream_t>(stream_)) == cudaSuccess ? GPTQ2D_OK : GPTQ2D_ERR_CUDA;
 }
 
 }  // extern "C"

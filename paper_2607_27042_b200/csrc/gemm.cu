@@ -1,5 +1,7 @@
 // The library's own fp64 GEMM kernel: one CTA per 128 x 128 output tile, DMMA mainloop.
 #include "dmma_gemm.cuh"
+#include "dmma_tma.cuh"
+#include "tma_host.cuh"
 #include "gemm.cuh"
 
 namespace gptq2d {
@@ -94,8 +96,152 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(GemmArgs p) {
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// The same GEMM with TMA-fed operand slabs (dmma_tma.cuh): used whenever both operands are 16-byte
+// aligned with even leading dimensions.  Ragged edges need no special loop here: parts of a box that
+// lie outside the tensor read as zeros.
+constexpr int GEMM_TMA_NSTAGE = 4;
+constexpr size_t GEMM_TMA_SMEM = (size_t)GEMM_TMA_NSTAGE * TMA_STAGE_BYTES + 1024;   // + slack to align the ring to 1024 B
+
+// pair q (0..3) of row-fragment a: two horizontally adjacent elements of the tile held by this lane
+template <bool B_KCONTIG>
+__device__ __forceinline__ void acc_pair(const Acc &acc, int a, int q, int wn, int t, int &col, double &x0, double &x1) {
+    if (B_KCONTIG) {
+        const int bq = q >> 1, j = q & 1;
+        col = wn * 32 + bq * 16 + 4 * t + 2 * j;
+        x0 = acc.v[a][2 * bq][j];
+        x1 = acc.v[a][2 * bq + 1][j];
+    } else {
+        col = acc_col<false>(wn, q, t, 0);
+        x0 = acc.v[a][q][0];
+        x1 = acc.v[a][q][1];
+    }
+}
+
+template <bool A_KCONTIG, bool B_KCONTIG, bool SLAB_SYNC>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+gemm_tma_kernel(GemmArgs p, const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                unsigned *abort) {
+    extern __shared__ __align__(16) double smem_raw[];
+    __shared__ __align__(8) unsigned long long bars[2 * GEMM_TMA_NSTAGE];
+    const int tn = blockIdx.x, tm = blockIdx.y, bz = blockIdx.z;
+    if (p.lower_tiles_only && tn > tm) return;
+    const int m0 = tm * BM, n0 = tn * BN;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int wm = warp >> 2, wn = warp & 3, g = lane >> 2, t = lane & 3;
+    // aligned to 1024 bytes by an offset into the shared array (pointer arithmetic keeps the shared address space)
+    double *stages = smem_raw + (((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u) >> 3);
+
+    TmaRing ring;
+    tma_ring_init<GEMM_TMA_NSTAGE, GEMM_THREADS / 32>(ring, bars, stages, tid);
+    __syncthreads();
+
+    const int k_lo = p.b_lower ? min(p.K, n0) : 0;
+    const int k_hi = p.a_lower ? min(p.K, m0 + BM) : p.K;
+    Acc acc;
+    acc.zero();
+    if (k_hi > k_lo) {
+        TmaOperand A{&mapA, m0, k_lo, bz}, B{&mapB, n0, k_lo, bz};
+        const int nk = (k_hi - k_lo + TMA_BK - 1) / TMA_BK;
+        if (!gemm_tma_mainloop<A_KCONTIG, B_KCONTIG, GEMM_TMA_NSTAGE, SLAB_SYNC ? 1 : -1>(acc, ring, A, B, nk, warp, lane, abort))
+            return;
+    }
+
+    if (p.sumsq_partials) {
+        double s = 0.0;
+#pragma unroll
+        for (int a = 0; a < 8; ++a)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                double x0 = p.alpha * acc.v[a][b][0], x1 = p.alpha * acc.v[a][b][1];
+                s = fma(x0, x0, s);
+                s = fma(x1, x1, s);
+            }
+        // NOTE: the order of this sum differs from the cp.async kernel's (another element-to-lane map)
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        __shared__ double wsum[8];
+        if (lane == 0) wsum[warp] = s;
+        __syncthreads();
+        if (tid == 0) {
+            double tot = 0.0;
+            for (int w = 0; w < 8; ++w) tot += wsum[w];
+            p.sumsq_partials[((long)bz * gridDim.y + tm) * gridDim.x + tn] = tot;
+        }
+        return;
+    }
+
+    double *Cb = p.C + (long)bz * p.strideC;
+    const bool vec = ((((uintptr_t)Cb) & 15) == 0) && ((p.ldc & 1) == 0);
+#pragma unroll
+    for (int a = 0; a < 8; ++a) {
+        const int r = m0 + acc_row<A_KCONTIG>(wm, a, g);
+        if (r >= p.M) continue;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            int col;
+            double x0, x1;
+            acc_pair<B_KCONTIG>(acc, a, q, wn, t, col, x0, x1);
+            const int c = n0 + col;
+            if (c >= p.N) continue;
+            double *dst = Cb + (long)r * p.ldc + c;
+            x0 *= p.alpha; x1 *= p.alpha;
+            if (c + 1 < p.N && vec) {
+                double2 o;
+                if (p.beta != 0.0) {
+                    double2 old = *reinterpret_cast<const double2 *>(dst);
+                    o.x = fma(p.beta, old.x, x0);
+                    o.y = fma(p.beta, old.y, x1);
+                } else {
+                    o.x = x0;
+                    o.y = x1;
+                }
+                *reinterpret_cast<double2 *>(dst) = o;
+            } else {
+                dst[0] = (p.beta != 0.0) ? fma(p.beta, dst[0], x0) : x0;
+                if (c + 1 < p.N) dst[1] = (p.beta != 0.0) ? fma(p.beta, dst[1], x1) : x1;
+            }
+        }
+    }
+}
+
+static int g_gemm_tma_mode = 1;       // 0: cp.async kernel only; 1: TMA-fed kernel; 2: TMA-fed kernel with a barrier per slab
+void gemm_set_tma_mode(int mode) { g_gemm_tma_mode = mode; }
+
+template <bool AK, bool BKc, bool SS>
+static cudaError_t launch_tma_variant(const GemmArgs &g, const CUtensorMap &mapA, const CUtensorMap &mapB, cudaStream_t stream) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tma_kernel<AK, BKc, SS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GEMM_TMA_SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(gemm_tma_kernel<AK, BKc, SS>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
+    dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.batch);
+    gemm_tma_kernel<AK, BKc, SS><<<grid, GEMM_THREADS, GEMM_TMA_SMEM, stream>>>(g, mapA, mapB, g.abort);
+    return cudaGetLastError();
+}
+
+// false: this GEMM cannot take the TMA path (alignment, no encoder); *err holds a launch error if it was tried
+template <bool AK, bool BKc>
+static bool try_launch_tma(const GemmArgs &g, cudaStream_t stream, cudaError_t *err) {
+    if (g_gemm_tma_mode == 0) return false;
+    CUtensorMap mapA, mapB;
+    // op(A) is M x K: stored M x K (k contiguous) if AK, else K x M (m contiguous)
+    const bool okA = AK ? encode_f64_matrix_map(&mapA, g.A, g.M, g.K, g.lda, g.batch, g.strideA, 16, 128)
+                        : encode_f64_matrix_map(&mapA, g.A, g.K, g.M, g.lda, g.batch, g.strideA, 16, 16);
+    if (!okA) return false;
+    // op(B) is K x N: stored N x K (k contiguous) if BKc, else K x N (n contiguous)
+    const bool okB = BKc ? encode_f64_matrix_map(&mapB, g.B, g.N, g.K, g.ldb, g.batch, g.strideB, 16, 128)
+                         : encode_f64_matrix_map(&mapB, g.B, g.K, g.N, g.ldb, g.batch, g.strideB, 16, 16);
+    if (!okB) return false;
+    *err = g_gemm_tma_mode == 2 ? launch_tma_variant<AK, BKc, true>(g, mapA, mapB, stream)
+                                : launch_tma_variant<AK, BKc, false>(g, mapA, mapB, stream);
+    return true;
+}
+
 template <bool AK, bool BKc>
 static cudaError_t launch_t(const GemmArgs &g, cudaStream_t stream) {
+    cudaError_t terr = cudaSuccess;
+    if (try_launch_tma<AK, BKc>(g, stream, &terr)) return terr;
     using SL = SlabLayout<AK, BKc>;
     size_t smem = (size_t)SL::STAGE_DOUBLES * GEMM_NSTAGE * sizeof(double);
     // Function attributes are kept per device: set them on every call (two cheap host-side calls), so that

@@ -23,9 +23,14 @@ struct GemmArgs {
     int b_lower;            // op(B) is lower triangular (K x N, zero for k < n): tile column tn starts at k = 128 tn
     double *sumsq_partials; // if non-null: do not store C; write sum(C^2) of each CTA tile
                             // to sumsq_partials[tile index] (tiles_m * tiles_n * batch entries)
+    unsigned *abort;        // optional device word: raised if a bounded wait of the TMA-fed kernel runs out
+                            // (the tile is then not written); NULL: nobody is told
 };
 
 // Enqueues the GEMM on `stream`.  Returns cudaSuccess or the launch error.
 cudaError_t launch_gemm(const GemmArgs &g, cudaStream_t stream);
+// 1 (default): operands that are 16-byte aligned with even leading dimensions go through the TMA-fed kernel;
+// 2: the same with a CTA barrier per slab; 0: everything through the cp.async kernel (comparison runs).
+void gemm_set_tma_mode(int mode);
 
 }  // namespace gptq2d

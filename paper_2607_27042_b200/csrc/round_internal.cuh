@@ -59,6 +59,12 @@ size_t round_tiled_workspace_bytes(int m, int n);
 // device array inside the workspace: for each row of 128 x 128 tiles, how many of its tiles are swept
 unsigned *round_tiled_rowdone(void *ws, int m, int n);
 int launch_round_tiled(const TiledParams &p, void *ws, size_t ws_bytes, cudaStream_t stream);
+// The sixteen-warp kernel for large resident problems (round_fused.cu).  Modes: 0 never, 1 where it pays
+// (default), 2 whenever the operands allow it (tests).
+void round_fused_set_mode(int mode);
+// fp32 mode, tiled (round_tiled_f32.cu): X, L, U as fp64 device arrays, narrowed into the workspace
+size_t round_tiled_f32_workspace_bytes(int m, int n);
+int launch_round_tiled_f32(const TiledParams &p, void *ws, size_t ws_bytes, cudaStream_t stream);
 // many matrices in one launch (fp64 tiled sweep); `info` is shared, `min_margin` (optional) gets one value per matrix
 constexpr int BATCH_MAX_COUNT = 8192;     // matrix index has 13 bits in a ready-ring entry
 constexpr int BATCH_MAX_DIM = 32768;      // tile coordinates have 8 bits there

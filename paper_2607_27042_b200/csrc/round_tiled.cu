@@ -1001,6 +1001,18 @@ static TiledLayout tiled_layout(int m, int n) {
 }
 
 size_t round_tiled_workspace_bytes(int m, int n) { return tiled_layout(m, n).total; }
+
+// the same layout for the sixteen-warp kernel (round_fused.cu), which shares the workspace format
+struct TiledLayoutView {
+    int ntm, ntn;
+    size_t q_off, flags_off, quad_off, qdep_off, qprog_off, rowdone_off, e_off, c_off, total;
+};
+TiledLayoutView round_tiled_layout_view(int m, int n) {
+    const TiledLayout l = tiled_layout(m, n);
+    return TiledLayoutView{l.ntm, l.ntn, l.q_off, l.flags_off, l.quad_off, l.qdep_off, l.qprog_off, l.rowdone_off,
+                           l.e_off, l.c_off, l.total};
+}
+int launch_round_fused(const TiledParams &in, void *ws, size_t ws_bytes, cudaStream_t stream, bool force);
 unsigned *round_tiled_rowdone(void *ws, int m, int n) {
     return reinterpret_cast<unsigned *>(static_cast<char *>(ws) + tiled_layout(m, n).rowdone_off);
 }
@@ -1008,6 +1020,11 @@ unsigned *round_tiled_rowdone(void *ws, int m, int n) {
 int launch_round_tiled(const TiledParams &in, void *ws, size_t ws_bytes, cudaStream_t stream) {
     TiledLayout l = tiled_layout(in.m, in.n);
     if (ws_bytes < l.total) return GPTQ2D_ERR_WORKSPACE;
+    {
+        // large resident problems: far contractions and quadrant tasks side by side on every SM
+        const int st = launch_round_fused(in, ws, ws_bytes, stream, false);
+        if (st != -1) return st;
+    }
     char *w = static_cast<char *>(ws);
     TiledKernelParams p{};
     p.m = in.m; p.n = in.n; p.ntm = l.ntm; p.ntn = l.ntn;

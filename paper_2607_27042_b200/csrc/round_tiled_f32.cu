@@ -1,0 +1,452 @@
+// GPTQ-2D sweep in fp32 (the optional reduced-precision mode), tiled.
+//
+// X, L and U are rounded to fp32 and every operation of Algorithm 3 is carried out in fp32; the order of
+// the sums is that of the tile restatement (Eq. 11, Eq. 15-17), not of the literal algorithm: for the
+// 64 x 64 tile (I, J) with rows r and columns c
+//     Cd = sum_{I' < I} L[r, I'] E[I', c]        Rt = sum_{J' < J} C[r, J'] U[J', c]
+// and Algorithm 3 on the tile alone, started from Y = X[r, c] + Rt + Cd and C = Cd with the diagonal
+// blocks L[r, r] and U[c, c], gives the tile's Z, E and C = L E.  fp32 has no tensor-core path that keeps
+// fp32 operands exact (TF32 truncates them), so the two contractions are a register-tiled FFMA loop:
+// 256 threads, a 4 x 4 piece of the tile per thread and contraction, operand slabs of 16 staged through
+// shared memory with cp.async.
+//
+// One persistent, cooperatively launched grid, two CTAs per SM.  Tiles are claimed wave by wave (I + J
+// ascending) from one atomic counter; a CTA folds the source tiles in as their flags come up -- the far
+// ones first, the tile above and the tile to the left last -- and then sweeps its tile.  While one CTA
+// of an SM sits in the dependent chain of its in-tile sweep the other one multiplies.  A tile only waits
+// for tiles of earlier waves, which were claimed earlier, so the earliest unfinished tile can always run.
+//
+// In-tile sweep: one anti-diagonal per step, four threads per row.  Row i of the tile is only ever
+// written by its own four threads -- they apply the downward pushes INTO row i (regrouped by target row:
+// the targets (i, s - i') of all sources i' < i on anti-diagonal s are contiguous, and so are the
+// coefficients L[i][i']) and the rightward push OF row i's entry -- so the only thing that crosses rows is
+// the vector of errors of the current anti-diagonal: one CTA barrier per step.
+#include "common.cuh"
+#include "dmma_gemm.cuh"          // cp.async helpers
+#include "round_internal.cuh"
+
+namespace gptq2d {
+namespace f32 {
+
+constexpr int TS = 64;             // tile edge
+constexpr int THREADS = 256;
+constexpr int KS = 16;             // slab depth
+constexpr int NSTAGE = 6;          // cp.async ring; it lives where the in-tile matrices go afterwards
+constexpr int LDA = KS + 4;        // A slab [64 rows][16 k], row stride 20 floats: 16-byte rows, conflict-free float4 reads
+constexpr int LDB = TS + 4;        // B slab [16 k][64 cols], row stride 68 floats
+constexpr int A_FLOATS = TS * LDA, B_FLOATS = KS * LDB, STAGE_FLOATS = A_FLOATS + B_FLOATS;
+constexpr int LDT = TS + 4;        // in-tile matrices, row stride 68 floats: the 8 rows x 4 lanes of a warp hit 32 different banks
+                                   // in the push loops (bank = 4 row -+ lane)
+constexpr int TMAT = TS * LDT;
+constexpr int SWEEP_FLOATS = 4 * TMAT + 2 * TS, RING_FLOATS = NSTAGE * STAGE_FLOATS;
+constexpr size_t SMEM_BYTES = (size_t)(SWEEP_FLOATS > RING_FLOATS ? SWEEP_FLOATS : RING_FLOATS) * sizeof(float);
+
+struct Params {
+    int m, n, nti, ntj, ntiles;
+    long mp, np;                   // padded extents (multiples of 64): leading dimension of E32 / C32 is np
+    const double *X; long ldx;
+    int *Z; long ldz;
+    double *Euser; long lde;
+    const float *L32; long ldl;    // m x m (leading dimension padded to a multiple of 4)
+    const float *U32; long ldu;
+    float *E32, *C32;
+    unsigned *counter, *abort, *flags;
+    double *max_abs_e;
+    int *info;
+    unsigned long long spin_limit;
+};
+
+__device__ __forceinline__ void cp_async16f(float *smem, const float *gmem, int src_bytes) {
+    unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gmem), "r"(src_bytes) : "memory");
+}
+
+// tile index in claim order -> (I, J): wave by wave, I ascending inside a wave
+__device__ __forceinline__ void decode_tile(int task, int nti, int ntj, int &I, int &J) {
+    int tt = task;
+    for (int w = 0; w < nti + ntj - 1; ++w) {
+        const int lo = max(0, w - ntj + 1), hi = min(nti - 1, w);
+        const int cnt = hi - lo + 1;
+        if (tt < cnt) { I = lo + tt; J = w - I; return; }
+        tt -= cnt;
+    }
+    I = J = 0;
+}
+
+// One source tile: acc += A (64 x 64, [row][k], leading dimension lda) * B (64 x 64, [k][col], ldb), both fully
+// inside padded or zero-filled storage except that rows of A beyond `a_rows` and columns of B beyond `b_cols`
+// (ragged edge of a user matrix) are read as zeros.  K is streamed in four slabs of 16.
+struct Gemm {
+    float *stages;
+    int tid, ty, tx;
+    // copy plan: A slab = 64 rows x 16 k = 256 chunks of 4 floats (one per thread); B slab = 16 k x 64 cols likewise
+    __device__ __forceinline__ void issue(int stage, const float *A, long lda, int a_rows, int a_kmax, const float *B, long ldb,
+                                          int b_cols, int b_kmax, int k0) const {
+        float *As = stages + stage * STAGE_FLOATS, *Bs = As + A_FLOATS;
+        {
+            const int r = tid >> 2, kc = (tid & 3) * 4;
+            int nv = (r < a_rows) ? a_kmax - (k0 + kc) : 0;          // floats valid from kc on
+            nv = nv < 0 ? 0 : (nv > 4 ? 4 : nv);
+            cp_async16f(As + r * LDA + kc, nv ? A + (long)r * lda + k0 + kc : A, nv * 4);
+        }
+        {
+            const int kr = tid >> 4, cc = (tid & 15) * 4;
+            int nv = (k0 + kr < b_kmax) ? b_cols - cc : 0;
+            nv = nv < 0 ? 0 : (nv > 4 ? 4 : nv);
+            cp_async16f(Bs + kr * LDB + cc, nv ? B + (long)(k0 + kr) * ldb + cc : B, nv * 4);
+        }
+    }
+    __device__ __forceinline__ void multiply(float (&acc)[4][4], int stage) const {
+        const float *As = stages + stage * STAGE_FLOATS, *Bs = As + A_FLOATS;
+#pragma unroll
+        for (int k4 = 0; k4 < KS; k4 += 4) {
+            float4 a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = *reinterpret_cast<const float4 *>(As + (ty * 4 + i) * LDA + k4);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) b[k] = *reinterpret_cast<const float4 *>(Bs + (k4 + k) * LDB + tx * 4);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float av[4] = {a[i].x, a[i].y, a[i].z, a[i].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    acc[i][0] = fmaf(av[k], b[k].x, acc[i][0]);
+                    acc[i][1] = fmaf(av[k], b[k].y, acc[i][1]);
+                    acc[i][2] = fmaf(av[k], b[k].z, acc[i][2]);
+                    acc[i][3] = fmaf(av[k], b[k].w, acc[i][3]);
+                }
+            }
+        }
+    }
+};
+
+__global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
+    extern __shared__ __align__(16) float smem[];
+    __shared__ int s_task;
+    __shared__ int s_ok;
+    __shared__ double s_red[THREADS / 32];
+    __shared__ unsigned long long s_badkey;
+    float *stages = smem;
+    // the contraction's accumulators are registers, so the in-tile matrices reuse the ring's memory
+    float *Ys = smem, *Cs = Ys + TMAT, *Ld = Cs + TMAT, *Ud = Ld + TMAT;
+    float *ebuf = Ud + TMAT;                       // [2][64]: errors of the current anti-diagonal, by source row
+    const int tid = threadIdx.x;
+    Gemm gm{stages, tid, tid >> 4, tid & 15};
+    double max_abs_e = 0.0;
+    if (tid == 0) s_badkey = ~0ull;
+
+    for (;;) {
+        __syncthreads();
+        if (tid == 0) {
+            int task = -1;
+            if (ld_relaxed_u32(p.abort) == 0u) {
+                task = (int)atomicAdd(p.counter, 1u);
+                if (task >= p.ntiles) task = -1;
+            }
+            s_task = task;
+        }
+        __syncthreads();
+        const int task = s_task;
+        if (task < 0) break;
+        int I, J;
+        decode_tile(task, p.nti, p.ntj, I, J);
+        const int row0 = I * TS, col0 = J * TS;
+
+        // ---- 1. the two contractions.  Source list: tiles (0..I-2, J) through L, tiles (I, 0..J-2) through U, then
+        // the tile above and the tile to the left (the newest ones, still being swept when this tile is claimed).
+        float cd[4][4], rt[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) cd[i][j] = rt[i][j] = 0.f;
+        const int nsrc = I + J, nslab = nsrc * (TS / KS);
+        bool ok = true;
+        // slab g of the flattened list belongs to source g / 4; operands of a source (all threads compute them)
+        struct Src { const float *A, *B; long lda, ldb; int a_rows, a_kmax, b_cols, b_kmax, dir; const unsigned *flag; };
+        auto source = [&](int sidx) {
+            int dir, k;
+            const int na = max(0, I - 1), nl = max(0, J - 1);        // older sources of each direction
+            if (sidx < na) { dir = 0; k = sidx; }
+            else if (sidx < na + nl) { dir = 1; k = sidx - na; }
+            else if (sidx == na + nl && I > 0) { dir = 0; k = I - 1; }
+            else { dir = 1; k = J - 1; }
+            Src r;
+            r.dir = dir;
+            if (dir == 0) {          // L[r, rows of tile k] * E[rows of tile k, c]
+                r.A = p.L32 + (long)row0 * p.ldl + (long)k * TS; r.lda = p.ldl;
+                r.a_rows = min(TS, p.m - row0); r.a_kmax = min(TS, p.m - k * TS);
+                r.B = p.E32 + (long)k * TS * p.np + col0; r.ldb = p.np; r.b_cols = TS; r.b_kmax = TS;
+                r.flag = p.flags + (long)k * p.ntj + J;
+            } else {                 // C[r, columns of tile k] * U[columns of tile k, c]
+                r.A = p.C32 + (long)row0 * p.np + (long)k * TS; r.lda = p.np; r.a_rows = TS; r.a_kmax = TS;
+                r.B = p.U32 + (long)k * TS * p.ldu + col0; r.ldb = p.ldu;
+                r.b_cols = min(TS, p.n - col0); r.b_kmax = min(TS, p.n - k * TS);
+                r.flag = p.flags + (long)I * p.ntj + k;
+            }
+            return r;
+        };
+        // Issues slab g (all threads).  The first slab of a source waits, bounded, for the source tile's flag;
+        // returns false if that wait ran out.
+        auto issue_slab = [&](int g) -> bool {
+            const Src sr = source(g >> 2);
+            if ((g & 3) == 0) {
+                if (tid == 0) {
+                    unsigned long long it = 0;
+                    int good = 1;
+                    while (ld_acquire_u32(sr.flag) == 0u) {
+                        if (++it > p.spin_limit || ld_relaxed_u32(p.abort) != 0u) {
+                            report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -9, task, (int)blockIdx.x);
+                            atomicExch(p.abort, 1u);
+                            good = 0;
+                            break;
+                        }
+                        __nanosleep(100);
+                    }
+                    s_ok = good;
+                }
+                __syncthreads();
+                const bool good = s_ok != 0;
+                __syncthreads();                       // s_ok may be rewritten by the next wait
+                if (!good) return false;
+            }
+            gm.issue(g % NSTAGE, sr.A, sr.lda, sr.a_rows, sr.a_kmax, sr.B, sr.ldb, sr.b_cols, sr.b_kmax, (g & 3) * KS);
+            return true;
+        };
+        for (int g = 0; g < NSTAGE - 1 && ok; ++g) {
+            if (g < nslab) ok = issue_slab(g);
+            cp_async_commit();
+        }
+        for (int g = 0; g < nslab && ok; ++g) {
+            cp_async_wait<NSTAGE - 2>();
+            __syncthreads();                           // slab g has landed; everyone is past slab g - 1, whose stage is free
+            if (g + NSTAGE - 1 < nslab) ok = issue_slab(g + NSTAGE - 1);
+            cp_async_commit();
+            if (!ok) break;
+            if (source(g >> 2).dir == 0) gm.multiply(cd, g % NSTAGE); else gm.multiply(rt, g % NSTAGE);
+        }
+        cp_async_wait<0>();
+        __syncthreads();
+        if (!ok) break;
+
+        // ---- 2. Y = X + Rt + Cd, C = Cd; diagonal blocks of the factors (strict triangles, zero elsewhere)
+        {
+            const int ty = tid >> 4, tx = tid & 15;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int r = ty * 4 + i, c = tx * 4 + j, gr = row0 + r, gc = col0 + c;
+                    const float x = (gr < p.m && gc < p.n) ? (float)__ldg(p.X + (long)gr * p.ldx + gc) : 0.f;
+                    Cs[r * LDT + c] = cd[i][j];
+                    Ys[r * LDT + c] = (x + rt[i][j]) + cd[i][j];
+                }
+            if (tid < 2 * TS) ebuf[tid] = 0.f;
+            for (int e = tid; e < TS * TS; e += THREADS) {
+                const int r = e >> 6, c = e & 63;
+                const int gr = row0 + r, gcl = row0 + c;       // L block: rows / columns of the row range
+                Ld[r * LDT + c] = (c < r && gr < p.m) ? p.L32[(long)gr * p.ldl + gcl] : 0.f;
+                const int ur = col0 + r, uc = col0 + c;        // U block: rows / columns of the column range
+                Ud[r * LDT + c] = (c > r && uc < p.n) ? p.U32[(long)ur * p.ldu + uc] : 0.f;
+            }
+        }
+        __syncthreads();
+
+        // ---- 3. Algorithm 3 on the tile: 127 anti-diagonals.  Thread group `row` (4 lanes) owns row `row`.
+        {
+            const int row = tid >> 2, sub = tid & 3;
+            float *yrow = Ys + row * LDT, *crow = Cs + row * LDT;
+            const float *lrow = Ld + row * LDT;
+            unsigned long long badkey = ~0ull;
+            for (int s = 0; s < 2 * TS - 1; ++s) {
+                float *eb = ebuf + (s & 1) * TS;
+                const int j = s - row;                      // this row's entry on anti-diagonal s, if 0 <= j < 64
+                const bool active = j >= 0 && j < TS;
+                float cfold = 0.f;
+                if (active) {
+                    // every lane of the group computes the entry (same values); lane 0 publishes and stores
+                    const float y = yrow[j];
+                    const float z = rintf(y);
+                    const float e = z - y;                  // E = Z - Y
+                    cfold = crow[j] + e;                    // fold, L_ii = 1
+                    if (sub == 0) {
+                        eb[row] = e;
+                        const int gr = row0 + row, gc = col0 + j;
+                        if (gr < p.m && gc < p.n) {
+                            if (!(fabsf(y) < 2147483648.f)) {
+                                const unsigned long long key = ((unsigned long long)(gr + gc) << 42) |
+                                                               ((isfinite(y) ? 1ull : 0ull) << 41) |
+                                                               ((unsigned long long)gr << 20) | (unsigned long long)gc;
+                                if (key < badkey) badkey = key;
+                                p.Z[(long)gr * p.ldz + gc] = 0;
+                            } else {
+                                p.Z[(long)gr * p.ldz + gc] = (int)z;
+                            }
+                            if (p.Euser) p.Euser[(long)gr * p.lde + gc] = (double)e;
+                            max_abs_e = fmax(max_abs_e, (double)fabsf(e));
+                        }
+                    }
+                }
+                __syncwarp();
+                if (active && sub == 0) { yrow[j] = eb[row]; crow[j] = cfold; }     // E where Y was, final C = (L E)_ij
+                __syncthreads();
+                // downward pushes INTO this row from the sources i' < row of this anti-diagonal: lane `sub` takes
+                // i' = lo + sub, lo + sub + 4, ...  All loads of a batch are issued before the first store, so the
+                // chain of a step is one shared-memory round trip, not one per source (targets are distinct columns).
+                const int lo = max(0, s - (TS - 1)), hi = min(min(TS - 1, s), row - 1);
+#pragma unroll
+                for (int k0 = 0; k0 < TS / 4; k0 += 8) {
+                    if (lo + 4 * k0 > hi) break;                    // (uniform over the 4 lanes up to the last batch)
+                    float lv[8], ev[8], cv[8], yv[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const int ip = lo + sub + 4 * (k0 + k);
+                        const bool v = ip <= hi;
+                        const int ic = v ? ip : lo, c = s - ic;
+                        lv[k] = v ? lrow[ic] : 0.f;
+                        ev[k] = eb[ic];
+                        cv[k] = crow[c];
+                        yv[k] = yrow[c];
+                    }
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const int ip = lo + sub + 4 * (k0 + k);
+                        if (ip <= hi) {
+                            const float mm = lv[k] * ev[k];
+                            crow[s - ip] = cv[k] + mm;
+                            yrow[s - ip] = yv[k] + mm;
+                        }
+                    }
+                }
+                __syncwarp();
+                // rightward push OF this row's entry (its C is final)
+                if (active) {
+                    const float *urow = Ud + j * LDT;
+#pragma unroll
+                    for (int k0 = 0; k0 < TS / 4; k0 += 8) {
+                        if (j + 1 + 4 * k0 >= TS) break;
+                        float uv[8], yv[8];
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const int c = j + 1 + sub + 4 * (k0 + k);
+                            const int cc = c < TS ? c : TS - 1;
+                            uv[k] = urow[cc];
+                            yv[k] = yrow[cc];
+                        }
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const int c = j + 1 + sub + 4 * (k0 + k);
+                            if (c < TS) yrow[c] = fmaf(cfold, uv[k], yv[k]);
+                        }
+                    }
+                }
+                __syncwarp();
+            }
+            if (badkey != ~0ull) atomicMin(&s_badkey, badkey);
+        }
+        __syncthreads();
+
+        // ---- 4. results of the tile: E and C to the workspace, then the flag
+        for (int e = tid; e < TS * TS; e += THREADS) {
+            const int r = e >> 6, c = e & 63;
+            const long at = (long)(row0 + r) * p.np + col0 + c;
+            p.E32[at] = Ys[r * LDT + c];
+            p.C32[at] = Cs[r * LDT + c];
+        }
+        __syncthreads();
+        if (tid == 0) {
+            __threadfence();
+            st_release_u32(p.flags + (long)I * p.ntj + J, 1u);
+            if (s_badkey != ~0ull) {
+                const unsigned long long k = s_badkey;
+                report(p.info, ((k >> 41) & 1ull) ? GPTQ2D_ERR_INT_OVERFLOW : GPTQ2D_ERR_NONFINITE,
+                       (int)((k >> 20) & 0x1fffffull), (int)(k & 0xfffffull), 0);
+                s_badkey = ~0ull;
+            }
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) max_abs_e = fmax(max_abs_e, __shfl_xor_sync(0xffffffffu, max_abs_e, o));
+    if ((tid & 31) == 0) s_red[tid >> 5] = max_abs_e;
+    __syncthreads();
+    if (tid == 0) {
+        double v = 0.0;
+        for (int w = 0; w < THREADS / 32; ++w) v = fmax(v, s_red[w]);
+        if (v > 0.0) atomic_max_nonneg_double(p.max_abs_e, v);
+    }
+}
+
+// fp64 matrix -> fp32 copy with a leading dimension padded to a multiple of 4 (16-byte rows for cp.async)
+__global__ void narrow_kernel(float *dst, long ldd, const double *src, long lds, int rows, int cols) {
+    const long total = (long)rows * ldd;
+    for (long idx = (long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long)gridDim.x * blockDim.x) {
+        const long r = idx / ldd;
+        const int c = (int)(idx - r * ldd);
+        dst[idx] = c < cols ? (float)src[r * lds + c] : 0.f;
+    }
+}
+
+static size_t pad256(size_t x) { return (x + 255) / 256 * 256; }
+struct Layout {
+    int nti, ntj;
+    long mp, np, ldl, ldu;
+    size_t flags_off, l_off, u_off, e_off, c_off, total;
+};
+static Layout layout(int m, int n) {
+    Layout l;
+    l.nti = (m + TS - 1) / TS; l.ntj = (n + TS - 1) / TS;
+    l.mp = (long)l.nti * TS; l.np = (long)l.ntj * TS;
+    l.ldl = ((long)m + 3) / 4 * 4; l.ldu = ((long)n + 3) / 4 * 4;
+    l.flags_off = 256;
+    l.l_off = l.flags_off + pad256((size_t)l.nti * l.ntj * sizeof(unsigned));
+    l.u_off = l.l_off + pad256((size_t)m * l.ldl * sizeof(float));
+    l.e_off = l.u_off + pad256((size_t)n * l.ldu * sizeof(float));
+    l.c_off = l.e_off + pad256((size_t)l.mp * l.np * sizeof(float));
+    l.total = l.c_off + pad256((size_t)l.mp * l.np * sizeof(float));
+    return l;
+}
+
+}  // namespace f32
+
+size_t round_tiled_f32_workspace_bytes(int m, int n) { return f32::layout(m, n).total; }
+
+int launch_round_tiled_f32(const TiledParams &in, void *ws, size_t ws_bytes, cudaStream_t stream) {
+    using namespace f32;
+    const Layout l = layout(in.m, in.n);
+    if (ws_bytes < l.total) return GPTQ2D_ERR_WORKSPACE;
+    char *w = static_cast<char *>(ws);
+    Params p{};
+    p.m = in.m; p.n = in.n; p.nti = l.nti; p.ntj = l.ntj; p.ntiles = l.nti * l.ntj;
+    p.mp = l.mp; p.np = l.np;
+    p.X = in.X; p.ldx = in.ldx; p.Z = in.Z; p.ldz = in.ldz; p.Euser = in.E; p.lde = in.lde;
+    float *L32 = reinterpret_cast<float *>(w + l.l_off), *U32 = reinterpret_cast<float *>(w + l.u_off);
+    p.L32 = L32; p.ldl = l.ldl; p.U32 = U32; p.ldu = l.ldu;
+    p.E32 = reinterpret_cast<float *>(w + l.e_off);
+    p.C32 = reinterpret_cast<float *>(w + l.c_off);
+    p.counter = reinterpret_cast<unsigned *>(w);
+    p.abort = reinterpret_cast<unsigned *>(w) + 1;
+    p.flags = reinterpret_cast<unsigned *>(w + l.flags_off);
+    p.max_abs_e = workspace_max_abs_e(ws);
+    p.info = in.info;
+    p.spin_limit = SPIN_LIMIT;
+    if (cudaMemsetAsync(w, 0, l.l_off, stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;      // header and flags
+    int dev = 0, sms = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+    narrow_kernel<<<sms * 4, 256, 0, stream>>>(L32, l.ldl, in.L, in.ldl, in.m, in.m);
+    narrow_kernel<<<sms * 4, 256, 0, stream>>>(U32, l.ldu, in.U, in.ldu, in.n, in.n);
+    if (cudaGetLastError() != cudaSuccess) return GPTQ2D_ERR_CUDA;
+    if (cudaFuncSetAttribute(round_tiled_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
+        return GPTQ2D_ERR_CUDA;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, round_tiled_f32_kernel, THREADS, SMEM_BYTES) != cudaSuccess ||
+        per_sm < 1)
+        return GPTQ2D_ERR_CUDA;
+    if (per_sm > 2) per_sm = 2;
+    int grid = sms * per_sm;
+    if (grid > p.ntiles) grid = p.ntiles;
+    void *args[] = {&p};
+    if (cudaLaunchCooperativeKernel((const void *)round_tiled_f32_kernel, dim3(grid), dim3(THREADS), args, SMEM_BYTES, stream) !=
+        cudaSuccess)
+        return GPTQ2D_ERR_CUDA;
+    return GPTQ2D_OK;
+}
+
+}  // namespace gptq2d

@@ -16,7 +16,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libgptq2d.so")
 
-FP64, FP32, FP64_UNTILED, FP64_PULL = 0, 1, 2, 3
+FP64, FP32, FP64_UNTILED, FP64_PULL, FP32_UNTILED = 0, 1, 2, 3, 4
 
 OK = 0
 STATUS_NAMES = {
@@ -36,7 +36,7 @@ EXPORTS = (
     "gptq2d_round_f32in_workspace_bytes", "gptq2d_round_f32in",
     "gptq2d_round_blocked_workspace_bytes", "gptq2d_round_blocked",
     "gptq2d_factor_batched_workspace_bytes", "gptq2d_factor_batched",
-    "gptq2d_internal_test_hook",
+    "gptq2d_internal_test_hook", "gptq2d_internal_gemm",
 )
 FACTOR_SMALL_MAX = 128
 
@@ -99,6 +99,8 @@ def _load():
     lib.gptq2d_objective.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, sz, vp, vp]
     lib.gptq2d_round_static.restype = i32
     lib.gptq2d_round_static.argtypes = [i32, i32, vp, lng, vp, lng, vp, lng, vp, lng, vp, lng, vp, vp, vp]
+    lib.gptq2d_internal_gemm.restype = i32
+    lib.gptq2d_internal_gemm.argtypes = [i32, i32, i32, i32, i32, c.c_double, vp, lng, vp, lng, c.c_double, vp, lng, vp]
     lib.gptq2d_internal_test_hook.restype = i32
     lib.gptq2d_internal_test_hook.argtypes = [i32, lng]
     lib.gptq2d_round_static_max_dim.restype = sz
@@ -412,6 +414,21 @@ def gptq2d_internal_test_hook(key, value):
     st = _lib.gptq2d_internal_test_hook(int(key), int(value))
     if st != OK:
         raise Gptq2dError(st)
+
+
+def gptq2d_internal_gemm(A, B, C, transa=False, transb=False, alpha=1.0, beta=0.0, stream=None):
+    """C = alpha op(A) op(B) + beta C through the library's own fp64 product (2-D CUDA float64 tensors,
+    unit inner stride).  Returns C."""
+    M, N = C.shape
+    K = A.shape[0] if transa else A.shape[1]
+    pA, lda = _mat(A, torch.float64, "A")
+    pB, ldb = _mat(B, torch.float64, "B")
+    pC, ldc = _mat(C, torch.float64, "C")
+    st = _lib.gptq2d_internal_gemm(int(transa), int(transb), M, N, K, float(alpha), pA, lda, pB, ldb, float(beta),
+                                   pC, ldc, _stream_ptr(stream))
+    if st != OK:
+        raise Gptq2dError(st)
+    return C
 
 
 def gptq2d_round_static_max_dim():

@@ -382,3 +382,36 @@ def test_reverse_order_is_the_forward_order_on_the_index_reversed_problem(m, n, 
     assert abs(margin - rev["margin"]) < 1e-10 and np.max(np.abs(E - rev["E"])) < 1e-9
     bad = rev["Z"].copy(); bad[m // 2, n // 2] += 1
     assert O.certificate_margin_reverse(X, bad, Lr, Ur)[0] < 0
+
+
+def test_fp32_statement_of_algorithm_3_is_pinned_to_the_fp64_trajectory():
+    """The single-precision restatement of Algorithm 3 (the reference of the fp32 mode): where every pre-rounding
+    value is far from a tie (margin >> fp32 error) it must land on the fp64 trajectory, which the brute force and
+    the explicit Kronecker definition pin; with exactly representable data (dyadic factors, quarter-integer X) the
+    fp32 arithmetic is exact and E must agree to the last bit; A = B = I reduces to round-to-nearest."""
+    found = 0
+    for seed in range(40):
+        X, A, B = W.general_bases(14, 11, seed)
+        L, U, _, _ = O.feedback_factors(A, B)
+        ref = O.sweep_gptq2d(X, L, U)
+        if ref["margin"] < 2e-3:
+            continue
+        got = O.sweep_gptq2d_fp32(X, L, U)
+        assert np.array_equal(got["Z"], ref["Z"]), seed
+        assert np.max(np.abs(got["E"].astype(np.float64) - ref["E"])) < 2e-4
+        assert got["E"].dtype == np.float32
+        found += 1
+    assert found >= 5
+    rng = np.random.default_rng(3)
+    m, n = 9, 12
+    L = np.tril(rng.integers(-2, 3, size=(m, m)) / 4.0, -1) + np.eye(m)
+    U = np.triu(rng.integers(-2, 3, size=(n, n)) / 4.0, 1) + np.eye(n)
+    X = rng.integers(-40, 41, size=(m, n)) / 4.0 + 0.125          # never a tie: every Y is an odd multiple of 1/8 ... 1/2^k
+    ref = O.sweep_gptq2d(X, L, U)
+    got = O.sweep_gptq2d_fp32(X, L, U)
+    if ref["margin"] > 1e-6:                                        # exact dyadic arithmetic in both precisions
+        assert np.array_equal(got["Z"], ref["Z"])
+        assert np.array_equal(got["E"].astype(np.float64), ref["E"])
+    Xr = rng.standard_normal((6, 7)) * 5
+    got = O.sweep_gptq2d_fp32(Xr, np.eye(6), np.eye(7))
+    assert np.array_equal(got["Z"], np.rint(Xr.astype(np.float32)).astype(np.int64))
