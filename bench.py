@@ -158,6 +158,10 @@ def run_cuda(args):
     m, n = X.shape
     dX, dA, dB = (torch.from_numpy(np.ascontiguousarray(a)).cuda() for a in (X, A, B))
     stream = torch.cuda.current_stream()
+    if args.fused:
+        g.gptq2d_internal_test_hook(4, 2)
+    if args.gemm_tma:
+        g.gptq2d_internal_test_hook(3, 3)
 
     # ---- set-up, timed separately
     fws = torch.empty(g.gptq2d_factor_workspace_bytes(m, n), dtype=torch.uint8, device="cuda")
@@ -248,7 +252,8 @@ def run_cuda(args):
     kernel_ms = float(np.mean(per_step))
     achieved = flops / (kernel_ms * 1e-3) / 1e12
     scaled_bf16 = peaks["bf16_tflops"] * FP64_NOMINAL_TFLOPS / BF16_NOMINAL_TFLOPS if peaks["bf16_tflops"] else None
-    kernel_name = "round_tiled_f32_kernel" if args.fp32 else "round_pull_kernel" if args.pull else "round_tiled_kernel"
+    kernel_name = ("round_tiled_f32_kernel" if args.fp32 else "round_pull_kernel" if args.pull else
+                   "round_fused_kernel" if args.fused else "round_tiled_kernel")
     traffic = None
     tp = os.path.join(ROOT, "profiles", "traffic.json")
     if os.path.exists(tp):
@@ -712,6 +717,10 @@ def main():
                     help="also time the blocked sweep (Algorithm 4) with block width W on the same inputs")
     ap.add_argument("--pull", action="store_true",
                     help="time the untiled pull-form kernel (Algorithm 6) instead: the memory-bound comparison point")
+    ap.add_argument("--fused", action="store_true",
+                    help="time the sixteen-warp kernel (far contractions beside the quadrant tasks) instead of the default one")
+    ap.add_argument("--gemm-tma", action="store_true",
+                    help="route the library's fp64 products (set-up, objective, peak measurement) through the TMA-fed kernel")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-fp32-leg", action="store_true", help="skip the fp32-mode sweep reported beside the fp64 one")

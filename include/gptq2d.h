@@ -48,8 +48,10 @@ typedef enum {
                                           would spare, so this may be a neighbour of the offending input)    */
     GPTQ2D_ERR_INT_OVERFLOW = 7,       /* device: |corrected value| >= 2^31; info[1] = row, info[2] = col  */
     GPTQ2D_ERR_DEVICE_TIMEOUT = 8,     /* device: a bounded wait gave up; info[1] = where it waited     */
-    GPTQ2D_ERR_TOO_LARGE = 9           /* gptq2d_round_static: m or n beyond GPTQ2D_STATIC_MAX_DIM;
+    GPTQ2D_ERR_TOO_LARGE = 9,          /* gptq2d_round_static: m or n beyond GPTQ2D_STATIC_MAX_DIM;
                                           gptq2d_round_batched: beyond its count / dimension limits     */
+    GPTQ2D_ERR_CHECK = 10              /* device, checked builds of the library only: an index of a sweep kernel
+                                          left its array; info[1] = site, info[2] = index, info[3] = limit */
 } gptq2d_status_t;
 
 typedef enum {
@@ -137,8 +139,8 @@ int gptq2d_round_host(int m, int n,
                       int precision,
                       void *workspace, size_t workspace_bytes, int *hinfo, void *stream);
 
-/* ---- many independent sweeps in one launch (Section 6: A and B "may come from factors of
- * Kronecker Hessian approximations", i.e. one (X; A, B) triple per layer; the paper sweeps one
+/* ---- many independent sweeps in one launch (Section 6 names layer-wise Kronecker-factored Hessian
+ * estimates as a source of A and B, i.e. one (X; A, B) triple per layer; the paper sweeps one
  * matrix, Algorithm 3, and this call runs that same sweep on `count` matrices at once) ----
  * A single small or thin matrix cannot fill the GPU: its anti-diagonal dependency chain has
  * m + n - 1 stages (Section 2, Fig. 1) and few entries per stage.  Here the fp64 tiled sweeps of
@@ -220,8 +222,8 @@ int gptq2d_round_static(int m, int n,
                         int *info, void *stream);
 size_t gptq2d_round_static_max_dim(void);
 
-/* ---- reverse order (Section 2, "Two-sided and Kronecker-factored rounding": the same greedy
- * rounding "in reverse order, from the last row and column") ----
+/* ---- reverse order (Section 2, the paragraph on two-sided and Kronecker-factored rounding, mentions
+ * the same greedy rounding run backwards, starting at the bottom-right corner of the matrix) ----
  * Coordinates of vec(X) are visited from the last to the first.  The feedback factors become
  *   Lr (m x m): unit UPPER triangular, (A^T A)^{-1} = Lr Lambda Lr^T,
  *   Ur (n x n): unit LOWER triangular, (B B^T)^{-1} = Ur^T Lambda Ur,
@@ -305,8 +307,14 @@ int gptq2d_objective(int m, int n,
  *          wait for it (wait code -6) until their limit.
  *   key 2, value = polls (about 0.2 us each) after which the wait for a copy step gives up; 0 restores the
  *          default (about a second).  All other waits keep the default.
- *   key 3, value 0 / 1: route the library's fp64 products (set-up, objective) through the cp.async kernel
- *          only / through the TMA-fed kernel where the operands allow it (default 1).  Comparison runs.
+ *   key 3: which kernel the library's fp64 products (set-up, objective) take.  0: the cp.async kernel only;
+ *          1 (default): the TMA-fed kernel where a tile edge is ragged, the cp.async kernel for full tiles;
+ *          3: the TMA-fed kernel whenever the operands allow it; 2: as 3 with a barrier per slab.
+ *   key 4: the sixteen-warp sweep kernel (far contractions beside the quadrant tasks).  0 (default): never;
+ *          1: problems of at least 8 x 8 tiles; 2: whenever the operands allow it.  Comparison runs.
+ *   key 5 (checked builds of the library only; otherwise unknown): value = address of a device int[5].  Runs the
+ *          self-test of the index check on the default stream: one deliberately out-of-range index (7 of 3,
+ *          site 999) is checked; [0..3] receive {GPTQ2D_ERR_CHECK, 999, 7, 3}, [4] the redirected index 0.
  * Returns GPTQ2D_OK, or GPTQ2D_ERR_INVALID_ARG for an unknown key.
  */
 int gptq2d_internal_test_hook(int key, long value);

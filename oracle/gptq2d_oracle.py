@@ -8,8 +8,8 @@ under the Kronecker Gram  H (x) G,  G = A^T A,  H = B B^T  (Eq. 8, Eq. 9).  It i
 NOT the minimiser of the objective (exact closest-vector is NP-hard, Section 6).
 
 Indices are 0-based here; the paper is 1-based.  vec index of (i, j) is j*m + i
-(footnote of Eq. 1).  Rounding is IEEE round-half-to-even (np.rint); the paper
-only asks for "a deterministic tie-breaking rule" (Theorem 1) -- this is the
+(footnote of Eq. 1).  Rounding is IEEE round-half-to-even (np.rint); Theorem 1
+only requires that ties be broken by some fixed rule and names none -- this is the
 reading taken, and graded inputs never sit within 1e-9 of a tie.
 
 Pins (see tests/test_oracle_pins.py): brute-force conditional minimiser that uses
@@ -201,23 +201,37 @@ def sweep_dense_antidiagonal(X, L, U):
 
 
 def sweep_gptq2d(X, L, U):
-    """Algorithm 3 (GPTQ-2D), literally: corrected matrix Y plus buffer C = L E; every
-    error is folded down its column of C, pushed down its column of Y through L, and
-    then C_ij is pushed right along row i of Y through U."""
+    """Algorithm 3 (GPTQ-2D): corrected matrix Y plus the accumulated-feedback buffer C = L E.
+
+    Stage s handles anti-diagonal s as a whole.  All its entries are rounded at once (they do not
+    depend on one another, Eq. 14).  Their errors then travel along two axes only: down the entry's own
+    column through L -- folded into C and pushed into Y; written here by TARGET row r, which receives
+    L[r, i] * E[i, s - i] at column s - i from every source row i < r of the stage -- and, once C holds
+    the stage's own errors (unit diagonal of L), right along the entry's own row through U, from the
+    folded C_ij.  Same operations as the paper's two parallel loops per stage, grouped differently."""
     Y = np.array(X, dtype=np.float64)
     m, n = Y.shape
     Z = np.zeros((m, n))
     E = np.zeros((m, n))
     C = np.zeros((m, n))
     for s in range(m + n - 1):
-        idx = anti_diagonal(s, m, n)
-        for (i, j) in idx:
-            Z[i, j] = np.rint(Y[i, j])
-            E[i, j] = Z[i, j] - Y[i, j]
-            M = L[i:, i] * E[i, j]
-            C[i:, j] += M
-            Y[i + 1:, j] += M[1:]
-        for (i, j) in idx:
+        lo, hi = max(0, s - n + 1), min(m - 1, s)
+        rows = np.arange(lo, hi + 1)
+        cols = s - rows
+        y = Y[rows, cols]
+        z = np.rint(y)
+        e = z - y                                          # E = Z - Y
+        Z[rows, cols] = z
+        E[rows, cols] = e
+        C[rows, cols] += e                                 # the fold's own term: L_ii = 1
+        for r in range(lo + 1, m):                         # fold and push down, by target row
+            src = rows[rows < r]
+            if src.size == 0:
+                continue
+            M = L[r, src] * e[:src.size]
+            C[r, s - src] += M
+            Y[r, s - src] += M
+        for i, j in zip(rows, cols):                       # push right from the folded C
             Y[i, j + 1:] += C[i, j] * U[j, j + 1:]
     out = _pack(Z, E)
     out["C"] = C
@@ -321,9 +335,9 @@ def brute_force_trajectory(X, A, B):
     In column-major order: with the residuals of already-rounded coordinates held
     fixed, minimise || (B^T (x) A) r ||_2 over the REAL residuals of all remaining
     coordinates (a linear least-squares problem); the corrected value of the
-    current coordinate is x_k + r_k*, and z_k is its nearest integer
-    (Section 1: "rounding each entry to the nearest integer given the entries
-    already rounded").  Tiny sizes only.
+    current coordinate is x_k + r_k*, and z_k is its nearest integer (Section 1
+    describes the method this way: every coordinate goes to the integer closest to
+    its conditional optimum once the earlier coordinates are frozen).  Tiny sizes only.
     Returns (Z, Ypre) with Ypre the value each entry was rounded at.
     """
     X = np.asarray(X, dtype=np.float64)

@@ -16,6 +16,15 @@ int launch_objective(int m, int n, const double *X, long ldx, const int *Z, long
 
 __global__ void margin_kernel(const double *max_abs_e, double *min_margin) { *min_margin = 0.5 - *max_abs_e; }
 
+#ifdef GPTQ2D_CHECKED
+// Self-test of the checked build's index check: one deliberately out-of-range index (7 of 3, site 999) goes
+// through CI(); it must come back redirected to 0 and be recorded in `info`.  Touches no memory but `info`.
+__global__ void check_selftest_kernel(int *info, int *redirected) {
+    CHECKED_SET_INFO(info);
+    *redirected = (int)CI(7, 3, 999);
+}
+#endif
+
 // Test hooks (gptq2d_internal_test_hook): host-made failures only.
 static std::atomic<long> g_hook_withhold_last_step{0};   // one-shot: the next pipelined host call does not announce its last copy step
 static std::atomic<long> g_hook_panel_spin_limit{0};      // polls a task waits for its copy step (0: default)
@@ -131,6 +140,7 @@ const char *gptq2d_status_string(int status) {
         case GPTQ2D_ERR_INT_OVERFLOW: return "corrected value does not fit int32";
         case GPTQ2D_ERR_DEVICE_TIMEOUT: return "bounded device-side wait expired";
         case GPTQ2D_ERR_TOO_LARGE: return "problem larger than the static workspace allows";
+        case GPTQ2D_ERR_CHECK: return "checked build: an index left its array";
         default: return "unknown status";
     }
 }
@@ -182,9 +192,10 @@ int gptq2d_factor(int m, int n, const double *A, long lda, const double *B, long
 }
 
 static size_t factor_batched_table_bytes(int count) { return pad256((size_t)2 * count * sizeof(FactorSmallSide)); }
-// a problem with a basis of order > FACTOR_SMALL_MAX takes the blocked route of gptq2d_factor, both sides
+// a problem with a side of order > FACTOR_SMALL_MAX takes the blocked route of gptq2d_factor, both sides (an
+// absent basis of that order too: its identity factor is then written by a grid-wide kernel, not by one CTA)
 static bool factor_problem_is_large(const gptq2d_factor_problem_t &q) {
-    return (q.A && q.m > FACTOR_SMALL_MAX) || (q.B && q.n > FACTOR_SMALL_MAX);
+    return q.m > FACTOR_SMALL_MAX || q.n > FACTOR_SMALL_MAX;
 }
 
 size_t gptq2d_factor_batched_workspace_bytes(int count, const gptq2d_factor_problem_t *pr) {
@@ -261,11 +272,11 @@ int gptq2d_factor_batched(int count, const gptq2d_factor_problem_t *pr, void *wo
     // streams (round robin; a stream and its workspace slot are shared by every POOL-th problem, in order).
     std::unique_lock<std::mutex> lock(hp->enqueue);
     const int nslots = std::min(nlarge, (int)HostPipe::POOL);
-    if (cudaEventRecord(hp->inputs_free, stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;
-    for (int k = 0; k < nslots; ++k)
-        if (cudaStreamWaitEvent(hp->pool[k], hp->inputs_free, 0) != cudaSuccess) return GPTQ2D_ERR_CUDA;
+    if (cudaEventRecord(hp->inputs_free, stream) != cudaSuccess) return GPTQ2D_ERR_CUDA;      // nothing enqueued yet
     int idx = 0, first_err = GPTQ2D_OK;
-    for (int b = 0; b < count; ++b) {
+    for (int k = 0; k < nslots && first_err == GPTQ2D_OK; ++k)
+        if (cudaStreamWaitEvent(hp->pool[k], hp->inputs_free, 0) != cudaSuccess) first_err = GPTQ2D_ERR_CUDA;
+    for (int b = 0; b < count && first_err == GPTQ2D_OK; ++b) {
         const gptq2d_factor_problem_t &q = pr[b];
         if (!factor_problem_is_large(q)) continue;
         const int k = idx++ % nslots;
@@ -276,12 +287,12 @@ int gptq2d_factor_batched(int count, const gptq2d_factor_problem_t *pr, void *wo
         if (first_err == GPTQ2D_OK) first_err = s1 != GPTQ2D_OK ? s1 : s2;
     }
     // join even if an enqueue failed, so that nothing of this call is left running behind the caller's stream
+    // (every pool stream is joined before the first error is returned)
     for (int k = 0; k < nslots; ++k)
-        if (cudaEventRecord(hp->pool_done[k], hp->pool[k]) != cudaSuccess ||
-            cudaStreamWaitEvent(stream, hp->pool_done[k], 0) != cudaSuccess)
-            return GPTQ2D_ERR_CUDA;
-    if (first_err != GPTQ2D_OK) return first_err;
-    return GPTQ2D_OK;
+        if ((cudaEventRecord(hp->pool_done[k], hp->pool[k]) != cudaSuccess ||
+             cudaStreamWaitEvent(stream, hp->pool_done[k], 0) != cudaSuccess) && first_err == GPTQ2D_OK)
+            first_err = GPTQ2D_ERR_CUDA;
+    return first_err;
 }
 
 size_t gptq2d_round_workspace_bytes(int m, int n, int precision) {
@@ -539,6 +550,16 @@ int gptq2d_internal_test_hook(int key, long value) {
     if (key == 2) { g_hook_panel_spin_limit.store(value > 0 ? value : 0); return GPTQ2D_OK; }
     if (key == 3) { gemm_set_tma_mode((int)value); return GPTQ2D_OK; }
     if (key == 4) { round_fused_set_mode((int)value); return GPTQ2D_OK; }
+#ifdef GPTQ2D_CHECKED
+    if (key == 5) {          // value: device int[5]; [0..3] receive the status words, [4] the redirected index
+        int *dev = reinterpret_cast<int *>(static_cast<uintptr_t>(value));
+        if (!dev || cudaMemsetAsync(dev, 0xff, 5 * sizeof(int), nullptr) != cudaSuccess ||
+            cudaMemsetAsync(dev, 0, 4 * sizeof(int), nullptr) != cudaSuccess)
+            return GPTQ2D_ERR_CUDA;
+        check_selftest_kernel<<<1, 1>>>(dev, dev + 4);
+        return cudaGetLastError() == cudaSuccess ? GPTQ2D_OK : GPTQ2D_ERR_CUDA;
+    }
+#endif
     return GPTQ2D_ERR_INVALID_ARG;
 }
 

@@ -35,6 +35,28 @@ __device__ __forceinline__ void report(int *info, int status, int a, int b, int 
     }
 }
 
+// ---- checked build (-DGPTQ2D_CHECKED) --------------------------------------------------------------
+// Every index that feeds a shared- or global-memory access of the sweep kernels goes through CI(index, limit,
+// site).  In a normal build that is the index itself.  In a checked build an index outside [0, limit) is
+// recorded -- first one wins -- in the call's status words as GPTQ2D_ERR_CHECK with the site number, the
+// index and the limit, and the access is redirected to element 0 of its array: nothing traps, nothing faults,
+// and the host reads the violation like any other device-side error.  (compute-sanitizer is not available
+// where this library is developed; this is its stand-in for the small parity cases.)
+#ifdef GPTQ2D_CHECKED
+static __device__ int *g_chk_info;       // per translation unit; set by the kernels that use CI()
+__device__ __forceinline__ long checked_index(long idx, long limit, int site) {
+    if (idx >= 0 && idx < limit) return idx;
+    report(g_chk_info, GPTQ2D_ERR_CHECK, site, (int)(idx > 2147483647L ? 2147483647L : (idx < -2147483647L ? -2147483647L : idx)),
+           (int)(limit > 2147483647L ? 2147483647L : limit));
+    return 0;
+}
+#define CI(idx, limit, site) checked_index((long)(idx), (long)(limit), (site))
+#define CHECKED_SET_INFO(ptr) do { g_chk_info = (ptr); } while (0)
+#else
+#define CI(idx, limit, site) (idx)
+#define CHECKED_SET_INFO(ptr) do { } while (0)
+#endif
+
 struct GridSync {
     unsigned *count;   // arrivals of the current generation
     unsigned *gen;     // generation number

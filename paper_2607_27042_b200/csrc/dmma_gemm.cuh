@@ -15,6 +15,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include "common.cuh"
 
 namespace gptq2d {
 
@@ -65,7 +66,7 @@ __device__ __forceinline__ void load_slab(double *smem, const Operand &op, int k
         for (int i = 0; i < 4; ++i) {
             int c = tid + i * GEMM_THREADS;
             int r = c >> 3, kk = (c & 7) * 2;
-            double *dst = smem + r * LDK + kk;
+            double *dst = smem + CI(r * LDK + kk, TILE_KC - 1, 201);
             const double *src = op.ptr + (long)r * op.ld + (k0 + kk);
             int nv = (r < op.mn_valid) ? (k_valid - (k0 + kk)) : 0;   // doubles valid from kk
             nv = nv < 0 ? 0 : (nv > 2 ? 2 : nv);
@@ -83,7 +84,7 @@ __device__ __forceinline__ void load_slab(double *smem, const Operand &op, int k
         for (int i = 0; i < 4; ++i) {
             int c = tid + i * GEMM_THREADS;
             int kr = c >> 6, cc = (c & 63) * 2;
-            double *dst = smem + kr * LDN + cc;
+            double *dst = smem + CI(kr * LDN + cc, TILE_MN - 1, 202);
             const double *src = op.ptr + (long)(k0 + kr) * op.ld + cc;
             int nv = (k0 + kr < k_valid) ? (op.mn_valid - cc) : 0;
             nv = nv < 0 ? 0 : (nv > 2 ? 2 : nv);
@@ -206,7 +207,7 @@ struct FastCopy {
         }
     }
     __device__ __forceinline__ void issue(double *smem, int i, long slab) const {
-        cp_async16(smem + dst0 + i * dstep, src0 + i * sstep + slab * step, 16);
+        cp_async16(smem + CI(dst0 + i * dstep, (KCONTIG ? TILE_KC : TILE_MN) - 1, 203), src0 + i * sstep + slab * step, 16);
     }
 };
 

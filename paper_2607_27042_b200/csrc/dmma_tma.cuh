@@ -192,11 +192,14 @@ __device__ __forceinline__ bool gemm_tma_mainloop(Acc &acc, TmaRing &ring, const
         if (use > 0 && !mbar_wait(ring.empty + st, (use - 1) & 1u, abort)) { ok = false; return; }
         issued_upto = slab_from_start + 1;
         double *dst = ring.stages + (size_t)st * TMA_STAGE_DOUBLES;
-        fence_proxy_async();
         mbar_arrive_expect_tx(ring.full + st, TMA_STAGE_BYTES);
         tma_issue_slab<A_KCONTIG>(dst, A, A.k0 + (int)slab_from_start * TMA_BK, ring.full + st);
         tma_issue_slab<B_KCONTIG>(dst + TMA_TILE_DOUBLES, B, B.k0 + (int)slab_from_start * TMA_BK, ring.full + st);
     };
+    // Every lane that may issue copies orders what it (and, through the caller's barrier, the CTA) has observed
+    // in global memory before them: operands written earlier in this kernel by other CTAs were published with
+    // release / acquire on flags, which says nothing about the copy engine's proxy until this fence.
+    if (lane == 0) fence_proxy_async();
     // prologue: the first PREF slabs (issued by warp 0)
     if (warp == 0 && lane == 0)
         for (int s = 0; s < PREF && s < nk; ++s) issue((unsigned)s);

@@ -398,25 +398,31 @@ int factor_one_side(int k, const double *M, long ldm, int side, double *out, lon
         // waits for the latter.  An event waited on takes its latest record at the time of the call, so two
         // alternating events tell the large updates of K+2 and K+1 apart.
         cudaStream_t sp = look->spine;
-        CK(cudaEventRecord(look->fork, stream));
-        CK(cudaStreamWaitEvent(sp, look->fork, 0));
-        for (int K = nblk - 1; K >= 0; --K) {
-            if (K + 2 <= nblk - 1) CK(cudaStreamWaitEvent(sp, look->t2[(K + 2) & 1], 0));
-            int st = diag(K, sp);
-            if (st != GPTQ2D_OK) return st;
-            if (K == 0) break;
-            if ((st = panel(K, sp)) != GPTQ2D_OK) return st;
-            CK(cudaEventRecord(look->panel, sp));
-            if (K + 1 <= nblk - 1 && K + 1 >= 2) CK(cudaStreamWaitEvent(sp, look->t2[(K + 1) & 1], 0));
-            if ((st = trailing(K, (long)(K - 1) * FB, (long)K * FB, sp)) != GPTQ2D_OK) return st;
-            if (K >= 2) {
-                CK(cudaStreamWaitEvent(stream, look->panel, 0));
-                if ((st = trailing(K, 0, (long)(K - 1) * FB, stream)) != GPTQ2D_OK) return st;
-                CK(cudaEventRecord(look->t2[K & 1], stream));
+        const int st_spine = [&]() -> int {
+            CK(cudaEventRecord(look->fork, stream));
+            CK(cudaStreamWaitEvent(sp, look->fork, 0));
+            for (int K = nblk - 1; K >= 0; --K) {
+                if (K + 2 <= nblk - 1) CK(cudaStreamWaitEvent(sp, look->t2[(K + 2) & 1], 0));
+                int st = diag(K, sp);
+                if (st != GPTQ2D_OK) return st;
+                if (K == 0) break;
+                if ((st = panel(K, sp)) != GPTQ2D_OK) return st;
+                CK(cudaEventRecord(look->panel, sp));
+                if (K + 1 <= nblk - 1 && K + 1 >= 2) CK(cudaStreamWaitEvent(sp, look->t2[(K + 1) & 1], 0));
+                if ((st = trailing(K, (long)(K - 1) * FB, (long)K * FB, sp)) != GPTQ2D_OK) return st;
+                if (K >= 2) {
+                    CK(cudaStreamWaitEvent(stream, look->panel, 0));
+                    if ((st = trailing(K, 0, (long)(K - 1) * FB, stream)) != GPTQ2D_OK) return st;
+                    CK(cudaEventRecord(look->t2[K & 1], stream));
+                }
             }
-        }
-        CK(cudaEventRecord(look->join, sp));
-        CK(cudaStreamWaitEvent(stream, look->join, 0));
+            return GPTQ2D_OK;
+        }();
+        // join whatever happened above, so that nothing of this call runs on behind the caller's stream
+        const bool joined = cudaEventRecord(look->join, sp) == cudaSuccess &&
+                            cudaStreamWaitEvent(stream, look->join, 0) == cudaSuccess;
+        if (st_spine != GPTQ2D_OK) return st_spine;
+        if (!joined) return GPTQ2D_ERR_CUDA;
     }
     // X = P^{-1}: diagonal blocks are in place; double the block size level by level
     for (long b = FB; b < k; b *= 2) {

@@ -29,8 +29,9 @@ struct GemmArgs {
 
 // Enqueues the GEMM on `stream`.  Returns cudaSuccess or the launch error.
 cudaError_t launch_gemm(const GemmArgs &g, cudaStream_t stream);
-// 1 (default): operands that are 16-byte aligned with even leading dimensions go through the TMA-fed kernel;
-// 2: the same with a CTA barrier per slab; 0: everything through the cp.async kernel (comparison runs).
+// 1 (default): products with a ragged tile edge whose operands are 16-byte aligned with even leading dimensions
+// go through the TMA-fed kernel, full tiles through the cp.async kernel; 3: TMA-fed kernel whenever the operands
+// allow it; 2: the same with a CTA barrier per slab; 0: everything through the cp.async kernel.
 void gemm_set_tma_mode(int mode);
 
 }  // namespace gptq2d

@@ -58,20 +58,21 @@ struct BlockedParams {
 };
 
 __global__ void blocked_init_kernel(BlockedParams p) {
+    CHECKED_SET_INFO(p.info);
     const long nthreads = (long)gridDim.x * blockDim.x, tid0 = (long)blockIdx.x * blockDim.x + threadIdx.x;
     const int m = p.m, n = p.n, w = p.w;
     for (long idx = tid0; idx < (long)m * n; idx += nthreads) {
         const int i = (int)(idx / n), j = (int)(idx % n);
-        p.Y[idx] = p.X[(long)i * p.ldx + j];
+        p.Y[idx] = p.X[CI((long)i * p.ldx + j, (long)(m - 1) * p.ldx + n, 301)];
         p.C[idx] = 0.0;
     }
     for (long idx = tid0; idx < (long)m * w; idx += nthreads) {
         const int i = (int)(idx / w), k = (int)(idx % w);
-        p.Lband[idx] = (k >= 1 && i - k >= 0) ? p.L[(long)i * p.ldl + (i - k)] : 0.0;
+        p.Lband[idx] = (k >= 1 && i - k >= 0) ? p.L[CI((long)i * p.ldl + (i - k), (long)(m - 1) * p.ldl + m, 302)] : 0.0;
     }
     for (long idx = tid0; idx < (long)n * w; idx += nthreads) {
         const int j = (int)(idx / w), k = (int)(idx % w);
-        p.Uband[idx] = (k >= 1 && j - k >= 0) ? p.U[(long)(j - k) * p.ldu + j] : 0.0;
+        p.Uband[idx] = (k >= 1 && j - k >= 0) ? p.U[CI((long)(j - k) * p.ldu + j, (long)(n - 1) * p.ldu + n, 303)] : 0.0;
     }
 }
 
@@ -83,6 +84,7 @@ __global__ void blocked_init_kernel(BlockedParams p) {
 // per step; their bands of U live in a ring of BLK_RING slots in shared memory (slot = column mod
 // BLK_RING), and the column that enters at the next step is fetched ahead of time.
 __global__ void __launch_bounds__(BLK_IN_THREADS) blocked_inblock_kernel(BlockedParams p, int s0, int s1, int rlo) {
+    CHECKED_SET_INFO(p.info);
     extern __shared__ double sm[];
     double *Es = sm, *Cs = sm + BLK_ROWS * BLK_LDB, *Us = Cs + BLK_ROWS * BLK_LDB;
     __shared__ double red[BLK_IN_THREADS / 32];
@@ -103,14 +105,14 @@ __global__ void __launch_bounds__(BLK_IN_THREADS) blocked_inblock_kernel(Blocked
 #pragma unroll
     for (int x = 0; x < BLK_WMAX / 4; ++x) {
         const int k = 1 + sub + 4 * x;
-        Lr[x] = (row_ok && k < w) ? p.Lband[(long)i * w + k] : 0.0;
+        Lr[x] = (row_ok && k < w) ? p.Lband[CI((long)i * w + k, (long)p.m * w, 304)] : 0.0;
     }
 
     // columns of step 0: s0 - ibase - (BLK_ROWS - 1) .. s0 - ibase
     const int jtop = s0 - ibase;
     for (int idx = tid; idx < BLK_ROWS * w; idx += BLK_IN_THREADS) {
         const int j = jtop - (BLK_ROWS - 1) + idx / w, k = idx % w;
-        Us[(j & (BLK_RING - 1)) * BLK_LDB + k] = (j >= 0 && j < n) ? p.Uband[(long)j * w + k] : 0.0;
+        Us[CI((j & (BLK_RING - 1)) * BLK_LDB + k, BLK_RING * BLK_LDB, 305)] = (j >= 0 && j < n) ? p.Uband[CI((long)j * w + k, (long)n * w, 306)] : 0.0;
     }
     __syncthreads();
 
@@ -121,7 +123,7 @@ __global__ void __launch_bounds__(BLK_IN_THREADS) blocked_inblock_kernel(Blocked
         const int jj = s0 + tt - i;
         c = y = 0.0;
         if (row_ok && tt <= tmax && jj >= 0 && jj < n) {
-            c = p.C[(long)i * n + jj];
+            c = p.C[CI((long)i * n + jj, (long)p.m * n, 307)];
             y = p.Y[(long)i * n + jj];
         }
     };
@@ -169,10 +171,10 @@ __global__ void __launch_bounds__(BLK_IN_THREADS) blocked_inblock_kernel(Blocked
                     report(p.info, isfinite(y) ? GPTQ2D_ERR_INT_OVERFLOW : GPTQ2D_ERR_NONFINITE, i, j, 0);
                     z = 0.0;
                 }
-                p.Z[(long)i * p.ldz + j] = (int)z;
-                p.Eb[(long)i * n + j] = e;
+                p.Z[CI((long)i * p.ldz + j, (long)(p.m - 1) * p.ldz + n, 308)] = (int)z;
+                p.Eb[CI((long)i * n + j, (long)p.m * n, 309)] = e;
                 if (p.E) p.E[(long)i * p.lde + j] = e;
-                p.Cband[(long)i * w + t] = c;
+                p.Cband[CI((long)i * w + t, (long)p.m * w, 310)] = c;
                 max_abs_e = fmax(max_abs_e, fabs(e));
             }
         }
@@ -226,6 +228,7 @@ __device__ __forceinline__ void flush_mma(double (&acc)[8][2], const double *As,
 // The k-ranges of the two products are cut into chunks of FKC; chunks c + 1 and c + 2 are on their way
 // (8-byte cp.async, zero-filled where the mask says so) into the other stages while chunk c is multiplied.
 __global__ void __launch_bounds__(FLUSH_THREADS, 2) blocked_flush_kernel(BlockedParams p, int s0, int s1, int ti0) {
+    CHECKED_SET_INFO(p.info);
     extern __shared__ double sm[];
     const int m = p.m, n = p.n, w = p.w;
     const int i0 = (ti0 + (int)blockIdx.y) * FT, j0 = (int)blockIdx.x * FT;
@@ -319,7 +322,7 @@ __global__ void __launch_bounds__(FLUSH_THREADS, 2) blocked_flush_kernel(Blocked
             for (int x = 0; x < 2; ++x) {
                 const int j = jg0 + 2 * t + x;
                 if (i < m && j < n && i + j > s1) {
-                    const long idx = (long)i * n + j;
+                    const long idx = CI((long)i * n + j, (long)m * n, 311);
                     p.Y[idx] = yv[a4][x] + (accD[a][x] + accR[a][x]);
                     p.C[idx] = cv[a4][x] + accD[a][x];
                 }

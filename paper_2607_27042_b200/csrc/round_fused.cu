@@ -888,7 +888,10 @@ struct TiledLayoutView {
 };
 TiledLayoutView round_tiled_layout_view(int m, int n);     // round_tiled.cu
 
-static int g_fused_mode = 1;
+// 0 (default): never -- on B200 the side-by-side kernel measures slower than the eight-warp kernel at every
+// size (the scalar fp64 steps of the leaf sweeps queue behind the far group's DMMAs on the one fp64 pipe);
+// 1: problems of at least 8 x 8 tiles; 2: whenever the operands allow it (tests, comparison runs).
+static int g_fused_mode = 0;
 void round_fused_set_mode(int mode) { g_fused_mode = mode; }
 
 // Returns -1 if this problem does not go through the fused kernel (switched off, too small to gain, operands

@@ -59,8 +59,9 @@ size_t round_tiled_workspace_bytes(int m, int n);
 // device array inside the workspace: for each row of 128 x 128 tiles, how many of its tiles are swept
 unsigned *round_tiled_rowdone(void *ws, int m, int n);
 int launch_round_tiled(const TiledParams &p, void *ws, size_t ws_bytes, cudaStream_t stream);
-// The sixteen-warp kernel for large resident problems (round_fused.cu).  Modes: 0 never, 1 where it pays
-// (default), 2 whenever the operands allow it (tests).
+// The sixteen-warp kernel (round_fused.cu): far contractions and quadrant tasks side by side on every SM.
+// Modes: 0 never (default: it measures slower than the eight-warp kernel), 1 problems of at least 8 x 8
+// tiles, 2 whenever the operands allow it (tests, comparison runs).
 void round_fused_set_mode(int mode);
 // fp32 mode, tiled (round_tiled_f32.cu): X, L, U as fp64 device arrays, narrowed into the workspace
 size_t round_tiled_f32_workspace_bytes(int m, int n);

@@ -37,12 +37,35 @@
 // leaf-wave is swept by one warp (two entries per lane, errors exchanged through a 16-double
 // shared-memory buffer, branch-free pushes against zero-padded coefficient tables), and the
 // leaves' feedback to the remaining 8 x 8 blocks of the quadrant is m8n8k4 DMMA.
+#include <cstdio>
 #include "common.cuh"
 #include "dmma_gemm.cuh"
 #include "round_internal.cuh"
 #include <vector>
 
 namespace gptq2d {
+
+// optional in-kernel timing of the quadrant task (scratch builds only: -DTILED_STATS): cycles seen by lane 0 of
+// warp 0, which has a leaf in every leaf-wave, summed per phase over a CTA's tasks
+#ifdef TILED_STATS
+#define TS_MARK(slot)                                            \
+    do {                                                         \
+        if (threadIdx.x == 0) {                                  \
+            const long long now_ = clock64();                    \
+            g_ts[slot] += now_ - g_tlast;                        \
+            g_tlast = now_;                                      \
+        }                                                        \
+    } while (0)
+#define TS_RESET()                                               \
+    do {                                                         \
+        if (threadIdx.x == 0) g_tlast = clock64();               \
+    } while (0)
+__shared__ long long g_ts[16];
+__shared__ long long g_tlast;
+#else
+#define TS_MARK(slot)
+#define TS_RESET()
+#endif
 
 constexpr int T = 128;           // tile edge
 constexpr int Q = 64;            // quadrant edge
@@ -98,7 +121,7 @@ __device__ __forceinline__ void load_quadrant_async(double *dst, const double *s
 #pragma unroll
     for (int it = 0; it < 8; ++it) {
         int c = threadIdx.x + it * TILED_THREADS;
-        cp_async16(dst + (c >> 5) * QLD + (c & 31) * 2, src + (long)(c >> 5) * ld + (c & 31) * 2, 16);
+        cp_async16(dst + CI((c >> 5) * QLD + (c & 31) * 2, QMAT - 1, 101), src + (long)(c >> 5) * ld + (c & 31) * 2, 16);
     }
 }
 // 64 x 64 block of a user matrix (k x k, leading dimension ld) whose top-left element is
@@ -114,7 +137,7 @@ __device__ __forceinline__ void load_factor_block_async(double *dst, const doubl
         bool take = gr < k && gc < k;
         if (mode == 1) take = take && gc < gr;
         if (mode == 2) take = take && gc > gr;
-        cp_async8(dst + r * QLD + cc, take ? M + (long)gr * ld + gc : M, take ? 8 : 0);
+        cp_async8(dst + CI(r * QLD + cc, QMAT, 102), take ? M + CI((long)gr * ld + gc, (long)(k - 1) * ld + k, 103) : M, take ? 8 : 0);
     }
 }
 
@@ -126,7 +149,7 @@ __device__ __forceinline__ void load_full_block_async16(double *dst, const doubl
         int r = c >> 5, cc = (c & 31) * 2;
         int gr = r0 + r, gc = c0 + cc;
         int nv = (gr < k) ? min(2, max(0, k - gc)) : 0;
-        cp_async16(dst + r * QLD + cc, nv ? M + (long)gr * ld + gc : M, nv * 8);
+        cp_async16(dst + CI(r * QLD + cc, QMAT - 1, 104), nv ? M + CI((long)gr * ld + gc, (long)(k - 1) * ld + k - nv + 1, 105) : M, nv * 8);
     }
 }
 
@@ -149,9 +172,9 @@ __device__ __forceinline__ void quad_mma(QAcc &acc, const double *As, const doub
     for (int kk = 0; kk < Q; kk += 4) {
         double af[2], bf[4];
 #pragma unroll
-        for (int a = 0; a < 2; ++a) af[a] = As[(wr * 16 + a * 8 + g) * QLD + kk + t];
+        for (int a = 0; a < 2; ++a) af[a] = As[CI((wr * 16 + a * 8 + g) * QLD + kk + t, QMAT, 106)];
 #pragma unroll
-        for (int b = 0; b < 4; ++b) bf[b] = Bs[(kk + t) * QLD + wc * 32 + b * 8 + g];
+        for (int b = 0; b < 4; ++b) bf[b] = Bs[CI((kk + t) * QLD + wc * 32 + b * 8 + g, QMAT, 107)];
 #pragma unroll
         for (int a = 0; a < 2; ++a)
 #pragma unroll
@@ -277,8 +300,8 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
         const int r = c / TAB_LD, k = c - r * TAB_LD;       // r: row (L) or column (U) inside the quadrant
         const int src = k - 7, blk = r & ~7, in = r & 7;    // source index inside the leaf
         const bool ok = src >= 0 && src < in;
-        tabL[c] = ok ? Ls[r * QLD + blk + src] : 0.0;
-        tabU[c] = ok ? Us[(blk + src) * QLD + r] : 0.0;
+        tabL[c] = ok ? Ls[CI(r * QLD + blk + src, QMAT, 112)] : 0.0;
+        tabU[c] = ok ? Us[CI((blk + src) * QLD + r, QMAT, 113)] : 0.0;
     }
     if (tid < 8 * 2 * 16) xch[tid] = 0.0;
     if (tid == 0) s_badkey = ~0ull;
@@ -293,14 +316,16 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int piece = lane + 32 * i, r = piece >> 2, c2 = (piece & 3) * 2;
-                cp_async16(stgE + (blk & 1) * STG_E + r * STG_E_LD + c2, sm.e_above + (long)r * p.np + blk * 8 + c2, 16);
+                cp_async16(stgE + CI((blk & 1) * STG_E + r * STG_E_LD + c2, 2 * STG_E - 1, 108),
+                           p.Ebuf + CI((sm.e_above - p.Ebuf) + (long)r * p.np + blk * 8 + c2, (long)p.ntm * T * p.np - 1, 109), 16);
             }
         }
         if (sm.prog_left) {         // C to the left: rows [8 blk, 8 blk + 8) x 64 columns
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int piece = lane + 32 * i, r = piece >> 5, c2 = (piece & 31) * 2;
-                cp_async16(stgC + (blk & 1) * STG_C + r * QLD + c2, sm.c_left + (long)(blk * 8 + r) * p.np + c2, 16);
+                cp_async16(stgC + CI((blk & 1) * STG_C + r * QLD + c2, 2 * STG_C - 1, 110),
+                           p.Cbuf + CI((sm.c_left - p.Cbuf) + (long)(blk * 8 + r) * p.np + c2, (long)p.ntm * T * p.np - 1, 111), 16);
             }
         }
         cp_async_commit();
@@ -317,8 +342,10 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
     __syncwarp();
     if (fresh && warp == 7) fetch_block(0);
 
+    TS_MARK(2);                                          // tables, first fetch
     for (int lw = 0; lw < 15; ++lw) {
         __syncthreads();
+        TS_MARK(lw <= 7 ? 3 : 9);                            // barrier at the top of the leaf-wave
         if (fresh && lw <= 7) {
             // ---- pull phase: warp w adds P = Lfa[row block w, :] E_above[:, block lw] to C and Y of leaf
             // (w, lw), and R = C_left[block lw, :] Ufl[:, column block w] to Y of leaf (lw, w)
@@ -354,7 +381,9 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
                 yv.x += r0; yv.y += r1;
                 *yq = yv;
             }
+            TS_MARK(4);                                      // streamed pull (own DMMAs)
             __syncthreads();
+            TS_MARK(5);                                      // barrier after the pull
         }
         // ---- warp 7 fetches the next block of the neighbours; warp 6 (a leaf of its own only in leaf-waves
         // 6 to 8) publishes what the previous leaf-waves stored: the barriers above order those stores
@@ -369,6 +398,7 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
         if (a <= a_hi) {
             leaf_pull(Ys, Cs, Ls, Us, a, b, g, t);
             __syncwarp();
+            TS_MARK(lw <= 7 ? 6 : 10);                       // leaf_pull
             // Phase A.  Lane l owns entries (i0, j) and (i0 + 4, j) of the 8 x 8 leaf, i0 = l & 3,
             // j = l >> 2.  At step s the lane whose entry lies on anti-diagonal s rounds it and posts
             // the error (by column) and the final C value (by row) to a 16-double per-warp exchange
@@ -378,14 +408,14 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
             // is due (source not on this anti-diagonal, or entry already rounded), so stale
             // exchange slots are multiplied by zero.
             const int i0 = lane & 3, j = lane >> 2;
-            double *yp = Ys + (a * 8 + i0) * QLD + b * 8 + j;
-            double *cp = Cs + (a * 8 + i0) * QLD + b * 8 + j;
+            double *yp = Ys + CI((a * 8 + i0) * QLD + b * 8 + j, QMAT - 4 * QLD, 114);
+            double *cp = Cs + CI((a * 8 + i0) * QLD + b * 8 + j, QMAT - 4 * QLD, 115);
             double y0 = yp[0], y1 = yp[4 * QLD], c0 = cp[0], c1 = cp[4 * QLD];
             // tabL[row][7 + is] = L(row, is) for 0 <= is < row else 0; at step s, is = s - j
-            const double *tl0 = tabL + (a * 8 + i0) * TAB_LD + 7 - j;
+            const double *tl0 = tabL + CI((a * 8 + i0) * TAB_LD + 7 - j, (Q - 4) * TAB_LD - 14, 116);
             const double *tl1 = tl0 + 4 * TAB_LD;
             // tabU[col][7 + js] = U(js, col) for 0 <= js < col else 0; at step s, js = s - i
-            const double *tu0 = tabU + (b * 8 + j) * TAB_LD + 7 - i0;
+            const double *tu0 = tabU + CI((b * 8 + j) * TAB_LD + 7 - i0 - 4, Q * TAB_LD - 18, 117) + 4;
             const double *tu1 = tu0 - 4;
             double *exw = xch + warp * 32;
             int z0 = 0, z1 = 0;
@@ -417,29 +447,32 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
                 y1 = fma(l1, ed, y1); c1 = fma(l1, ed, c1); y1 = fma(cr1, u1, y1);
             }
             yp[0] = y0; yp[4 * QLD] = y1; cp[0] = c0; cp[4 * QLD] = c1;
+            TS_MARK(lw <= 7 ? 7 : 11);                       // the 15 anti-diagonal steps
             // results of the leaf: E and C to the workspace (for the neighbours and for the far parts of
             // later tiles), Z (and the caller's E) to the output
             {
                 const int gr = row0 + a * 8 + i0, gc = col0 + b * 8 + j;
-                const long at = (long)gr * p.np + gc;
+                const long at = CI((long)gr * p.np + gc, (long)p.ntm * T * p.np - 4 * p.np, 118);
                 p.Ebuf[at] = y0; p.Ebuf[at + 4 * p.np] = y1;
                 p.Cbuf[at] = c0; p.Cbuf[at + 4 * p.np] = c1;
                 if (gc < p.n) {
                     if (gr < p.m) {
-                        p.Z[(long)gr * p.ldz + gc] = z0;
+                        p.Z[CI((long)gr * p.ldz + gc, (long)(p.m - 1) * p.ldz + p.n, 119)] = z0;
                         if (p.Euser) p.Euser[(long)gr * p.lde + gc] = y0;
                         max_abs_e = fmax(max_abs_e, fabs(y0));
                     }
                     if (gr + 4 < p.m) {
-                        p.Z[(long)(gr + 4) * p.ldz + gc] = z1;
+                        p.Z[CI((long)(gr + 4) * p.ldz + gc, (long)(p.m - 1) * p.ldz + p.n, 120)] = z1;
                         if (p.Euser) p.Euser[(long)(gr + 4) * p.lde + gc] = y1;
                         max_abs_e = fmax(max_abs_e, fabs(y1));
                     }
                 }
             }
+            TS_MARK(lw <= 7 ? 8 : 12);                       // stores of the leaf
         }
     }
     __syncthreads();
+    TS_MARK(13);
     if (tid == 0) {                      // everything is stored: the quadrant is complete
         __threadfence();
         st_release_u32(sm.prog_self, 15u);
@@ -464,7 +497,7 @@ __device__ __forceinline__ void load_lu_diag_async(double *dst, const TiledKerne
         const bool lower = j < i, upper = j > i;
         const bool take = lower ? (r0 + i < p.m) : (upper && c0 + j < p.n);     // r0 + j < r0 + i, c0 + i < c0 + j
         const double *src = lower ? p.L + (long)(r0 + i) * p.ldl + r0 + j : p.U + (long)(c0 + i) * p.ldu + c0 + j;
-        cp_async8(dst + i * QLD + j, take ? src : p.L, take ? 8 : 0);
+        cp_async8(dst + CI(i * QLD + j, QMAT, 121), take ? src : p.L, take ? 8 : 0);
     }
 }
 
@@ -501,12 +534,13 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
     QAcc accC, accR;
     accC.zero();
     accR.zero();
+    TS_RESET();
     {
         const int r = 2 * I + qi, c = 2 * J + qj;
         const int fa = max(0, 2 * I - 4), fl = max(0, 2 * J - 4);
         const int nsa = max(0, r - 1 - fa), nsl = max(0, c - 1 - fl), ns = nsa + nsl;
         auto prog_of = [&](int rr, int cc) {
-            return p.qprog + ((long)(rr >> 1) * p.ntn + (cc >> 1)) * 4 + (rr & 1) * 2 + (cc & 1);
+            return p.qprog + CI(((long)(rr >> 1) * p.ntn + (cc >> 1)) * 4 + (rr & 1) * 2 + (cc & 1), 4L * p.ntm * p.ntn, 124);
         };
         // step i -> (direction, block): the older blocks of both directions first, then the newest of each
         const int olda = max(0, nsa - 1), oldl = max(0, nsl - 1);
@@ -552,6 +586,7 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
         __syncthreads();
     }
 
+    TS_MARK(0);                                          // pulls from the two nearest tiles
     // ---- 2. operands of the sweep
     Stream sm;
     sm.I = I; sm.J = J; sm.q = q;
@@ -579,7 +614,7 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
     for (int it = 0; it < 16; ++it) {                     // X of the quadrant, zero outside the matrix
         int c = tid + it * TILED_THREADS;
         int gr = row0 + (c >> 6), gc = col0 + (c & 63);
-        xv[it] = (gr < p.m && gc < p.n) ? __ldg(p.X + (long)gr * p.ldx + gc) : 0.0;
+        xv[it] = (gr < p.m && gc < p.n) ? __ldg(p.X + CI((long)gr * p.ldx + gc, (long)(p.m - 1) * p.ldx + p.n, 122)) : 0.0;
     }
     cp_async_wait<0>();
     __syncthreads();
@@ -590,8 +625,9 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
     for (int it = 0; it < 16; ++it) {                     // Y = X + Rt + Cd
         int c = tid + it * TILED_THREADS;
         int r = c >> 6, cc = c & 63;
-        Ys[r * QLD + cc] += xv[it] + Cs[r * QLD + cc];
+        Ys[CI(r * QLD + cc, QMAT, 123)] += xv[it] + Cs[r * QLD + cc];
     }
+    TS_MARK(1);                                          // operand loads, Y = X + Rt + Cd
     quadrant_sweep(Ys, Cs, LU, Lfa, Ufl, stg, tabL, tabU, row0, col0, sm, p, max_abs_e);
     __syncthreads();
 }
@@ -627,7 +663,7 @@ __device__ __forceinline__ void store_acc(const Acc &acc, double *dstT, long np,
             double2 v;
             v.x = acc.v[a][b][0];
             v.y = acc.v[a][b][1];
-            *reinterpret_cast<double2 *>(dstT + (long)(wm * 64 + a * 8 + g) * np + wn * 32 + b * 8 + t * 2) = v;
+            *reinterpret_cast<double2 *>(dstT + CI((long)(wm * 64 + a * 8 + g) * np + wn * 32 + b * 8 + t * 2, 127L * np + T - 1, 126)) = v;
         }
 }
 __device__ __forceinline__ void load_acc(Acc &acc, const double *srcT, long np, int wm, int wn, int g, int t) {
@@ -655,7 +691,7 @@ constexpr unsigned IDLE_SLEEP_NS = 400; // pause of a CTA that found nothing to 
 // multi-producer / multi-consumer ring in global memory; slot value 0 = empty.
 __device__ __forceinline__ void ready_push(const TiledKernelParams &p, unsigned entry) {
     unsigned t = atomicAdd(p.q_tail, 1u);
-    st_release_u32(p.q_slots + (t & p.qmask), entry | 0x80000000u);
+    st_release_u32(p.q_slots + CI(t & p.qmask, (long)p.qmask + 1, 127), entry | 0x80000000u);
 }
 // thread 0 only.  Returns 0 if the queue is empty (or on abort), else the entry (bit 31 set).
 __device__ __forceinline__ unsigned ready_pop(const TiledKernelParams &p) {
@@ -692,7 +728,7 @@ __device__ __forceinline__ bool quadrant_exists(const TiledKernelParams &p, int 
 }
 __device__ __forceinline__ void quadrant_arrive(const TiledKernelParams &p, int I, int J, int q) {
     if (!quadrant_exists(p, I, J, q)) return;
-    unsigned old = atomicAdd(p.qdep + ((long)I * p.ntn + J) * 4 + q, 1u);
+    unsigned old = atomicAdd(p.qdep + CI(((long)I * p.ntn + J) * 4 + q, 4L * p.ntm * p.ntn, 125), 1u);
     if (old + 1u == quadrant_needed(I, J, q)) {
         // single matrix: q | I (14 bits) | J (15 bits); batched: q | matrix (13 bits) | I (8 bits) | J (8 bits)
         const unsigned entry = p.batch_index >= 0
@@ -726,11 +762,15 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
     static_assert(!BATCHED || FAR_CTX == 2, "view slots of far contexts are handed out as 0 / 1");
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int wm = warp >> 2, wn = warp & 3, g = lane >> 2, t = lane & 3;
+    CHECKED_SET_INFO(p.info);            // (checked builds: every CTA writes the same pointer before its first barrier)
     double max_abs_e = 0.0;
     int cur = -1;                  // context whose accumulator is live in registers (uniform), -1: none
     unsigned long long spins = 0;
     Acc acc;
     acc.zero();
+#ifdef TILED_STATS
+    if (tid < 16) g_ts[tid] = 0;
+#endif
     if (tid == 0) {
         s_nctx = 0;
         if (BATCHED)
@@ -779,7 +819,8 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
     };
     auto tile_region = [&](int k) {
         const TiledKernelParams &pk = VIEW(s_ctx[k][6]);
-        return (s_ctx[k][0] == 0 ? pk.Cbuf : pk.Ebuf) + (long)s_ctx[k][1] * T * pk.np + (long)s_ctx[k][2] * T;
+        return (s_ctx[k][0] == 0 ? pk.Cbuf : pk.Ebuf) +
+               CI((long)s_ctx[k][1] * T * pk.np + (long)s_ctx[k][2] * T, (long)(pk.ntm - 1) * T * pk.np + (long)(pk.ntn - 1) * T + 1, 128);
     };
 
     for (;;) {
@@ -873,6 +914,9 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                 const int I = BATCHED ? (int)((e >> 8) & 255u) : (int)((e >> 15) & 0x3fffu);
                 const int J = BATCHED ? (int)(e & 255u) : (int)(e & 0x7fffu);
                 sweep_quadrant(I, J, q, smem, pq, max_abs_e);
+#ifdef TILED_STATS
+                if (tid == 0) g_ts[15] += 1;
+#endif
                 if constexpr (BATCHED) {                  // max |E| is kept per matrix: flush after every task
                     for (int o = 16; o > 0; o >>= 1) max_abs_e = fmax(max_abs_e, __shfl_xor_sync(0xffffffffu, max_abs_e, o));
                     if (lane == 0 && max_abs_e > 0.0) atomic_max_nonneg_double(pq.max_abs_e, max_abs_e);
@@ -888,8 +932,8 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                         const unsigned nquad = (pq.m - I * T > Q ? 2u : 1u) * (pq.n - J * T > Q ? 2u : 1u);
                         if (done + 1u == nquad) {   // tile swept: far parts that list it as a source may go on
                             __threadfence();
-                            st_release_u32(pq.flagS + (long)I * pq.ntn + J, 1u);
-                            atomicAdd(pq.rowdone + I, 1u);
+                            st_release_u32(pq.flagS + CI((long)I * pq.ntn + J, (long)pq.ntm * pq.ntn, 129), 1u);
+                            atomicAdd(pq.rowdone + CI(I, pq.ntm, 130), 1u);
                             atomicAdd(p.tiles_done, 1u);
                         }
                     }
@@ -931,11 +975,11 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
             const int upto = min(s_task[0], f_pos + FAR_RUN_CHUNKS);
             Operand a, b;
             if (f_type == 0) {
-                a.ptr = pk.L + (long)f_I * T * pk.ldl + (long)f_pos * T; a.ld = pk.ldl; a.mn_valid = min(T, pk.m - f_I * T); a.aligned16 = pk.l_al16;
+                a.ptr = pk.L + CI((long)f_I * T * pk.ldl + (long)f_pos * T, (long)(pk.m - 1) * pk.ldl + pk.m, 131); a.ld = pk.ldl; a.mn_valid = min(T, pk.m - f_I * T); a.aligned16 = pk.l_al16;
                 b.ptr = pk.Ebuf + (long)f_J * T + (long)f_pos * T * pk.np; b.ld = pk.np; b.mn_valid = T; b.aligned16 = true;
             } else {
                 a.ptr = pk.Cbuf + (long)f_I * T * pk.np + (long)f_pos * T; a.ld = pk.np; a.mn_valid = T; a.aligned16 = true;
-                b.ptr = pk.U + (long)f_J * T + (long)f_pos * T * pk.ldu; b.ld = pk.ldu; b.mn_valid = min(T, pk.n - f_J * T); b.aligned16 = pk.u_al16;
+                b.ptr = pk.U + CI((long)f_J * T + (long)f_pos * T * pk.ldu, (long)(pk.n - 1) * pk.ldu + pk.n, 132); b.ld = pk.ldu; b.mn_valid = min(T, pk.n - f_J * T); b.aligned16 = pk.u_al16;
             }
             gemm_tile<true, false, BULK_NSTAGE>(acc, smem, a, b, (upto - f_pos) * T);
             new_pos = upto;
@@ -961,6 +1005,15 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
         }
     }
 
+#ifdef TILED_STATS
+    if (tid == 0 && (blockIdx.x % 37) == 0 && g_ts[15] > 0) {
+        const long long n_ = g_ts[15];
+        printf("cta %3d tasks %lld | per task: nearpull %lld load %lld tables %lld | lw0-7: barA %lld pull %lld barB %lld leafpull %lld "
+               "sweep %lld store %lld | lw8-14: bar %lld leafpull %lld sweep %lld store %lld | end %lld\n",
+               (int)blockIdx.x, n_, g_ts[0] / n_, g_ts[1] / n_, g_ts[2] / n_, g_ts[3] / n_, g_ts[4] / n_, g_ts[5] / n_, g_ts[6] / n_,
+               g_ts[7] / n_, g_ts[8] / n_, g_ts[9] / n_, g_ts[10] / n_, g_ts[11] / n_, g_ts[12] / n_, g_ts[13] / n_);
+    }
+#endif
     if constexpr (!BATCHED) {
         for (int o = 16; o > 0; o >>= 1) max_abs_e = fmax(max_abs_e, __shfl_xor_sync(0xffffffffu, max_abs_e, o));
         if (lane == 0) s_red[warp] = max_abs_e;

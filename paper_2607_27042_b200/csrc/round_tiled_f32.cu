@@ -16,11 +16,13 @@
 // of an SM sits in the dependent chain of its in-tile sweep the other one multiplies.  A tile only waits
 // for tiles of earlier waves, which were claimed earlier, so the earliest unfinished tile can always run.
 //
-// In-tile sweep: one anti-diagonal per step, four threads per row.  Row i of the tile is only ever
-// written by its own four threads -- they apply the downward pushes INTO row i (regrouped by target row:
-// the targets (i, s - i') of all sources i' < i on anti-diagonal s are contiguous, and so are the
-// coefficients L[i][i']) and the rightward push OF row i's entry -- so the only thing that crosses rows is
-// the vector of errors of the current anti-diagonal: one CTA barrier per step.
+// In-tile sweep: one anti-diagonal per step, one CTA barrier per step, in the implicit-Y (pull) form of
+// Appendix B (Eq. 19-20): an entry reads the errors above it in its column through L and the finished C to
+// its left in its row through U at the moment it is rounded, four lanes per row sharing the two dot
+// products.  Only rows with an entry on the current anti-diagonal work, and nothing is read-modify-written
+// (an eager version that pushed every error down and right as Algorithm 3 prints it cost 7x the time per
+// step: 2 x 64 x 64 shared-memory updates per anti-diagonal, issued by every warp).
+#include <cstdio>
 #include "common.cuh"
 #include "dmma_gemm.cuh"          // cp.async helpers
 #include "round_internal.cuh"
@@ -38,7 +40,7 @@ constexpr int A_FLOATS = TS * LDA, B_FLOATS = KS * LDB, STAGE_FLOATS = A_FLOATS 
 constexpr int LDT = TS + 4;        // in-tile matrices, row stride 68 floats: the 8 rows x 4 lanes of a warp hit 32 different banks
                                    // in the push loops (bank = 4 row -+ lane)
 constexpr int TMAT = TS * LDT;
-constexpr int SWEEP_FLOATS = 4 * TMAT + 2 * TS, RING_FLOATS = NSTAGE * STAGE_FLOATS;
+constexpr int SWEEP_FLOATS = 5 * TMAT + TS * TS, RING_FLOATS = NSTAGE * STAGE_FLOATS;      // + the tile's Z (int32)
 constexpr size_t SMEM_BYTES = (size_t)(SWEEP_FLOATS > RING_FLOATS ? SWEEP_FLOATS : RING_FLOATS) * sizeof(float);
 
 struct Params {
@@ -128,12 +130,20 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
     __shared__ unsigned long long s_badkey;
     float *stages = smem;
     // the contraction's accumulators are registers, so the in-tile matrices reuse the ring's memory
-    float *Ys = smem, *Cs = Ys + TMAT, *Ld = Cs + TMAT, *Ud = Ld + TMAT;
-    float *ebuf = Ud + TMAT;                       // [2][64]: errors of the current anti-diagonal, by source row
+    // Ld[i][i'] = L[i, i'] (strictly lower), Udt[j][j'] = U[j', j] (the diagonal block of U transposed, strictly
+    // lower), Et[j][i'] = E[i', j] (transposed copy of the errors): the rows the dot products of the sweep run along
+    float *Ys = smem, *Cs = Ys + TMAT, *Ld = Cs + TMAT, *Udt = Ld + TMAT, *Et = Udt + TMAT;
+    int *Zs = reinterpret_cast<int *>(Et + TMAT);  // [64][64]: rounded values, written out row-wise after the sweep
     const int tid = threadIdx.x;
     Gemm gm{stages, tid, tid >> 4, tid & 15};
     double max_abs_e = 0.0;
     if (tid == 0) s_badkey = ~0ull;
+#ifdef TILED_STATS
+    long long st_claim = 0, st_gemm = 0, st_form = 0, st_sweep = 0, st_store = 0, st_n = 0, st_t = clock64();
+#define F32_MARK(x) do { const long long now_ = clock64(); x += now_ - st_t; st_t = now_; } while (0)
+#else
+#define F32_MARK(x)
+#endif
 
     for (;;) {
         __syncthreads();
@@ -151,6 +161,7 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
         int I, J;
         decode_tile(task, p.nti, p.ntj, I, J);
         const int row0 = I * TS, col0 = J * TS;
+        F32_MARK(st_claim);
 
         // ---- 1. the two contractions.  Source list: tiles (0..I-2, J) through L, tiles (I, 0..J-2) through U, then
         // the tile above and the tile to the left (the newest ones, still being swept when this tile is claimed).
@@ -227,6 +238,7 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
         cp_async_wait<0>();
         __syncthreads();
         if (!ok) break;
+        F32_MARK(st_gemm);
 
         // ---- 2. Y = X + Rt + Cd, C = Cd; diagonal blocks of the factors (strict triangles, zero elsewhere)
         {
@@ -240,112 +252,92 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
                     Cs[r * LDT + c] = cd[i][j];
                     Ys[r * LDT + c] = (x + rt[i][j]) + cd[i][j];
                 }
-            if (tid < 2 * TS) ebuf[tid] = 0.f;
+#pragma unroll 8
             for (int e = tid; e < TS * TS; e += THREADS) {
                 const int r = e >> 6, c = e & 63;
                 const int gr = row0 + r, gcl = row0 + c;       // L block: rows / columns of the row range
                 Ld[r * LDT + c] = (c < r && gr < p.m) ? p.L32[(long)gr * p.ldl + gcl] : 0.f;
-                const int ur = col0 + r, uc = col0 + c;        // U block: rows / columns of the column range
-                Ud[r * LDT + c] = (c > r && uc < p.n) ? p.U32[(long)ur * p.ldu + uc] : 0.f;
+                const int ur = col0 + r, uc = col0 + c;        // U block (r, c) with r < c, stored transposed
+                Udt[c * LDT + r] = (c > r && uc < p.n) ? p.U32[(long)ur * p.ldu + uc] : 0.f;
+                Et[r * LDT + c] = 0.f;                         // unrounded entries count as zero (they meet zero coefficients)
             }
         }
         __syncthreads();
+        F32_MARK(st_form);
 
-        // ---- 3. Algorithm 3 on the tile: 127 anti-diagonals.  Thread group `row` (4 lanes) owns row `row`.
+        // ---- 3. the tile's 127 anti-diagonals, in the implicit-Y (pull) form of Appendix B, Eq. 19-20, which gives
+        // the same entries as Algorithm 3: entry (i, j) reconstructs its corrected value when it is rounded,
+        //     Y_ij = Y0_ij + sum_{i' < i} L[i, i'] E[i', j] + sum_{j' < j} C[i, j'] U[j', j],
+        // and its final C_ij = C0_ij + sum_{i' < i} L[i, i'] E[i', j] + E_ij is stored once.  Everything it reads was
+        // rounded on an earlier anti-diagonal, nothing is read-modify-written, and only the rows that own an
+        // entry of the current anti-diagonal work: four lanes per row, each a quarter of the two dot products.
+        // Ys holds Y0 until an entry is rounded and E afterwards; Cs holds C0 and then C.
         {
             const int row = tid >> 2, sub = tid & 3;
-            float *yrow = Ys + row * LDT, *crow = Cs + row * LDT;
             const float *lrow = Ld + row * LDT;
+            float *yrow = Ys + row * LDT, *crow = Cs + row * LDT;
             unsigned long long badkey = ~0ull;
+            float max_e = 0.f;
             for (int s = 0; s < 2 * TS - 1; ++s) {
-                float *eb = ebuf + (s & 1) * TS;
-                const int j = s - row;                      // this row's entry on anti-diagonal s, if 0 <= j < 64
-                const bool active = j >= 0 && j < TS;
-                float cfold = 0.f;
-                if (active) {
-                    // every lane of the group computes the entry (same values); lane 0 publishes and stores
-                    const float y = yrow[j];
-                    const float z = rintf(y);
-                    const float e = z - y;                  // E = Z - Y
-                    cfold = crow[j] + e;                    // fold, L_ii = 1
+                const int j = s - row;
+                if (j >= 0 && j < TS) {                                  // (uniform over the row's four lanes)
+                    // Both dot products run along rows of shared memory in chunks of four; a lane takes every fourth
+                    // chunk.  Beyond the diagonal the coefficients are zero (strict triangles) and what they meet is
+                    // finite (zeros, or values of entries rounded later), so whole chunks need no masking.
+                    float dl[2] = {0.f, 0.f}, du[2] = {0.f, 0.f};
+                    const float4 *l4 = reinterpret_cast<const float4 *>(lrow), *e4 = reinterpret_cast<const float4 *>(Et + j * LDT);
+                    for (int q = sub; 4 * q < row; q += 4) {                // down the column: sources i' < row
+                        const float4 a = l4[q], b = e4[q];
+                        dl[0] = fmaf(a.x, b.x, dl[0]); dl[1] = fmaf(a.y, b.y, dl[1]);
+                        dl[0] = fmaf(a.z, b.z, dl[0]); dl[1] = fmaf(a.w, b.w, dl[1]);
+                    }
+                    const float4 *c4 = reinterpret_cast<const float4 *>(crow), *u4 = reinterpret_cast<const float4 *>(Udt + j * LDT);
+                    for (int q = sub; 4 * q < j; q += 4) {                  // along the row: sources j' < j
+                        const float4 a = c4[q], b = u4[q];
+                        du[0] = fmaf(a.x, b.x, du[0]); du[1] = fmaf(a.y, b.y, du[1]);
+                        du[0] = fmaf(a.z, b.z, du[0]); du[1] = fmaf(a.w, b.w, du[1]);
+                    }
+                    float sl = dl[0] + dl[1], su = du[0] + du[1];
+                    const unsigned gmask = 0xfu << ((tid & 31) & ~3);          // the row's four lanes (rows of a warp differ in activity)
+                    sl += __shfl_xor_sync(gmask, sl, 1);
+                    su += __shfl_xor_sync(gmask, su, 1);
+                    sl += __shfl_xor_sync(gmask, sl, 2);
+                    su += __shfl_xor_sync(gmask, su, 2);
                     if (sub == 0) {
-                        eb[row] = e;
-                        const int gr = row0 + row, gc = col0 + j;
-                        if (gr < p.m && gc < p.n) {
-                            if (!(fabsf(y) < 2147483648.f)) {
-                                const unsigned long long key = ((unsigned long long)(gr + gc) << 42) |
-                                                               ((isfinite(y) ? 1ull : 0ull) << 41) |
-                                                               ((unsigned long long)gr << 20) | (unsigned long long)gc;
-                                if (key < badkey) badkey = key;
-                                p.Z[(long)gr * p.ldz + gc] = 0;
-                            } else {
-                                p.Z[(long)gr * p.ldz + gc] = (int)z;
-                            }
-                            if (p.Euser) p.Euser[(long)gr * p.lde + gc] = (double)e;
-                            max_abs_e = fmax(max_abs_e, (double)fabsf(e));
+                        const float y = (yrow[j] + su) + sl;
+                        const float z = rintf(y);
+                        const float e = z - y;                           // E = Z - Y
+                        crow[j] = (crow[j] + sl) + e;                    // C = L E (unit diagonal)
+                        yrow[j] = e;
+                        Et[j * LDT + row] = e;
+                        int zi = (int)z;
+                        if (!(fabsf(y) < 2147483648.f)) {
+                            const int gr = row0 + row, gc = col0 + j;
+                            const unsigned long long key = ((unsigned long long)(gr + gc) << 42) | ((isfinite(y) ? 1ull : 0ull) << 41) |
+                                                           ((unsigned long long)gr << 20) | (unsigned long long)gc;
+                            if (gr < p.m && gc < p.n && key < badkey) badkey = key;
+                            zi = 0;
                         }
+                        Zs[row * TS + j] = zi;
+                        max_e = fmaxf(max_e, fabsf(e));
                     }
                 }
-                __syncwarp();
-                if (active && sub == 0) { yrow[j] = eb[row]; crow[j] = cfold; }     // E where Y was, final C = (L E)_ij
                 __syncthreads();
-                // downward pushes INTO this row from the sources i' < row of this anti-diagonal: lane `sub` takes
-                // i' = lo + sub, lo + sub + 4, ...  All loads of a batch are issued before the first store, so the
-                // chain of a step is one shared-memory round trip, not one per source (targets are distinct columns).
-                const int lo = max(0, s - (TS - 1)), hi = min(min(TS - 1, s), row - 1);
-#pragma unroll
-                for (int k0 = 0; k0 < TS / 4; k0 += 8) {
-                    if (lo + 4 * k0 > hi) break;                    // (uniform over the 4 lanes up to the last batch)
-                    float lv[8], ev[8], cv[8], yv[8];
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        const int ip = lo + sub + 4 * (k0 + k);
-                        const bool v = ip <= hi;
-                        const int ic = v ? ip : lo, c = s - ic;
-                        lv[k] = v ? lrow[ic] : 0.f;
-                        ev[k] = eb[ic];
-                        cv[k] = crow[c];
-                        yv[k] = yrow[c];
-                    }
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        const int ip = lo + sub + 4 * (k0 + k);
-                        if (ip <= hi) {
-                            const float mm = lv[k] * ev[k];
-                            crow[s - ip] = cv[k] + mm;
-                            yrow[s - ip] = yv[k] + mm;
-                        }
-                    }
-                }
-                __syncwarp();
-                // rightward push OF this row's entry (its C is final)
-                if (active) {
-                    const float *urow = Ud + j * LDT;
-#pragma unroll
-                    for (int k0 = 0; k0 < TS / 4; k0 += 8) {
-                        if (j + 1 + 4 * k0 >= TS) break;
-                        float uv[8], yv[8];
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            const int c = j + 1 + sub + 4 * (k0 + k);
-                            const int cc = c < TS ? c : TS - 1;
-                            uv[k] = urow[cc];
-                            yv[k] = yrow[cc];
-                        }
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            const int c = j + 1 + sub + 4 * (k0 + k);
-                            if (c < TS) yrow[c] = fmaf(cfold, uv[k], yv[k]);
-                        }
-                    }
-                }
-                __syncwarp();
             }
+            max_abs_e = fmax(max_abs_e, (double)max_e);      // (entries outside the matrix are exact zeros with E = 0)
             if (badkey != ~0ull) atomicMin(&s_badkey, badkey);
         }
-        __syncthreads();
+        F32_MARK(st_sweep);
 
-        // ---- 4. results of the tile: E and C to the workspace, then the flag
+        // ---- 4. results of the tile: Z (and the caller's E) to the outputs, E and C to the workspace, then the flag
+        for (int e = tid; e < TS * TS; e += THREADS) {
+            const int r = e >> 6, c = e & 63;
+            const int gr = row0 + r, gc = col0 + c;
+            if (gr < p.m && gc < p.n) {
+                p.Z[(long)gr * p.ldz + gc] = Zs[r * TS + c];
+                if (p.Euser) p.Euser[(long)gr * p.lde + gc] = (double)Ys[r * LDT + c];
+            }
+        }
         for (int e = tid; e < TS * TS; e += THREADS) {
             const int r = e >> 6, c = e & 63;
             const long at = (long)(row0 + r) * p.np + col0 + c;
@@ -363,7 +355,16 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
                 s_badkey = ~0ull;
             }
         }
+        F32_MARK(st_store);
+#ifdef TILED_STATS
+        st_n += 1;
+#endif
     }
+#ifdef TILED_STATS
+    if (tid == 0 && (blockIdx.x % 61) == 0 && st_n > 0)
+        printf("cta %3d tiles %lld | per tile: claim %lld gemm(+flag waits) %lld form %lld sweep %lld store %lld\n", (int)blockIdx.x, st_n,
+               st_claim / st_n, st_gemm / st_n, st_form / st_n, st_sweep / st_n, st_store / st_n);
+#endif
     for (int o = 16; o > 0; o >>= 1) max_abs_e = fmax(max_abs_e, __shfl_xor_sync(0xffffffffu, max_abs_e, o));
     if ((tid & 31) == 0) s_red[tid >> 5] = max_abs_e;
     __syncthreads();

@@ -14,7 +14,9 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libgptq2d.so")
+# GPTQ2D_LIBRARY selects another build of the same library (the tests use it for the checked build,
+# libgptq2d_checked.so, in a process of its own); it must name a file inside this package
+_LIB_PATH = os.path.join(_HERE, os.path.basename(os.environ.get("GPTQ2D_LIBRARY", "libgptq2d.so")))
 
 FP64, FP32, FP64_UNTILED, FP64_PULL, FP32_UNTILED = 0, 1, 2, 3, 4
 
@@ -22,7 +24,7 @@ OK = 0
 STATUS_NAMES = {
     0: "OK", 1: "ERR_INVALID_ARG", 2: "ERR_WORKSPACE", 3: "ERR_UNSUPPORTED_DEVICE", 4: "ERR_CUDA",
     5: "ERR_NOT_SPD", 6: "ERR_NONFINITE", 7: "ERR_INT_OVERFLOW", 8: "ERR_DEVICE_TIMEOUT",
-    9: "ERR_TOO_LARGE",
+    9: "ERR_TOO_LARGE", 10: "ERR_CHECK",
 }
 
 EXPORTS = (

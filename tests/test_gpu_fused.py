@@ -1,7 +1,7 @@
 """The sixteen-warp sweep kernel (far contractions fed by TMA beside the quadrant tasks on every SM) against
-the CPU oracle.  By default it only takes problems of at least 8 x 8 tiles; the test hook forces it onto
-every shape its operands allow, so that ragged tiles, single rows / columns of tiles and matrices with no far
-part at all go through it too.  Z must be bit-exact against the oracle (nested Algorithm 5 on certified
+the CPU oracle.  It is not the default path (it measures slower than the eight-warp kernel); the test hook
+forces it onto every shape its operands allow, so that ragged tiles, single rows / columns of tiles and
+matrices with no far part at all go through it.  Z must be bit-exact against the oracle (nested Algorithm 5 on certified
 inputs), E within 1e-9, runs repeatable bit for bit, and equal in Z to the eight-warp kernel."""
 import numpy as np
 import pytest
@@ -36,7 +36,7 @@ def _run(g, X, L, U, mode):
         torch.cuda.synchronize()
         g.check_info(info)
     finally:
-        g.gptq2d_internal_test_hook(4, 1)
+        g.gptq2d_internal_test_hook(4, 0)
     return Z, E, float(mm.cpu()[0])
 
 
@@ -67,7 +67,7 @@ def test_fused_kernel_mid_size_with_library_factors(g):
         pytest.fail("no certified seed")
     dX, dA, dB = (torch.from_numpy(a).cuda() for a in (X, A, B))
     Ld, Ud, _, _, finfo = g.gptq2d_factor(dA, dB)
-    Z, E, mm = _run(g, dX, Ld, Ud, 1)                    # 10 x 12 tiles: the default dispatch takes the fused kernel
+    Z, E, mm = _run(g, dX, Ld, Ud, 2)
     g.check_info(finfo)
     Zh = Z.cpu().numpy().astype(np.int64)
     assert np.array_equal(Zh, ref["Z"])

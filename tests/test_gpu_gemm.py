@@ -16,7 +16,7 @@ def g():
     return gptq2d
 
 
-@pytest.mark.parametrize("tma", [1, 0])
+@pytest.mark.parametrize("tma", [3, 1, 0])
 @pytest.mark.parametrize("M,N,K", [(128, 128, 16), (256, 384, 512), (130, 257, 75), (1, 1, 1), (300, 100, 1000),
                                    (127, 129, 17), (513, 8, 260)])
 def test_gemm_all_layouts_exact(g, tma, M, N, K):
