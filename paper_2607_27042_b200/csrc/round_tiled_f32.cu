@@ -125,7 +125,7 @@ struct Gemm {
 __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
     extern __shared__ __align__(16) float smem[];
     __shared__ int s_task;
-    __shared__ int s_ok;
+    __shared__ int s_ok, s_upto;
     __shared__ double s_red[THREADS / 32];
     __shared__ unsigned long long s_badkey;
     float *stages = smem;
@@ -196,30 +196,42 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
             }
             return r;
         };
-        // Issues slab g (all threads).  The first slab of a source waits, bounded, for the source tile's flag;
-        // returns false if that wait ran out.
-        auto issue_slab = [&](int g) -> bool {
-            const Src sr = source(g >> 2);
-            if ((g & 3) == 0) {
-                if (tid == 0) {
-                    unsigned long long it = 0;
-                    int good = 1;
-                    while (ld_acquire_u32(sr.flag) == 0u) {
-                        if (++it > p.spin_limit || ld_relaxed_u32(p.abort) != 0u) {
-                            report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -9, task, (int)blockIdx.x);
-                            atomicExch(p.abort, 1u);
-                            good = 0;
-                            break;
-                        }
-                        __nanosleep(100);
+        // Sources [0, ready_upto) are known to be swept.  The list is scanned by the whole CTA at once (one flag per
+        // thread, the first unset position by a shared-memory minimum), so that a tile whose far sources are all
+        // done -- the usual case -- pays two barriers for the lot instead of a global round trip per source; only
+        // when the next source in line is still being swept does one thread wait for it, bounded.
+        int ready_upto = 0;
+        auto scan_ready = [&](int from) -> bool {         // all threads; false if the bounded wait ran out
+            if (tid == 0) {
+                unsigned long long it = 0;
+                int good = 1;
+                const Src sr = source(from);
+                while (ld_acquire_u32(sr.flag) == 0u) {
+                    if (++it > p.spin_limit || ld_relaxed_u32(p.abort) != 0u) {
+                        report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -9, task, (int)blockIdx.x);
+                        atomicExch(p.abort, 1u);
+                        good = 0;
+                        break;
                     }
-                    s_ok = good;
+                    __nanosleep(100);
                 }
-                __syncthreads();
-                const bool good = s_ok != 0;
-                __syncthreads();                       // s_ok may be rewritten by the next wait
-                if (!good) return false;
+                s_ok = good;
+                s_upto = nsrc;
             }
+            __syncthreads();
+            for (int k = from + 1 + tid; k < nsrc; k += THREADS)
+                if (ld_acquire_u32(source(k).flag) == 0u) atomicMin(&s_upto, k);
+            __syncthreads();
+            const bool good = s_ok != 0;
+            ready_upto = s_upto;
+            __syncthreads();                              // s_ok / s_upto may be rewritten by the next scan
+            return good;
+        };
+        // Issues slab g (all threads); returns false if a wait ran out.
+        auto issue_slab = [&](int g) -> bool {
+            const int sidx = g >> 2;
+            if (sidx >= ready_upto && !scan_ready(sidx)) return false;
+            const Src sr = source(sidx);
             gm.issue(g % NSTAGE, sr.A, sr.lda, sr.a_rows, sr.a_kmax, sr.B, sr.ldb, sr.b_cols, sr.b_kmax, (g & 3) * KS);
             return true;
         };
