@@ -7,8 +7,8 @@
 // and Algorithm 3 on the tile alone, started from Y = X[r, c] + Rt + Cd and C = Cd with the diagonal
 // blocks L[r, r] and U[c, c], gives the tile's Z, E and C = L E.  fp32 has no tensor-core path that keeps
 // fp32 operands exact (TF32 truncates them), so the two contractions are a register-tiled FFMA loop:
-// 256 threads, a 4 x 4 piece of the tile per thread and contraction, operand slabs of 16 staged through
-// shared memory with cp.async.
+// 256 threads, a 4 x 4 piece of the tile per thread and contraction, operand slabs of 32 staged through
+// shared memory with cp.async (one CTA barrier per slab: at 16 the barrier was the first stall reason).
 //
 // One persistent, cooperatively launched grid, two CTAs per SM.  Tiles are claimed wave by wave (I + J
 // ascending) from one atomic counter; a CTA folds the source tiles in as their flags come up -- the far
@@ -32,9 +32,10 @@ namespace f32 {
 
 constexpr int TS = 64;             // tile edge
 constexpr int THREADS = 256;
-constexpr int KS = 16;             // slab depth
-constexpr int NSTAGE = 6;          // cp.async ring; it lives where the in-tile matrices go afterwards
-constexpr int LDA = KS + 4;        // A slab [64 rows][16 k], row stride 20 floats: 16-byte rows, conflict-free float4 reads
+constexpr int KS = 64;             // slab depth
+constexpr int SPS = TS / KS;       // slabs per source tile
+constexpr int NSTAGE = 3;          // cp.async ring; it lives where the in-tile matrices go afterwards
+constexpr int LDA = KS + 4;        // A slab [64 rows][KS k], row stride KS + 4 floats: 16-byte rows, conflict-free float4 reads
 constexpr int LDB = TS + 4;        // B slab [16 k][64 cols], row stride 68 floats
 constexpr int A_FLOATS = TS * LDA, B_FLOATS = KS * LDB, STAGE_FLOATS = A_FLOATS + B_FLOATS;
 constexpr int LDT = TS + 4;        // in-tile matrices, row stride 68 floats: the 8 rows x 4 lanes of a warp hit 32 different banks
@@ -77,22 +78,26 @@ __device__ __forceinline__ void decode_tile(int task, int nti, int ntj, int &I, 
 
 // One source tile: acc += A (64 x 64, [row][k], leading dimension lda) * B (64 x 64, [k][col], ldb), both fully
 // inside padded or zero-filled storage except that rows of A beyond `a_rows` and columns of B beyond `b_cols`
-// (ragged edge of a user matrix) are read as zeros.  K is streamed in four slabs of 16.
+// (ragged edge of a user matrix) are read as zeros.  K is streamed in SPS slabs of KS.
 struct Gemm {
     float *stages;
     int tid, ty, tx;
-    // copy plan: A slab = 64 rows x 16 k = 256 chunks of 4 floats (one per thread); B slab = 16 k x 64 cols likewise
+    // copy plan: A slab = 64 rows x KS k, B slab = KS k x 64 columns, in chunks of 4 floats, KS / 16 of each per thread
     __device__ __forceinline__ void issue(int stage, const float *A, long lda, int a_rows, int a_kmax, const float *B, long ldb,
                                           int b_cols, int b_kmax, int k0) const {
         float *As = stages + stage * STAGE_FLOATS, *Bs = As + A_FLOATS;
-        {
-            const int r = tid >> 2, kc = (tid & 3) * 4;
+#pragma unroll
+        for (int h = 0; h < KS / 16; ++h) {               // A slab: 64 rows x KS k, chunks of 4 floats
+            const int c = tid + h * THREADS;
+            const int r = c / (KS / 4), kc = (c % (KS / 4)) * 4;
             int nv = (r < a_rows) ? a_kmax - (k0 + kc) : 0;          // floats valid from kc on
             nv = nv < 0 ? 0 : (nv > 4 ? 4 : nv);
             cp_async16f(As + r * LDA + kc, nv ? A + (long)r * lda + k0 + kc : A, nv * 4);
         }
-        {
-            const int kr = tid >> 4, cc = (tid & 15) * 4;
+#pragma unroll
+        for (int h = 0; h < KS / 16; ++h) {               // B slab: KS k x 64 columns
+            const int c = tid + h * THREADS;
+            const int kr = c >> 4, cc = (c & 15) * 4;
             int nv = (k0 + kr < b_kmax) ? b_cols - cc : 0;
             nv = nv < 0 ? 0 : (nv > 4 ? 4 : nv);
             cp_async16f(Bs + kr * LDB + cc, nv ? B + (long)(k0 + kr) * ldb + cc : B, nv * 4);
@@ -170,7 +175,7 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
         for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int j = 0; j < 4; ++j) cd[i][j] = rt[i][j] = 0.f;
-        const int nsrc = I + J, nslab = nsrc * (TS / KS);
+        const int nsrc = I + J, nslab = nsrc * SPS;
         bool ok = true;
         // slab g of the flattened list belongs to source g / 4; operands of a source (all threads compute them)
         struct Src { const float *A, *B; long lda, ldb; int a_rows, a_kmax, b_cols, b_kmax, dir; const unsigned *flag; };
@@ -229,10 +234,10 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
         };
         // Issues slab g (all threads); returns false if a wait ran out.
         auto issue_slab = [&](int g) -> bool {
-            const int sidx = g >> 2;
+            const int sidx = g / SPS;
             if (sidx >= ready_upto && !scan_ready(sidx)) return false;
             const Src sr = source(sidx);
-            gm.issue(g % NSTAGE, sr.A, sr.lda, sr.a_rows, sr.a_kmax, sr.B, sr.ldb, sr.b_cols, sr.b_kmax, (g & 3) * KS);
+            gm.issue(g % NSTAGE, sr.A, sr.lda, sr.a_rows, sr.a_kmax, sr.B, sr.ldb, sr.b_cols, sr.b_kmax, (g % SPS) * KS);
             return true;
         };
         for (int g = 0; g < NSTAGE - 1 && ok; ++g) {
@@ -245,7 +250,7 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
             if (g + NSTAGE - 1 < nslab) ok = issue_slab(g + NSTAGE - 1);
             cp_async_commit();
             if (!ok) break;
-            if (source(g >> 2).dir == 0) gm.multiply(cd, g % NSTAGE); else gm.multiply(rt, g % NSTAGE);
+            if (source(g / SPS).dir == 0) gm.multiply(cd, g % NSTAGE); else gm.multiply(rt, g % NSTAGE);
         }
         cp_async_wait<0>();
         __syncthreads();
