@@ -40,6 +40,9 @@ constexpr int Q = 64;             // quadrant edge
 constexpr int QLD = 68;           // shared-memory row stride of quadrant matrices (68 mod 16 == 4)
 constexpr int QMAT = Q * QLD;
 constexpr int TAB_LD = 24;        // row stride of the leaf coefficient tables (22 used)
+// far warps pause between slabs while the SM's quadrant group sweeps leaves: measured 42.6 ms at 8192^2 against
+// 40.5 without (the far group loses more than the chain gains), 7.9 against 10.2 ms at 4096^2; off
+constexpr bool FUSED_THROTTLE = false;
 constexpr int F_WARPS = 8;        // far warps: 2 x 2 (64 x 32 each) or 4 x 2 (32 x 32 each)
 constexpr int F_THREADS = 32 * F_WARPS;
 constexpr int F_FRAGS_M = 32 / F_WARPS;   // row fragments of a far warp
@@ -457,7 +460,7 @@ __device__ __forceinline__ void quadrant_sweep(double *Ys, double *Cs, const dou
 
 // One quadrant task (see round_tiled.cu, sweep_quadrant).  qs: the group's shared memory.
 __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *qs, double *xch, unsigned long long *s_badkey,
-                                               const FusedParams &p, double &max_abs_e, int qtid) {
+                                               const FusedParams &p, double &max_abs_e, int qtid, volatile int *qsweeping) {
     double *Ys = qs, *Cs = qs + QMAT, *LU = qs + 2 * QMAT, *AUX = qs + 3 * QMAT;
     double *tabL = AUX, *tabU = tabL + Q * TAB_LD, *stg = tabU + Q * TAB_LD;
     const int warp = qtid >> 5, lane = qtid & 31, g = lane >> 2, t = lane & 3;
@@ -570,7 +573,9 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *qs, 
         Ys[rr * QLD + cc] += Xs[rr * 64 + cc] + Cs[rr * QLD + cc];
     }
     QSYNC();                                              // Xs is dead: the tables are built over it
+    if (FUSED_THROTTLE && qtid == 0) *qsweeping = 1;
     quadrant_sweep(Ys, Cs, LU, lfa, ufl, stg, tabL, tabU, xch, s_badkey, row0, col0, sm, p, max_abs_e, qtid);
+    if (FUSED_THROTTLE && qtid == 0) *qsweeping = 0;
     QSYNC();
 }
 
@@ -614,7 +619,8 @@ struct FarRing {
 // acc += rowop[128 rows at y = row_y, k from k0] * colop[k from k0, 64 columns at x = col_x], nk slabs of 16.
 // Called by the eight far warps with uniform arguments.  Returns false if a wait ran out.
 __device__ __forceinline__ bool far_mainloop(FAcc &acc, FarRing &ring, const CUtensorMap *mapA, const CUtensorMap *mapB,
-                                             int row_y, int col_x, int k0, int nk, int warp, int lane, unsigned *abort) {
+                                             int row_y, int col_x, int k0, int nk, int warp, int lane, unsigned *abort,
+                                             const volatile int *stand_back) {
     constexpr int PREF = F_NSTAGE - 1;
     const int wm = warp >> 1, wn = warp & 1, g = lane >> 2, t = lane & 3;
     bool ok = true;
@@ -647,6 +653,13 @@ __device__ __forceinline__ bool far_mainloop(FAcc &acc, FarRing &ring, const CUt
     for (int kt = 0; kt < nk; ++kt) {
         const unsigned c = ring.slabs + (unsigned)kt;
         const unsigned st = c % F_NSTAGE, use = c / F_NSTAGE;
+        if (FUSED_THROTTLE) {
+            // The scalar fp64 steps of a leaf sweep queue behind DMMAs on the sub-partition's one fp64 pipe, so while
+            // this SM's quadrant group is inside its leaf-waves the far warps pause between slabs (bounded: the flag
+            // is cleared at the end of every quadrant task).
+            unsigned pause = 0;
+            while (*stand_back != 0 && ++pause < 200000u) __nanosleep(200);
+        }
         if (!__all_sync(0xffffffffu, mbar_wait(ring.full + st, use & 1u, abort))) { ok = false; kt_stop = kt; break; }
         const double *S = ring.stages + (size_t)st * F_STAGE_DOUBLES;
         const bool my_turn = (kt + PREF < nk) && ((kt & (F_WARPS - 1)) == warp);
@@ -706,10 +719,13 @@ round_fused_kernel(FusedParams p, const __grid_constant__ CUtensorMap mapL, cons
     __shared__ double xch[8 * 2 * 16];
     __shared__ unsigned long long s_badkey;
     __shared__ int s_ftask, s_fupto, s_fok;
+    __shared__ volatile int s_qsweeping;       // the quadrant group is inside its leaf-waves: the far group stands back
     __shared__ unsigned s_qpop;
     __shared__ int s_qstate;
     __shared__ double s_red[GROUP / 32];
     // aligned to 1024 bytes by an offset into the shared array (pointer arithmetic keeps the shared address space)
+    if (threadIdx.x == 0) s_qsweeping = 0;
+    __syncthreads();
     double *ring_mem = smem_raw + (((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u) >> 3);
     double *qs = ring_mem + F_NSTAGE * F_STAGE_DOUBLES;
     const int tid = threadIdx.x;
@@ -774,8 +790,8 @@ round_fused_kernel(FusedParams p, const __grid_constant__ CUtensorMap mapL, cons
                 if (upto < 0) { ok = false; break; }
                 STAT_T0(tm);
                 const int nk = (upto - pos) * (T / TMA_BK);
-                if (type == 0) ok = far_mainloop(acc, ring, &mapL, &mapE, I * T, J * T + h * FN, pos * T, nk, warp, lane, p.abort);
-                else ok = far_mainloop(acc, ring, &mapC, &mapU, I * T, J * T + h * FN, pos * T, nk, warp, lane, p.abort);
+                if (type == 0) ok = far_mainloop(acc, ring, &mapL, &mapE, I * T, J * T + h * FN, pos * T, nk, warp, lane, p.abort, &s_qsweeping);
+                else ok = far_mainloop(acc, ring, &mapC, &mapU, I * T, J * T + h * FN, pos * T, nk, warp, lane, p.abort, &s_qsweeping);
                 // a wait that ran out in one warp ends the far part for the whole group
                 if (!ok && lane == 0) {
                     report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -7, task, (int)blockIdx.x);
@@ -844,7 +860,7 @@ round_fused_kernel(FusedParams p, const __grid_constant__ CUtensorMap mapL, cons
         if (state != 1) break;
         const int q = (int)((e >> 29) & 3u), I = (int)((e >> 15) & 0x3fffu), J = (int)(e & 0x7fffu);
         STAT_T0(tt);
-        sweep_quadrant(I, J, q, qs, xch, &s_badkey, p, max_abs_e, qtid);
+        sweep_quadrant(I, J, q, qs, xch, &s_badkey, p, max_abs_e, qtid, &s_qsweeping);
         STAT_ADD(sq_task, tt);
 #ifdef FUSED_STATS
         sq_n += 1;
