@@ -95,7 +95,7 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *bar, unsigned pari
     }
 }
 
-// 3-D tiled copy global -> shared (own CTA), completion reported to `bar`.  No cluster multicast.
+// 3-D tiled copy global -> shared (own CTA), completion reported to `bar`.  Every CTA fetches its own copy.
 __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, int x, int y, int z, unsigned long long *bar) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];\n" ::"r"(

@@ -9,7 +9,7 @@
 // fixed roles that share nothing but the device-wide scheduler words:
 //   * warps 0-7, the FAR group: claim far parts wave by wave from one atomic counter and run them as a
 //     DMMA contraction on a 128 x 64 register accumulator, operand slabs brought in by TMA
-//     (cp.async.bulk.tensor, 128-byte swizzle, per-CTA, no multicast) through a three-stage mbarrier
+//     (cp.async.bulk.tensor, 128-byte swizzle; every CTA fetches its own copy) through a three-stage mbarrier
 //     ring.  The group synchronises only with itself (mbarriers, one named barrier per far part).
 //   * warps 8-15, the QUADRANT group: serve the ready ring; a quadrant task is the one of round_tiled.cu
 //     (pulls from the two nearest tiles, then 15 leaf-waves streamed from its two neighbours) on the

@@ -98,3 +98,18 @@ def test_fp32_mismatch_fraction_and_objective_gap_are_bounded(g, name, make):
     assert np.max(np.abs(E)) <= 0.5 + 1e-5
     o64 = O.objective(X, ref64["Z"], A, B)
     assert abs(O.objective(X, Z, A, B) - o64) <= 1e-3 * o64
+
+
+def test_fp32_ragged_multi_wave_repeatable_and_close_to_fp64(g):
+    """Many tile-waves, ragged last tiles in both directions: two runs bit-identical (the claim order differs from
+    run to run, the arithmetic must not), and the rounding stays close to the fp64 sweep of the same inputs."""
+    X, A, B = W.headline_like(1000, 1300, 17)
+    L, U, _, _ = O.feedback_factors(A, B)
+    Z1, E1, m1 = run(g, X, L, U, g.FP32)
+    Z2, E2, m2 = run(g, X, L, U, g.FP32)
+    assert np.array_equal(Z1, Z2) and np.array_equal(E1, E2) and m1 == m2
+    Z64, _, _ = run(g, X, L, U, g.FP64)
+    assert float(np.mean(Z1 != Z64)) <= 0.05
+    o64 = O.objective(X, Z64, A, B)
+    assert abs(O.objective(X, Z1, A, B) - o64) <= 1e-3 * o64
+    assert np.max(np.abs(E1)) <= 0.5 + 1e-5
