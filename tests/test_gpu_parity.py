@@ -132,6 +132,26 @@ def test_factor_triangular_shortcut_needs_no_oracle(g):
     assert np.allclose(Ld.cpu().numpy(), np.linalg.inv(A) @ np.diag(np.diag(A)), atol=1e-11)
 
 
+def test_factor_two_level_blocking_ragged(g):
+    """Orders of 16 block rows and more take the two-level route of the set-up (128-row steps inside outer blocks
+    of 512 rows, rank-512 updates above them); 2100 and 2300 give ragged last blocks at both levels and one side
+    with a last outer block of a single block row."""
+    m, n = 2100, 2177
+    X, A, B = W.general_bases(m, n, 5)
+    A = A + np.sqrt(m) * np.eye(m)
+    B = B + np.sqrt(n) * np.eye(n)
+    L, U, lamL, lamU = O.feedback_factors(A, B)
+    Ld, Ud, dL, dU, info = g.gptq2d_factor(dev(A), dev(B))
+    torch.cuda.synchronize()
+    g.check_info(info)
+    Ld, Ud = Ld.cpu().numpy(), Ud.cpu().numpy()
+    assert np.array_equal(np.diag(Ld), np.ones(m)) and np.array_equal(np.triu(Ld, 1), np.zeros((m, m)))
+    assert np.array_equal(np.diag(Ud), np.ones(n)) and np.array_equal(np.tril(Ud, -1), np.zeros((n, n)))
+    assert np.max(np.abs(Ld - L)) < 1e-10 * max(1.0, np.max(np.abs(L)))
+    assert np.max(np.abs(Ud - U)) < 1e-10 * max(1.0, np.max(np.abs(U)))
+    assert np.allclose(dL.cpu().numpy(), 1 / lamL, rtol=1e-10) and np.allclose(dU.cpu().numpy(), 1 / lamU, rtol=1e-10)
+
+
 # ------------------------------------------------------------------ mid sizes: cubic oracle + certificate
 @pytest.mark.parametrize("name,make", [
     ("c2_like", lambda s: W.llm_layer_like(384, 1408, s, samples=2048)),
