@@ -260,16 +260,29 @@ def sweep_blocked(X, L, U, w):
     for s0 in range(0, last + 1, w):
         s1 = min(s0 + w - 1, last)
         for s in range(s0, s1 + 1):
-            idx = anti_diagonal(s, m, n)
-            for (i, j) in idx:
-                Z[i, j] = np.rint(Y[i, j])
-                E[i, j] = Z[i, j] - Y[i, j]
-                end = min(s1 - j, m - 1) + 1              # rows of column j still inside the block
-                M = L[i:end, i] * E[i, j]
-                C[i:end, j] += M
-                Y[i + 1:end, j] += M[1:]
-            for (i, j) in idx:
-                end = min(s1 - i, n - 1) + 1              # columns of row i still inside the block
+            # one stage of the block, all its entries at once; the pushes stop at the block's last anti-diagonal
+            # s1: from source (i, s - i) the downward push reaches rows r with r + (s - i) <= s1, the rightward
+            # push columns c with i + c <= s1
+            lo, hi = max(0, s - n + 1), min(m - 1, s)
+            rows = np.arange(lo, hi + 1)
+            cols = s - rows
+            y = Y[rows, cols]
+            z = np.rint(y)
+            e = z - y
+            Z[rows, cols] = z
+            E[rows, cols] = e
+            C[rows, cols] += e                                  # unit diagonal of L
+            reach = s1 - s                                      # how many rows / columns a push may still travel
+            for r in range(lo + 1, min(m - 1, hi + reach) + 1):         # fold and push down, by target row
+                take = (rows < r) & (rows >= r - reach)
+                if not take.any():
+                    continue
+                src = rows[take]
+                M = L[r, src] * e[take]
+                C[r, s - src] += M
+                Y[r, s - src] += M
+            for i, j in zip(rows, cols):                        # push right from the folded C
+                end = min(s1 - i, n - 1) + 1
                 Y[i, j + 1:end] += C[i, j] * U[j, j + 1:end]
         # down flush: column j's part of the block is rows s0-j .. s1-j; everything below s1-j is later
         for j in range(n):
