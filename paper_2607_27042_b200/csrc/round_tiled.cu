@@ -62,6 +62,7 @@ namespace gptq2d {
     } while (0)
 __shared__ long long g_ts[16];
 __shared__ long long g_tlast;
+__shared__ long long g_sched[8];     // 0 quadrant tasks, 1 far main loop, 2 far park/unpark + flag scan, 3 idle, 4 looking for work, 5 far parts
 #else
 #define TS_MARK(slot)
 #define TS_RESET()
@@ -768,8 +769,14 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
     unsigned long long spins = 0;
     Acc acc;
     acc.zero();
+#ifndef TILED_STATS
+#define SC_MARK(slot)
+#endif
 #ifdef TILED_STATS
     if (tid < 16) g_ts[tid] = 0;
+    if (tid < 8) g_sched[tid] = 0;
+    long long sc_t = clock64();
+#define SC_MARK(slot) do { if (tid == 0) { const long long n_ = clock64(); g_sched[slot] += n_ - sc_t; sc_t = n_; } } while (0)
 #endif
     if (tid == 0) {
         s_nctx = 0;
@@ -890,6 +897,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
         }
         __syncthreads();
         const int state = s_state;
+        SC_MARK(4);
         if (state >= 3) break;
         if (state == 2) {
             if (++spins > p.spin_limit) {
@@ -900,6 +908,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                 break;
             }
             __nanosleep(s_nctx == 0 ? IDLE_SLEEP_NS : 100);
+            SC_MARK(3);
             continue;
         }
         spins = 0;
@@ -948,6 +957,7 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                 __syncthreads();
                 e = s_pop;
             }
+            SC_MARK(0);
             continue;
         }
 
@@ -981,7 +991,9 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
                 a.ptr = pk.Cbuf + (long)f_I * T * pk.np + (long)f_pos * T; a.ld = pk.np; a.mn_valid = T; a.aligned16 = true;
                 b.ptr = pk.U + CI((long)f_J * T + (long)f_pos * T * pk.ldu, (long)(pk.n - 1) * pk.ldu + pk.n, 132); b.ld = pk.ldu; b.mn_valid = min(T, pk.n - f_J * T); b.aligned16 = pk.u_al16;
             }
+            SC_MARK(2);
             gemm_tile<true, false, BULK_NSTAGE>(acc, smem, a, b, (upto - f_pos) * T);
+            SC_MARK(1);
             new_pos = upto;
         }
         if (new_pos >= f_nfar) {
@@ -1003,9 +1015,13 @@ __global__ void __launch_bounds__(TILED_THREADS, 1) round_tiled_kernel(TiledKern
         } else if (tid == 0) {
             s_ctx[k][3] = new_pos;
         }
+        SC_MARK(2);
     }
 
 #ifdef TILED_STATS
+    if (tid == 0 && (blockIdx.x % 37) == 0)
+        printf("cta %3d scheduler: quadrant tasks %lld far main loop %lld far park/scan %lld idle %lld looking %lld\n", (int)blockIdx.x,
+               g_sched[0], g_sched[1], g_sched[2], g_sched[3], g_sched[4]);
     if (tid == 0 && (blockIdx.x % 37) == 0 && g_ts[15] > 0) {
         const long long n_ = g_ts[15];
         printf("cta %3d tasks %lld | per task: nearpull %lld load %lld tables %lld | lw0-7: barA %lld pull %lld barB %lld leafpull %lld "

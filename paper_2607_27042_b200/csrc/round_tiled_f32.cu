@@ -7,8 +7,14 @@
 // and Algorithm 3 on the tile alone, started from Y = X[r, c] + Rt + Cd and C = Cd with the diagonal
 // blocks L[r, r] and U[c, c], gives the tile's Z, E and C = L E.  fp32 has no tensor-core path that keeps
 // fp32 operands exact (TF32 truncates them), so the two contractions are a register-tiled FFMA loop:
-// 256 threads, a 4 x 4 piece of the tile per thread and contraction, operand slabs of 32 staged through
-// shared memory with cp.async (one CTA barrier per slab: at 16 the barrier was the first stall reason).
+// 256 threads in four groups of 64; a group takes a quarter of every slab's depth and holds an 8 x 8 piece
+// of the whole 64 x 64 tile per thread (one shared-memory float per four FMAs; a 4 x 4 piece per thread
+// without the split needs twice the loads and ran at 30 % of the FMA pipe), and the four partial tiles are
+// added through shared memory when a contraction ends.  Both operands of a slab are stored depth-major
+// ([k][64 rows] and [k][64 columns]: L and C are kept transposed in the workspace for this), staged with
+// cp.async through a four-stage ring of slabs of 32.  A thread cannot hold two 8 x 8 accumulators, so a tile
+// runs three contractions one after the other: Rt over the older tiles of its row, Cd over its whole column
+// (the tile above comes last), Rt's last term from the tile to the left -- the newest sources still come last.
 //
 // One persistent, cooperatively launched grid, two CTAs per SM.  Tiles are claimed wave by wave (I + J
 // ascending) from one atomic counter; a CTA folds the source tiles in as their flags come up -- the far
@@ -31,18 +37,24 @@ namespace gptq2d {
 namespace f32 {
 
 constexpr int TS = 64;             // tile edge
-constexpr int THREADS = 256;
+constexpr int THREADS = 256;        // one CTA per SM
 constexpr int KS = 64;             // slab depth
 constexpr int SPS = TS / KS;       // slabs per source tile
-constexpr int NSTAGE = 3;          // cp.async ring; it lives where the in-tile matrices go afterwards
-constexpr int LDA = KS + 4;        // A slab [64 rows][KS k], row stride KS + 4 floats: 16-byte rows, conflict-free float4 reads
-constexpr int LDB = TS + 4;        // B slab [16 k][64 cols], row stride 68 floats
-constexpr int A_FLOATS = TS * LDA, B_FLOATS = KS * LDB, STAGE_FLOATS = A_FLOATS + B_FLOATS;
-constexpr int LDT = TS + 4;        // in-tile matrices, row stride 68 floats: the 8 rows x 4 lanes of a warp hit 32 different banks
-                                   // in the push loops (bank = 4 row -+ lane)
+constexpr int NSTAGE = 4;          // cp.async ring; it lives where the in-tile matrices go afterwards
+constexpr int KGROUPS = THREADS / 32;   // one warp a group, each KS / KGROUPS deep in every slab
+constexpr int KG = KS / KGROUPS;
+constexpr int LDB = TS + 4;        // both slabs are [KS k][64], row stride 68 floats
+constexpr int SLAB_FLOATS = KS * LDB, STAGE_FLOATS = 2 * SLAB_FLOATS;
+constexpr int PMAT = TS * LDB;     // a group's partial tile, staged with the slabs' row stride
+constexpr int RPT = TS * TS / 4 / THREADS;   // float4 pieces of a tile per thread (rows (t >> 4) + (THREADS / 16) h)
+constexpr int LDT = TS + 16;       // in-tile matrices, row stride 80 floats = 16 banks mod 32: the two rows x four lanes of a quarter-warp
+                                   // read eight different 16-byte columns of two neighbouring rows without a bank conflict
 constexpr int TMAT = TS * LDT;
-constexpr int SWEEP_FLOATS = 5 * TMAT + TS * TS, RING_FLOATS = NSTAGE * STAGE_FLOATS;      // + the tile's Z (int32)
-constexpr size_t SMEM_BYTES = (size_t)(SWEEP_FLOATS > RING_FLOATS ? SWEEP_FLOATS : RING_FLOATS) * sizeof(float);
+constexpr int SWEEP_FLOATS = 4 * TMAT + TS * TS, RING_FLOATS = NSTAGE * STAGE_FLOATS;      // + the tile's Z (int32)
+constexpr int PARK_FLOATS = 2 * TS * TS;      // finished partial sums (Rt of the older tiles, Cd) wait behind the ring
+constexpr int SMEM_FLOATS = RING_FLOATS + PARK_FLOATS > SWEEP_FLOATS ? RING_FLOATS + PARK_FLOATS : SWEEP_FLOATS;
+static_assert(KGROUPS * PMAT <= RING_FLOATS, "the four partial tiles are added through the drained ring");
+constexpr size_t SMEM_BYTES = (size_t)SMEM_FLOATS * sizeof(float);
 
 struct Params {
     int m, n, nti, ntj, ntiles;
@@ -50,9 +62,9 @@ struct Params {
     const double *X; long ldx;
     int *Z; long ldz;
     double *Euser; long lde;
-    const float *L32; long ldl;    // m x m (leading dimension padded to a multiple of 4)
+    const float *L32t; long ldl;   // L transposed, m x m: L32t[k][r] = L[r, k] (leading dimension padded to a multiple of 4)
     const float *U32; long ldu;
-    float *E32, *C32;
+    float *E32, *C32t;             // E: mp x np (leading dimension np); C transposed: np x mp (leading dimension mp)
     unsigned *counter, *abort, *flags;
     double *max_abs_e;
     int *info;
@@ -76,58 +88,64 @@ __device__ __forceinline__ void decode_tile(int task, int nti, int ntj, int &I, 
     I = J = 0;
 }
 
-// One source tile: acc += A (64 x 64, [row][k], leading dimension lda) * B (64 x 64, [k][col], ldb), both fully
-// inside padded or zero-filled storage except that rows of A beyond `a_rows` and columns of B beyond `b_cols`
-// (ragged edge of a user matrix) are read as zeros.  K is streamed in SPS slabs of KS.
+// One source tile: acc += A^T B with A (64 k x 64 rows, [k][row], leading dimension lda) and B (64 k x 64 columns,
+// [k][col], ldb), both fully inside padded or zero-filled storage except that rows of the tile beyond `a_rows`, columns
+// beyond `b_cols` and depths beyond `kmax` (ragged edge of a user matrix) are read as zeros.  K is streamed in SPS slabs.
 struct Gemm {
     float *stages;
-    int tid, ty, tx;
-    // copy plan: A slab = 64 rows x KS k, B slab = KS k x 64 columns, in chunks of 4 floats, KS / 16 of each per thread
-    __device__ __forceinline__ void issue(int stage, const float *A, long lda, int a_rows, int a_kmax, const float *B, long ldb,
-                                          int b_cols, int b_kmax, int k0) const {
-        float *As = stages + stage * STAGE_FLOATS, *Bs = As + A_FLOATS;
+    int tid, gk, ty, tx;           // group (quarter of the depth), position in the group's 8 x 8 thread grid
+    // copy plan: each slab is KS k x 64 entries in chunks of 4 floats, KS * 16 / THREADS chunks of each slab per thread
+    __device__ __forceinline__ void issue_one(float *S, const float *P, long ld, int valid, int kmax, int k0) const {
 #pragma unroll
-        for (int h = 0; h < KS / 16; ++h) {               // A slab: 64 rows x KS k, chunks of 4 floats
-            const int c = tid + h * THREADS;
-            const int r = c / (KS / 4), kc = (c % (KS / 4)) * 4;
-            int nv = (r < a_rows) ? a_kmax - (k0 + kc) : 0;          // floats valid from kc on
-            nv = nv < 0 ? 0 : (nv > 4 ? 4 : nv);
-            cp_async16f(As + r * LDA + kc, nv ? A + (long)r * lda + k0 + kc : A, nv * 4);
-        }
-#pragma unroll
-        for (int h = 0; h < KS / 16; ++h) {               // B slab: KS k x 64 columns
+        for (int h = 0; h < KS * 16 / THREADS; ++h) {
             const int c = tid + h * THREADS;
             const int kr = c >> 4, cc = (c & 15) * 4;
-            int nv = (k0 + kr < b_kmax) ? b_cols - cc : 0;
+            int nv = (k0 + kr < kmax) ? valid - cc : 0;              // floats valid from cc on
             nv = nv < 0 ? 0 : (nv > 4 ? 4 : nv);
-            cp_async16f(Bs + kr * LDB + cc, nv ? B + (long)(k0 + kr) * ldb + cc : B, nv * 4);
+            cp_async16f(S + kr * LDB + cc, nv ? P + (long)(k0 + kr) * ld + cc : P, nv * 4);
         }
     }
-    __device__ __forceinline__ void multiply(float (&acc)[4][4], int stage) const {
-        const float *As = stages + stage * STAGE_FLOATS, *Bs = As + A_FLOATS;
+    __device__ __forceinline__ void issue(int stage, const float *A, long lda, int a_rows, const float *B, long ldb, int b_cols,
+                                          int kmax, int k0) const {
+        float *As = stages + stage * STAGE_FLOATS;
+        issue_one(As, A, lda, a_rows, kmax, k0);
+        issue_one(As + SLAB_FLOATS, B, ldb, b_cols, kmax, k0);
+    }
+    // the thread's piece: rows 4 ty + (i & 3) + 16 (i >> 2), i < 16; columns 4 tx + (j & 3) + 32 (j >> 2), j < 8
+    __device__ __forceinline__ void multiply(float (&acc)[16][8], int stage) const {
+        const float *As = stages + stage * STAGE_FLOATS + gk * KG * LDB, *Bs = As + SLAB_FLOATS;
 #pragma unroll
-        for (int k4 = 0; k4 < KS; k4 += 4) {
-            float4 a[4], b[4];
+        for (int k = 0; k < KG; ++k) {
+            float av[16], bv[8];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) a[i] = *reinterpret_cast<const float4 *>(As + (ty * 4 + i) * LDA + k4);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) b[k] = *reinterpret_cast<const float4 *>(Bs + (k4 + k) * LDB + tx * 4);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float av[4] = {a[i].x, a[i].y, a[i].z, a[i].w};
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    acc[i][0] = fmaf(av[k], b[k].x, acc[i][0]);
-                    acc[i][1] = fmaf(av[k], b[k].y, acc[i][1]);
-                    acc[i][2] = fmaf(av[k], b[k].z, acc[i][2]);
-                    acc[i][3] = fmaf(av[k], b[k].w, acc[i][3]);
-                }
+            for (int h = 0; h < 4; ++h) {
+                const float4 a = *reinterpret_cast<const float4 *>(As + k * LDB + 16 * h + 4 * ty);
+                av[4 * h + 0] = a.x; av[4 * h + 1] = a.y; av[4 * h + 2] = a.z; av[4 * h + 3] = a.w;
             }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const float4 b = *reinterpret_cast<const float4 *>(Bs + k * LDB + 32 * h + 4 * tx);
+                bv[4 * h + 0] = b.x; bv[4 * h + 1] = b.y; bv[4 * h + 2] = b.z; bv[4 * h + 3] = b.w;
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+    }
+    // the group's partial tile to shared memory (row stride LDB)
+    __device__ __forceinline__ void stage_partial(const float (&acc)[16][8]) const {
+        float *P = stages + gk * PMAT;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            float *row = P + (4 * ty + (i & 3) + 16 * (i >> 2)) * LDB + 4 * tx;
+            *reinterpret_cast<float4 *>(row) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+            *reinterpret_cast<float4 *>(row + 32) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
         }
     }
 };
 
-__global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
+__global__ void __launch_bounds__(THREADS, 1) round_tiled_f32_kernel(Params p) {
     extern __shared__ __align__(16) float smem[];
     __shared__ int s_task;
     __shared__ int s_ok, s_upto;
@@ -135,16 +153,20 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
     __shared__ unsigned long long s_badkey;
     float *stages = smem;
     // the contraction's accumulators are registers, so the in-tile matrices reuse the ring's memory
-    // Ld[i][i'] = L[i, i'] (strictly lower), Udt[j][j'] = U[j', j] (the diagonal block of U transposed, strictly
-    // lower), Et[j][i'] = E[i', j] (transposed copy of the errors): the rows the dot products of the sweep run along
-    float *Ys = smem, *Cs = Ys + TMAT, *Ld = Cs + TMAT, *Udt = Ld + TMAT, *Et = Udt + TMAT;
+    // Udt[j][j'] = U[j', j] (the diagonal block of U transposed, strictly lower, first sub-diagonal apart in s_usub),
+    // Et[j][i'] = E[i', j] (transposed copy of the errors): the rows the dot products of the sweep run along.  The
+    // diagonal block of L lives in registers (a lane keeps its quarter of its row).
+    float *Ys = smem, *Cs = Ys + TMAT, *Udt = Cs + TMAT, *Et = Udt + TMAT;
     int *Zs = reinterpret_cast<int *>(Et + TMAT);  // [64][64]: rounded values, written out row-wise after the sweep
+    __shared__ float s_usub[TS];                   // U[j - 1, j] of the diagonal block
     const int tid = threadIdx.x;
-    Gemm gm{stages, tid, tid >> 4, tid & 15};
+    Gemm gm{stages, tid, tid >> 5, (tid & 31) >> 3, tid & 7};
+    float *park_rt = smem + RING_FLOATS, *park_cd = park_rt + TS * TS;     // [64][64] each, behind the ring
     double max_abs_e = 0.0;
     if (tid == 0) s_badkey = ~0ull;
 #ifdef TILED_STATS
-    long long st_claim = 0, st_gemm = 0, st_form = 0, st_sweep = 0, st_store = 0, st_n = 0, st_t = clock64();
+    long long sw_sums = 0, sw_round = 0, sw_bar = 0;
+    long long st_claim = 0, st_gemm = 0, st_form = 0, st_sweep = 0, st_store = 0, st_wait = 0, st_n = 0, st_t = clock64();
 #define F32_MARK(x) do { const long long now_ = clock64(); x += now_ - st_t; st_t = now_; } while (0)
 #else
 #define F32_MARK(x)
@@ -168,115 +190,175 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
         const int row0 = I * TS, col0 = J * TS;
         F32_MARK(st_claim);
 
-        // ---- 1. the two contractions.  Source list: tiles (0..I-2, J) through L, tiles (I, 0..J-2) through U, then
-        // the tile above and the tile to the left (the newest ones, still being swept when this tile is claimed).
-        float cd[4][4], rt[4][4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) cd[i][j] = rt[i][j] = 0.f;
-        const int nsrc = I + J, nslab = nsrc * SPS;
+        // ---- 1. the contractions, one accumulator at a time: Rt over the older tiles of the row (I, 0..J-2) through U,
+        // parked in shared memory; Cd over the column (0..I-1, J) through L (the tile above, still being swept when this
+        // tile is claimed, is its last source); Rt's last term from the tile to the left.
+        float acc[16][8];
         bool ok = true;
-        // slab g of the flattened list belongs to source g / 4; operands of a source (all threads compute them)
-        struct Src { const float *A, *B; long lda, ldb; int a_rows, a_kmax, b_cols, b_kmax, dir; const unsigned *flag; };
-        auto source = [&](int sidx) {
-            int dir, k;
-            const int na = max(0, I - 1), nl = max(0, J - 1);        // older sources of each direction
-            if (sidx < na) { dir = 0; k = sidx; }
-            else if (sidx < na + nl) { dir = 1; k = sidx - na; }
-            else if (sidx == na + nl && I > 0) { dir = 0; k = I - 1; }
-            else { dir = 1; k = J - 1; }
+        struct Src { const float *A, *B; long lda, ldb; int a_rows, b_cols, kmax; const unsigned *flag; };
+        auto source = [&](int dir, int k) {
             Src r;
-            r.dir = dir;
             if (dir == 0) {          // L[r, rows of tile k] * E[rows of tile k, c]
-                r.A = p.L32 + (long)row0 * p.ldl + (long)k * TS; r.lda = p.ldl;
-                r.a_rows = min(TS, p.m - row0); r.a_kmax = min(TS, p.m - k * TS);
-                r.B = p.E32 + (long)k * TS * p.np + col0; r.ldb = p.np; r.b_cols = TS; r.b_kmax = TS;
+                r.A = p.L32t + (long)k * TS * p.ldl + row0; r.lda = p.ldl; r.a_rows = min(TS, p.m - row0);
+                r.B = p.E32 + (long)k * TS * p.np + col0; r.ldb = p.np; r.b_cols = TS;
+                r.kmax = min(TS, p.m - k * TS);
                 r.flag = p.flags + (long)k * p.ntj + J;
             } else {                 // C[r, columns of tile k] * U[columns of tile k, c]
-                r.A = p.C32 + (long)row0 * p.np + (long)k * TS; r.lda = p.np; r.a_rows = TS; r.a_kmax = TS;
-                r.B = p.U32 + (long)k * TS * p.ldu + col0; r.ldb = p.ldu;
-                r.b_cols = min(TS, p.n - col0); r.b_kmax = min(TS, p.n - k * TS);
+                r.A = p.C32t + (long)k * TS * p.mp + row0; r.lda = p.mp; r.a_rows = TS;
+                r.B = p.U32 + (long)k * TS * p.ldu + col0; r.ldb = p.ldu; r.b_cols = min(TS, p.n - col0);
+                r.kmax = min(TS, p.n - k * TS);
                 r.flag = p.flags + (long)I * p.ntj + k;
             }
             return r;
         };
-        // Sources [0, ready_upto) are known to be swept.  The list is scanned by the whole CTA at once (one flag per
-        // thread, the first unset position by a shared-memory minimum), so that a tile whose far sources are all
-        // done -- the usual case -- pays two barriers for the lot instead of a global round trip per source; only
-        // when the next source in line is still being swept does one thread wait for it, bounded.
-        int ready_upto = 0;
-        auto scan_ready = [&](int from) -> bool {         // all threads; false if the bounded wait ran out
-            if (tid == 0) {
-                unsigned long long it = 0;
-                int good = 1;
-                const Src sr = source(from);
-                while (ld_acquire_u32(sr.flag) == 0u) {
-                    if (++it > p.spin_limit || ld_relaxed_u32(p.abort) != 0u) {
-                        report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -9, task, (int)blockIdx.x);
-                        atomicExch(p.abort, 1u);
-                        good = 0;
-                        break;
+        // One contraction: acc = sum over the sources k0 .. k1-1 of direction dir.  Sources [k0, ready_upto) are known to
+        // be swept.  The list is scanned by the whole CTA at once (one flag per thread, the first unset position by a
+        // shared-memory minimum), so that a tile whose far sources are all done -- the usual case -- pays two barriers
+        // for the lot instead of a global round trip per source; only when the next source in line is still being swept
+        // does one thread wait for it, bounded.  Returns with the ring drained.
+        auto contract = [&](int dir, int k0, int k1) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+            const int nslab = (k1 - k0) * SPS;
+            int ready_upto = k0;
+            auto scan_ready = [&](int from) -> bool {         // all threads; false if the bounded wait ran out
+#ifdef TILED_STATS
+                const long long w0_ = clock64();
+#endif
+                if (tid == 0) {
+                    unsigned long long it = 0;
+                    int good = 1;
+                    const Src sr = source(dir, from);
+                    while (ld_acquire_u32(sr.flag) == 0u) {
+                        if (++it > p.spin_limit || ld_relaxed_u32(p.abort) != 0u) {
+                            report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -9, task, (int)blockIdx.x);
+                            atomicExch(p.abort, 1u);
+                            good = 0;
+                            break;
+                        }
+                        __nanosleep(100);
                     }
-                    __nanosleep(100);
+                    s_ok = good;
+                    s_upto = k1;
                 }
-                s_ok = good;
-                s_upto = nsrc;
+                __syncthreads();
+                for (int k = from + 1 + tid; k < k1; k += THREADS)
+                    if (ld_acquire_u32(source(dir, k).flag) == 0u) atomicMin(&s_upto, k);
+                __syncthreads();
+                const bool good = s_ok != 0;
+                ready_upto = s_upto;
+                __syncthreads();                              // s_ok / s_upto may be rewritten by the next scan
+#ifdef TILED_STATS
+                st_wait += clock64() - w0_;
+#endif
+                return good;
+            };
+            auto issue_slab = [&](int g) -> bool {            // all threads; false if a wait ran out
+                const int k = k0 + g / SPS;
+                if (k >= ready_upto && !scan_ready(k)) return false;
+                const Src sr = source(dir, k);
+                gm.issue(g % NSTAGE, sr.A, sr.lda, sr.a_rows, sr.B, sr.ldb, sr.b_cols, sr.kmax, (g % SPS) * KS);
+                return true;
+            };
+            for (int g = 0; g < NSTAGE - 1 && ok; ++g) {
+                if (g < nslab) ok = issue_slab(g);
+                cp_async_commit();
+            }
+            for (int g = 0; g < nslab && ok; ++g) {
+                cp_async_wait<NSTAGE - 2>();
+                __syncthreads();                           // slab g has landed; everyone is past slab g - 1, whose stage is free
+                if (g + NSTAGE - 1 < nslab) ok = issue_slab(g + NSTAGE - 1);
+                cp_async_commit();
+                if (!ok) break;
+                gm.multiply(acc, g % NSTAGE);
+            }
+            cp_async_wait<0>();
+            __syncthreads();
+        };
+        // Sum of the groups' partial tiles; thread t gets rows (t >> 4) + (THREADS / 16) h, columns 4 (t & 15) .. + 3.  The ring
+        // is drained on entry and free again on return.
+        auto reduce = [&](float4 (&v)[RPT]) {
+            gm.stage_partial(acc);
+            __syncthreads();
+#pragma unroll
+            for (int h = 0; h < RPT; ++h) {
+                const float *q = stages + ((tid >> 4) + (THREADS / 16) * h) * LDB + 4 * (tid & 15);
+                float4 a = *reinterpret_cast<const float4 *>(q);
+#pragma unroll
+                for (int g = 1; g < KGROUPS; ++g) {
+                    const float4 b = *reinterpret_cast<const float4 *>(q + g * PMAT);
+                    a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+                }
+                v[h] = a;
             }
             __syncthreads();
-            for (int k = from + 1 + tid; k < nsrc; k += THREADS)
-                if (ld_acquire_u32(source(k).flag) == 0u) atomicMin(&s_upto, k);
-            __syncthreads();
-            const bool good = s_ok != 0;
-            ready_upto = s_upto;
-            __syncthreads();                              // s_ok / s_upto may be rewritten by the next scan
-            return good;
         };
-        // Issues slab g (all threads); returns false if a wait ran out.
-        auto issue_slab = [&](int g) -> bool {
-            const int sidx = g / SPS;
-            if (sidx >= ready_upto && !scan_ready(sidx)) return false;
-            const Src sr = source(sidx);
-            gm.issue(g % NSTAGE, sr.A, sr.lda, sr.a_rows, sr.a_kmax, sr.B, sr.ldb, sr.b_cols, sr.b_kmax, (g % SPS) * KS);
-            return true;
-        };
-        for (int g = 0; g < NSTAGE - 1 && ok; ++g) {
-            if (g < nslab) ok = issue_slab(g);
-            cp_async_commit();
-        }
-        for (int g = 0; g < nslab && ok; ++g) {
-            cp_async_wait<NSTAGE - 2>();
-            __syncthreads();                           // slab g has landed; everyone is past slab g - 1, whose stage is free
-            if (g + NSTAGE - 1 < nslab) ok = issue_slab(g + NSTAGE - 1);
-            cp_async_commit();
+        // A finished sum waits in shared memory while the next contraction runs; a thread reads back what it wrote itself.
+        const int own = (tid >> 4) * TS + 4 * (tid & 15);        // + (THREADS / 16) h rows
+        constexpr int OWN_STEP = (THREADS / 16) * TS;
+        float4 v4[RPT];
+        const bool far_rt = J > 1;
+        if (far_rt) {
+            contract(1, 0, J - 1);
             if (!ok) break;
-            if (source(g / SPS).dir == 0) gm.multiply(cd, g % NSTAGE); else gm.multiply(rt, g % NSTAGE);
+            reduce(v4);
+#pragma unroll
+            for (int h = 0; h < RPT; ++h) *reinterpret_cast<float4 *>(park_rt + own + h * OWN_STEP) = v4[h];
         }
-        cp_async_wait<0>();
-        __syncthreads();
-        if (!ok) break;
+        if (I > 0) {
+            contract(0, 0, I);
+            if (!ok) break;
+            reduce(v4);
+#pragma unroll
+            for (int h = 0; h < RPT; ++h) *reinterpret_cast<float4 *>(park_cd + own + h * OWN_STEP) = v4[h];
+        }
+        if (J > 0) {
+            contract(1, J - 1, J);
+            if (!ok) break;
+            reduce(v4);
+        }
+        float4 cdv[RPT], rtv[RPT];
+#pragma unroll
+        for (int h = 0; h < RPT; ++h) {
+            const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+            rtv[h] = J > 0 ? v4[h] : zero;
+            if (far_rt) {
+                const float4 q = *reinterpret_cast<const float4 *>(park_rt + own + h * OWN_STEP);
+                rtv[h] = make_float4(q.x + rtv[h].x, q.y + rtv[h].y, q.z + rtv[h].z, q.w + rtv[h].w);
+            }
+            cdv[h] = I > 0 ? *reinterpret_cast<const float4 *>(park_cd + own + h * OWN_STEP) : zero;
+        }
+        __syncthreads();                    // the in-tile matrices overlap the parked sums
         F32_MARK(st_gemm);
 
-        // ---- 2. Y = X + Rt + Cd, C = Cd; diagonal blocks of the factors (strict triangles, zero elsewhere)
+        // ---- 2. Y = X + Rt + Cd, C = Cd; the diagonal block of U (strictly upper, kept transposed; its first
+        // super-diagonal U[j-1, j] apart, see below)
         {
-            const int ty = tid >> 4, tx = tid & 15;
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int h = 0; h < RPT; ++h) {
+                const int r = (tid >> 4) + (THREADS / 16) * h, c = 4 * (tid & 15), gr = row0 + r, gc = col0 + c;
+                const float rt4[4] = {rtv[h].x, rtv[h].y, rtv[h].z, rtv[h].w}, cd4[4] = {cdv[h].x, cdv[h].y, cdv[h].z, cdv[h].w};
+                float y4[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    const int r = ty * 4 + i, c = tx * 4 + j, gr = row0 + r, gc = col0 + c;
-                    const float x = (gr < p.m && gc < p.n) ? (float)__ldg(p.X + (long)gr * p.ldx + gc) : 0.f;
-                    Cs[r * LDT + c] = cd[i][j];
-                    Ys[r * LDT + c] = (x + rt[i][j]) + cd[i][j];
+                    const float x = (gr < p.m && gc + j < p.n) ? (float)__ldg(p.X + (long)gr * p.ldx + gc + j) : 0.f;
+                    y4[j] = (x + rt4[j]) + cd4[j];
                 }
+                *reinterpret_cast<float4 *>(Cs + r * LDT + c) = cdv[h];
+                *reinterpret_cast<float4 *>(Ys + r * LDT + c) = make_float4(y4[0], y4[1], y4[2], y4[3]);
+                // unrounded entries count as zero (they meet zero coefficients)
+                *reinterpret_cast<float4 *>(Et + r * LDT + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            if (tid == 0) s_usub[0] = 0.f;
 #pragma unroll 8
             for (int e = tid; e < TS * TS; e += THREADS) {
-                const int r = e >> 6, c = e & 63;
-                const int gr = row0 + r, gcl = row0 + c;       // L block: rows / columns of the row range
-                Ld[r * LDT + c] = (c < r && gr < p.m) ? p.L32[(long)gr * p.ldl + gcl] : 0.f;
-                const int ur = col0 + r, uc = col0 + c;        // U block (r, c) with r < c, stored transposed
-                Udt[c * LDT + r] = (c > r && uc < p.n) ? p.U32[(long)ur * p.ldu + uc] : 0.f;
-                Et[r * LDT + c] = 0.f;                         // unrounded entries count as zero (they meet zero coefficients)
+                const int a = e >> 6, b = e & 63;              // U block entry (row a, column b), b along the contiguous direction
+                const int ur = col0 + a, uc = col0 + b;
+                const float v = (b > a && uc < p.n) ? p.U32[(long)ur * p.ldu + uc] : 0.f;
+                Udt[b * LDT + a] = (b == a + 1) ? 0.f : v;
+                if (b == a + 1) s_usub[b] = v;
             }
         }
         __syncthreads();
@@ -285,46 +367,95 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
         // ---- 3. the tile's 127 anti-diagonals, in the implicit-Y (pull) form of Appendix B, Eq. 19-20, which gives
         // the same entries as Algorithm 3: entry (i, j) reconstructs its corrected value when it is rounded,
         //     Y_ij = Y0_ij + sum_{i' < i} L[i, i'] E[i', j] + sum_{j' < j} C[i, j'] U[j', j],
-        // and its final C_ij = C0_ij + sum_{i' < i} L[i, i'] E[i', j] + E_ij is stored once.  Everything it reads was
-        // rounded on an earlier anti-diagonal, nothing is read-modify-written, and only the rows that own an
-        // entry of the current anti-diagonal work: four lanes per row, each a quarter of the two dot products.
+        // and its final C_ij = C0_ij + sum_{i' < i} L[i, i'] E[i', j] + E_ij is stored once.  Four lanes per row.  Of the
+        // two sums only the last terms, E[i-1, j] and C[i, j-1], come from the anti-diagonal just before; everything else
+        // was rounded at least two steps ago.  So a step is split: all four lanes form the sums WITHOUT their last terms for
+        // the row's NEXT entry (dot products along rows of shared memory, whose coefficients at and beyond the last
+        // term are stored as zeros: what they meet there -- zeros, unrounded values, or an entry being written
+        // this very step -- is finite and drops out), and the row's first lane rounds the CURRENT entry from the sums
+        // formed one step earlier plus the two last terms: one shared-memory load (E[i-1, j]; C[i, j-1] is its own
+        // previous result), one FMA, the rounding.  The two parts are independent, so the long one runs in the shadow of
+        // the dependent one; the CTA barrier per anti-diagonal stays.
         // Ys holds Y0 until an entry is rounded and E afterwards; Cs holds C0 and then C.
         {
             const int row = tid >> 2, sub = tid & 3;
-            const float *lrow = Ld + row * LDT;
+            const bool row_in = row0 + row < p.m;
+            // the lane's quarter of row `row` of the diagonal block of L: columns 4 (sub + 4 t) .. + 3, strictly lower,
+            // the first sub-diagonal entry L[i, i-1] apart
+            float lr[16];
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int ip = 4 * (sub + 4 * t) + e;
+                    lr[4 * t + e] = (ip < row - 1 && row_in) ? __ldg(p.L32t + (long)(row0 + ip) * p.ldl + row0 + row) : 0.f;
+                }
+            const float lsub = (row > 0 && row_in) ? __ldg(p.L32t + (long)(row0 + row - 1) * p.ldl + row0 + row) : 0.f;
+            const float4 *c4 = reinterpret_cast<const float4 *>(Cs + row * LDT) + sub;
+            const int w8 = (tid >> 5) * 8;                           // the warp's first row
+            const int tl = (w8 + 6 + 15) >> 4;                       // chunks of 16 rows that hold a source i' < row - 1 of the warp's last row
             float *yrow = Ys + row * LDT, *crow = Cs + row * LDT;
             unsigned long long badkey = ~0ull;
             float max_e = 0.f;
-            for (int s = 0; s < 2 * TS - 1; ++s) {
-                const int j = s - row;
-                if (j >= 0 && j < TS) {                                  // (uniform over the row's four lanes)
-                    // Both dot products run along rows of shared memory in chunks of four; a lane takes every fourth
-                    // chunk.  Beyond the diagonal the coefficients are zero (strict triangles) and what they meet is
-                    // finite (zeros, or values of entries rounded later), so whole chunks need no masking.
+            float base_y = 0.f, base_c = 0.f, c_last = 0.f;      // (first lane of the row)
+#ifdef TILED_STATS
+            long long sw_t = clock64();
+#define SW_MARK(x) do { const long long n_ = clock64(); x += n_ - sw_t; sw_t = n_; } while (0)
+#else
+#define SW_MARK(x)
+#endif
+            for (int s = -1; s < 2 * TS - 1; ++s) {
+                const int j = s - row, jn = j + 1;                        // the row's current and next entry
+                const bool cur_in = j >= 0 && j < TS, next_in = jn >= 0 && jn < TS;
+                // (loads first: what is stored further down cannot overtake them)
+                float e_up = 0.f, y0n = 0.f, c0n = 0.f, usubn = 0.f;
+                if (sub == 0) {
+                    if (cur_in && row > 0) e_up = Et[j * LDT + row - 1];
+                    if (next_in) { y0n = yrow[jn]; c0n = crow[jn]; usubn = s_usub[jn]; }
+                }
+                // Sums for the next entry, without their last terms.  Whole warps skip the step while none of their rows
+                // has a next entry; inside, every lane goes through the same loads and shuffles (rows of a warp differ in
+                // whether and how far they need them; a shuffle under a per-row mask would split the warp): the trip counts
+                // are those of the warp's longest row, and a chunk that holds no source of a shorter row meets zero
+                // coefficients.  Without the skipping the sweep is bound by issue slots and shared-memory bandwidth.
+                float sl = 0.f, su = 0.f;
+                const int jn_hi = s + 1 - w8;                            // next column of the warp's first row (the largest)
+                if (jn_hi >= 0 && jn_hi - 7 < TS) {
+                    const int jr = next_in ? jn : 0;
+                    const float4 *e4 = reinterpret_cast<const float4 *>(Et + jr * LDT) + sub, *u4 = reinterpret_cast<const float4 *>(Udt + jr * LDT) + sub;
+                    const int tu = min(4, (jn_hi + 14) >> 4);            // chunks of 16 columns that hold a source j' < jn - 1
                     float dl[2] = {0.f, 0.f}, du[2] = {0.f, 0.f};
-                    const float4 *l4 = reinterpret_cast<const float4 *>(lrow), *e4 = reinterpret_cast<const float4 *>(Et + j * LDT);
-                    for (int q = sub; 4 * q < row; q += 4) {                // down the column: sources i' < row
-                        const float4 a = l4[q], b = e4[q];
-                        dl[0] = fmaf(a.x, b.x, dl[0]); dl[1] = fmaf(a.y, b.y, dl[1]);
-                        dl[0] = fmaf(a.z, b.z, dl[0]); dl[1] = fmaf(a.w, b.w, dl[1]);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {                        // down the column: sources i' < row - 1
+                        if (t < tl) {
+                            const float4 b = e4[4 * t];
+                            dl[0] = fmaf(lr[4 * t + 0], b.x, dl[0]); dl[1] = fmaf(lr[4 * t + 1], b.y, dl[1]);
+                            dl[0] = fmaf(lr[4 * t + 2], b.z, dl[0]); dl[1] = fmaf(lr[4 * t + 3], b.w, dl[1]);
+                        }
                     }
-                    const float4 *c4 = reinterpret_cast<const float4 *>(crow), *u4 = reinterpret_cast<const float4 *>(Udt + j * LDT);
-                    for (int q = sub; 4 * q < j; q += 4) {                  // along the row: sources j' < j
-                        const float4 a = c4[q], b = u4[q];
-                        du[0] = fmaf(a.x, b.x, du[0]); du[1] = fmaf(a.y, b.y, du[1]);
-                        du[0] = fmaf(a.z, b.z, du[0]); du[1] = fmaf(a.w, b.w, du[1]);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {                        // along the row: sources j' < jn - 1
+                        if (t < tu) {
+                            const float4 a = c4[4 * t], b = u4[4 * t];
+                            du[0] = fmaf(a.x, b.x, du[0]); du[1] = fmaf(a.y, b.y, du[1]);
+                            du[0] = fmaf(a.z, b.z, du[0]); du[1] = fmaf(a.w, b.w, du[1]);
+                        }
                     }
-                    float sl = dl[0] + dl[1], su = du[0] + du[1];
-                    const unsigned gmask = 0xfu << ((tid & 31) & ~3);          // the row's four lanes (rows of a warp differ in activity)
-                    sl += __shfl_xor_sync(gmask, sl, 1);
-                    su += __shfl_xor_sync(gmask, su, 1);
-                    sl += __shfl_xor_sync(gmask, sl, 2);
-                    su += __shfl_xor_sync(gmask, su, 2);
-                    if (sub == 0) {
-                        const float y = (yrow[j] + su) + sl;
+                    sl = dl[0] + dl[1]; su = du[0] + du[1];
+                    sl += __shfl_xor_sync(0xffffffffu, sl, 1);
+                    su += __shfl_xor_sync(0xffffffffu, su, 1);
+                    sl += __shfl_xor_sync(0xffffffffu, sl, 2);
+                    su += __shfl_xor_sync(0xffffffffu, su, 2);
+                }
+                SW_MARK(sw_sums);
+                if (sub == 0) {
+                    if (cur_in) {
+                        const float t = lsub * e_up;                     // (lsub = 0 in row 0)
+                        const float y = base_y + t;
                         const float z = rintf(y);
                         const float e = z - y;                           // E = Z - Y
-                        crow[j] = (crow[j] + sl) + e;                    // C = L E (unit diagonal)
+                        c_last = (base_c + t) + e;                       // C = L E (unit diagonal)
+                        crow[j] = c_last;
                         yrow[j] = e;
                         Et[j * LDT + row] = e;
                         int zi = (int)z;
@@ -338,8 +469,14 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
                         Zs[row * TS + j] = zi;
                         max_e = fmaxf(max_e, fabsf(e));
                     }
+                    if (next_in) {
+                        base_c = c0n + sl;
+                        base_y = fmaf(c_last, usubn, (y0n + su) + sl);   // c_last: C[i, jn - 1], rounded just above
+                    }
                 }
+                SW_MARK(sw_round);
                 __syncthreads();
+                SW_MARK(sw_bar);
             }
             max_abs_e = fmax(max_abs_e, (double)max_e);      // (entries outside the matrix are exact zeros with E = 0)
             if (badkey != ~0ull) atomicMin(&s_badkey, badkey);
@@ -356,10 +493,9 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
             }
         }
         for (int e = tid; e < TS * TS; e += THREADS) {
-            const int r = e >> 6, c = e & 63;
-            const long at = (long)(row0 + r) * p.np + col0 + c;
-            p.E32[at] = Ys[r * LDT + c];
-            p.C32[at] = Cs[r * LDT + c];
+            const int a = e >> 6, b = e & 63;
+            p.E32[(long)(row0 + a) * p.np + col0 + b] = Ys[a * LDT + b];
+            p.C32t[(long)(col0 + a) * p.mp + row0 + b] = Cs[b * LDT + a];     // transposed: the next tiles read C depth-major
         }
         __syncthreads();
         if (tid == 0) {
@@ -378,9 +514,12 @@ __global__ void __launch_bounds__(THREADS, 2) round_tiled_f32_kernel(Params p) {
 #endif
     }
 #ifdef TILED_STATS
+    if (tid == 128 && (blockIdx.x % 61) == 0 && st_n > 0)
+        printf("cta %3d row 32 per step: sums %lld rounding %lld barrier %lld\n", (int)blockIdx.x, sw_sums / (st_n * 128), sw_round / (st_n * 128),
+               sw_bar / (st_n * 128));
     if (tid == 0 && (blockIdx.x % 61) == 0 && st_n > 0)
-        printf("cta %3d tiles %lld | per tile: claim %lld gemm(+flag waits) %lld form %lld sweep %lld store %lld\n", (int)blockIdx.x, st_n,
-               st_claim / st_n, st_gemm / st_n, st_form / st_n, st_sweep / st_n, st_store / st_n);
+        printf("cta %3d tiles %lld | per tile: claim %lld gemm(+flag waits) %lld of which flag scans and waits %lld form %lld sweep %lld store %lld\n",
+               (int)blockIdx.x, st_n, st_claim / st_n, st_gemm / st_n, st_wait / st_n, st_form / st_n, st_sweep / st_n, st_store / st_n);
 #endif
     for (int o = 16; o > 0; o >>= 1) max_abs_e = fmax(max_abs_e, __shfl_xor_sync(0xffffffffu, max_abs_e, o));
     if ((tid & 31) == 0) s_red[tid >> 5] = max_abs_e;
@@ -399,6 +538,25 @@ __global__ void narrow_kernel(float *dst, long ldd, const double *src, long lds,
         const long r = idx / ldd;
         const int c = (int)(idx - r * ldd);
         dst[idx] = c < cols ? (float)src[r * lds + c] : 0.f;
+    }
+}
+
+// the same, transposed: dst[c][r] = src[r][c] for a square matrix of order n; 32 x 32 pieces through shared memory, blocks of 32 x 8
+__global__ void narrow_transposed_kernel(float *dst, long ldd, const double *src, long lds, int n) {
+    __shared__ float t[32][33];
+    const int nb = (int)((ldd + 31) / 32);
+    for (long piece = blockIdx.x; piece < (long)nb * nb; piece += gridDim.x) {
+        const int r0 = (int)(piece / nb) * 32, c0 = (int)(piece % nb) * 32;
+        for (int i = threadIdx.y; i < 32; i += 8) {
+            const int r = r0 + i, c = c0 + threadIdx.x;
+            t[i][threadIdx.x] = (r < n && c < n) ? (float)src[(long)r * lds + c] : 0.f;
+        }
+        __syncthreads();
+        for (int i = threadIdx.y; i < 32; i += 8) {
+            const int c = c0 + i, r = r0 + threadIdx.x;                    // dst row c, column r
+            if (c < n && r < ldd) dst[(long)c * ldd + r] = t[threadIdx.x][i];
+        }
+        __syncthreads();
     }
 }
 
@@ -436,9 +594,9 @@ int launch_round_tiled_f32(const TiledParams &in, void *ws, size_t ws_bytes, cud
     p.mp = l.mp; p.np = l.np;
     p.X = in.X; p.ldx = in.ldx; p.Z = in.Z; p.ldz = in.ldz; p.Euser = in.E; p.lde = in.lde;
     float *L32 = reinterpret_cast<float *>(w + l.l_off), *U32 = reinterpret_cast<float *>(w + l.u_off);
-    p.L32 = L32; p.ldl = l.ldl; p.U32 = U32; p.ldu = l.ldu;
+    p.L32t = L32; p.ldl = l.ldl; p.U32 = U32; p.ldu = l.ldu;
     p.E32 = reinterpret_cast<float *>(w + l.e_off);
-    p.C32 = reinterpret_cast<float *>(w + l.c_off);
+    p.C32t = reinterpret_cast<float *>(w + l.c_off);
     p.counter = reinterpret_cast<unsigned *>(w);
     p.abort = reinterpret_cast<unsigned *>(w) + 1;
     p.flags = reinterpret_cast<unsigned *>(w + l.flags_off);
@@ -449,7 +607,7 @@ int launch_round_tiled_f32(const TiledParams &in, void *ws, size_t ws_bytes, cud
     int dev = 0, sms = 0, per_sm = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return GPTQ2D_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GPTQ2D_ERR_CUDA;
-    narrow_kernel<<<sms * 4, 256, 0, stream>>>(L32, l.ldl, in.L, in.ldl, in.m, in.m);
+    narrow_transposed_kernel<<<sms * 8, dim3(32, 8), 0, stream>>>(L32, l.ldl, in.L, in.ldl, in.m);
     narrow_kernel<<<sms * 4, 256, 0, stream>>>(U32, l.ldu, in.U, in.ldu, in.n, in.n);
     if (cudaGetLastError() != cudaSuccess) return GPTQ2D_ERR_CUDA;
     if (cudaFuncSetAttribute(round_tiled_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
@@ -457,7 +615,7 @@ int launch_round_tiled_f32(const TiledParams &in, void *ws, size_t ws_bytes, cud
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, round_tiled_f32_kernel, THREADS, SMEM_BYTES) != cudaSuccess ||
         per_sm < 1)
         return GPTQ2D_ERR_CUDA;
-    if (per_sm > 2) per_sm = 2;
+    if (per_sm > 1) per_sm = 1;
     int grid = sms * per_sm;
     if (grid > p.ntiles) grid = p.ntiles;
     void *args[] = {&p};
