@@ -6,28 +6,32 @@
 //     Cd = sum_{I' < I} L[r, I'] E[I', c]        Rt = sum_{J' < J} C[r, J'] U[J', c]
 // and Algorithm 3 on the tile alone, started from Y = X[r, c] + Rt + Cd and C = Cd with the diagonal
 // blocks L[r, r] and U[c, c], gives the tile's Z, E and C = L E.  fp32 has no tensor-core path that keeps
-// fp32 operands exact (TF32 truncates them), so the two contractions are a register-tiled FFMA loop:
-// 256 threads in four groups of 64; a group takes a quarter of every slab's depth and holds an 8 x 8 piece
-// of the whole 64 x 64 tile per thread (one shared-memory float per four FMAs; a 4 x 4 piece per thread
-// without the split needs twice the loads and ran at 30 % of the FMA pipe), and the four partial tiles are
-// added through shared memory when a contraction ends.  Both operands of a slab are stored depth-major
-// ([k][64 rows] and [k][64 columns]: L and C are kept transposed in the workspace for this), staged with
-// cp.async through a four-stage ring of slabs of 32.  A thread cannot hold two 8 x 8 accumulators, so a tile
-// runs three contractions one after the other: Rt over the older tiles of its row, Cd over its whole column
-// (the tile above comes last), Rt's last term from the tile to the left -- the newest sources still come last.
+// fp32 operands exact (TF32 truncates them), so the two contractions are a register-tiled FFMA loop.
+// The loop is bound by the shared-memory load pipe before the FMA pipe (a 16-byte load costs a warp four
+// cycles of it and feeds four operand words per lane), so the register piece is as large as the register
+// file allows: one CTA of 256 threads per SM, every WARP covers the whole 64 x 64 tile with a 16 x 8 piece
+// per lane (six loads per 128 FMAs) and takes an eighth of every slab's depth; the eight partial tiles are
+// added through shared memory when a contraction ends.  (History at 8192 x 8192: 4 x 4 pieces, two CTAs
+// per SM, 30 % of the FMA pipe, 52.6 ms; 8 x 8 pieces in 512 threads 41.6 ms; 16 x 8 in 256 threads
+// 38.7 ms.)  Both operands of a slab are stored depth-major ([k][64 rows] and [k][64 columns]: L and C are
+// kept transposed in the workspace for this), staged with cp.async through a four-stage ring of slabs of 64.
+// A thread cannot hold two accumulators of that size, so a tile runs three contractions one after the other:
+// Rt over the older tiles of its row, Cd over its whole column (the tile above comes last), Rt's last term
+// from the tile to the left -- the newest sources still come last; finished sums wait in shared memory.
 //
-// One persistent, cooperatively launched grid, two CTAs per SM.  Tiles are claimed wave by wave (I + J
-// ascending) from one atomic counter; a CTA folds the source tiles in as their flags come up -- the far
-// ones first, the tile above and the tile to the left last -- and then sweeps its tile.  While one CTA
-// of an SM sits in the dependent chain of its in-tile sweep the other one multiplies.  A tile only waits
-// for tiles of earlier waves, which were claimed earlier, so the earliest unfinished tile can always run.
+// One persistent, cooperatively launched grid, one CTA per SM.  Tiles are claimed wave by wave (I + J
+// ascending) from one atomic counter; a CTA folds the source tiles in as their flags come up and then
+// sweeps its tile.  A tile only waits for tiles of earlier waves, which were claimed earlier, so the
+// earliest unfinished tile can always run.  (Two slower CTAs per SM, one multiplying while the other
+// sweeps, lose: the tile above and the tile to the left are on every tile's critical path, and a CTA that
+// shares its SM takes twice as long over them.)
 //
 // In-tile sweep: one anti-diagonal per step, one CTA barrier per step, in the implicit-Y (pull) form of
 // Appendix B (Eq. 19-20): an entry reads the errors above it in its column through L and the finished C to
 // its left in its row through U at the moment it is rounded, four lanes per row sharing the two dot
-// products.  Only rows with an entry on the current anti-diagonal work, and nothing is read-modify-written
-// (an eager version that pushed every error down and right as Algorithm 3 prints it cost 7x the time per
-// step: 2 x 64 x 64 shared-memory updates per anti-diagonal, issued by every warp).
+// products; all of both sums except their last terms is formed one step ahead.  Nothing is read-modify-
+// written (an eager version that pushed every error down and right as Algorithm 3 prints it cost 7x the
+// time per step: 2 x 64 x 64 shared-memory updates per anti-diagonal, issued by every warp).
 #include <cstdio>
 #include "common.cuh"
 #include "dmma_gemm.cuh"          // cp.async helpers
@@ -96,10 +100,18 @@ struct Gemm {
     int tid, gk, ty, tx;           // group (quarter of the depth), position in the group's 8 x 8 thread grid
     // copy plan: each slab is KS k x 64 entries in chunks of 4 floats, KS * 16 / THREADS chunks of each slab per thread
     __device__ __forceinline__ void issue_one(float *S, const float *P, long ld, int valid, int kmax, int k0) const {
+        constexpr int RPH = THREADS / 16;                            // slab rows covered by one round of the CTA
+        const int kr0 = tid >> 4, cc = (tid & 15) * 4;
+        if (valid >= TS && kmax - k0 >= KS) {                        // interior slab: nothing to clip (uniform over the CTA)
+            float *sdst = S + kr0 * LDB + cc;
+            const float *g = P + (long)(k0 + kr0) * ld + cc;
 #pragma unroll
-        for (int h = 0; h < KS * 16 / THREADS; ++h) {
-            const int c = tid + h * THREADS;
-            const int kr = c >> 4, cc = (c & 15) * 4;
+            for (int h = 0; h < KS / RPH; ++h) cp_async16(sdst + h * RPH * LDB, g + (long)h * RPH * ld, 16);
+            return;
+        }
+#pragma unroll
+        for (int h = 0; h < KS / RPH; ++h) {
+            const int kr = kr0 + h * RPH;
             int nv = (k0 + kr < kmax) ? valid - cc : 0;              // floats valid from cc on
             nv = nv < 0 ? 0 : (nv > 4 ? 4 : nv);
             cp_async16f(S + kr * LDB + cc, nv ? P + (long)(k0 + kr) * ld + cc : P, nv * 4);
@@ -417,7 +429,9 @@ __global__ void __launch_bounds__(THREADS, 1) round_tiled_f32_kernel(Params p) {
                 // has a next entry; inside, every lane goes through the same loads and shuffles (rows of a warp differ in
                 // whether and how far they need them; a shuffle under a per-row mask would split the warp): the trip counts
                 // are those of the warp's longest row, and a chunk that holds no source of a shorter row meets zero
-                // coefficients.  Without the skipping the sweep is bound by issue slots and shared-memory bandwidth.
+                // coefficients.  The step is bound by the shared-memory load pipe (a 16-byte load costs a warp four to six
+                // cycles however many lanes use it; whole rows for all 64 rows are 96 loads a step), which is why chunks
+                // that hold no source are skipped by whole warps and the row of L stays in registers.
                 float sl = 0.f, su = 0.f;
                 const int jn_hi = s + 1 - w8;                            // next column of the warp's first row (the largest)
                 if (jn_hi >= 0 && jn_hi - 7 < TS) {
