@@ -315,6 +315,8 @@ int gptq2d_objective(int m, int n,
  *   key 5 (checked builds of the library only; otherwise unknown): value = address of a device int[5].  Runs the
  *          self-test of the index check on the default stream: one deliberately out-of-range index (7 of 3,
  *          site 999) is checked; [0..3] receive {GPTQ2D_ERR_CHECK, 999, 7, 3}, [4] the redirected index 0.
+ *   key 6: how the fp32 mode's contraction gets its operand slabs.  0 (default): bulk tensor copies (TMA) where
+ *          the driver offers tensor maps, cp.async otherwise; 1: cp.async always.  Comparison runs and tests.
  * Returns GPTQ2D_OK, or GPTQ2D_ERR_INVALID_ARG for an unknown key.
  */
 int gptq2d_internal_test_hook(int key, long value);

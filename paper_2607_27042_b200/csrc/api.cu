@@ -550,6 +550,7 @@ int gptq2d_internal_test_hook(int key, long value) {
     if (key == 2) { g_hook_panel_spin_limit.store(value > 0 ? value : 0); return GPTQ2D_OK; }
     if (key == 3) { gemm_set_tma_mode((int)value); return GPTQ2D_OK; }
     if (key == 4) { round_fused_set_mode((int)value); return GPTQ2D_OK; }
+    if (key == 6) { round_tiled_f32_set_tma_mode((int)value); return GPTQ2D_OK; }
 #ifdef GPTQ2D_CHECKED
     if (key == 5) {          // value: device int[5]; [0..3] receive the status words, [4] the redirected index
         int *dev = reinterpret_cast<int *>(static_cast<uintptr_t>(value));

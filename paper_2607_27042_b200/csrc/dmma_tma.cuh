@@ -104,6 +104,15 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *map, i
         : "memory");
 }
 
+// 2-D tiled copy global -> shared (own CTA), completion reported to `bar`
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, unsigned long long *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n" ::"r"(
+            smem_u32(dst)),
+        "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+        : "memory");
+}
+
 // ---- fragment <-> matrix index maps -----------------------------------------------------------
 __device__ __forceinline__ int frag_map_mn(int g) { return (g & 1) | (((g >> 1) & 1) << 3) | ((g >> 2) << 1); }
 // matrix row / column (inside the warp's 64- or 32-wide strip) that fragment f, position q (0..7) stands for

@@ -63,6 +63,7 @@ int launch_round_tiled(const TiledParams &p, void *ws, size_t ws_bytes, cudaStre
 // Modes: 0 never (default: it measures slower than the eight-warp kernel), 1 problems of at least 8 x 8
 // tiles, 2 whenever the operands allow it (tests, comparison runs).
 void round_fused_set_mode(int mode);
+void round_tiled_f32_set_tma_mode(int mode);
 // fp32 mode, tiled (round_tiled_f32.cu): X, L, U as fp64 device arrays, narrowed into the workspace
 size_t round_tiled_f32_workspace_bytes(int m, int n);
 int launch_round_tiled_f32(const TiledParams &p, void *ws, size_t ws_bytes, cudaStream_t stream);

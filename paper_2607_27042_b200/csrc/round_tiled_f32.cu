@@ -14,7 +14,10 @@
 // added through shared memory when a contraction ends.  (History at 8192 x 8192: 4 x 4 pieces, two CTAs
 // per SM, 30 % of the FMA pipe, 52.6 ms; 8 x 8 pieces in 512 threads 41.6 ms; 16 x 8 in 256 threads
 // 38.7 ms.)  Both operands of a slab are stored depth-major ([k][64 rows] and [k][64 columns]: L and C are
-// kept transposed in the workspace for this), staged with cp.async through a four-stage ring of slabs of 64.
+// kept transposed in the workspace for this) and arrive through a four-stage ring of slabs of 64: by bulk
+// tensor copies (TMA, one dense 64 x 64 box per operand and source, issued by one lane, counted by "full" /
+// "empty" mbarriers, no CTA barrier in the multiply loop, ragged edges by the copy engine's zero fill) where
+// the driver offers tensor maps, by cp.async with one CTA barrier per slab otherwise.
 // A thread cannot hold two accumulators of that size, so a tile runs three contractions one after the other:
 // Rt over the older tiles of its row, Cd over its whole column (the tile above comes last), Rt's last term
 // from the tile to the left -- the newest sources still come last; finished sums wait in shared memory.
@@ -33,8 +36,11 @@
 // written (an eager version that pushed every error down and right as Algorithm 3 prints it cost 7x the
 // time per step: 2 x 64 x 64 shared-memory updates per anti-diagonal, issued by every warp).
 #include <cstdio>
+#include <cstring>
 #include "common.cuh"
 #include "dmma_gemm.cuh"          // cp.async helpers
+#include "dmma_tma.cuh"           // mbarrier and bulk tensor copy helpers
+#include "tma_host.cuh"
 #include "round_internal.cuh"
 
 namespace gptq2d {
@@ -49,6 +55,9 @@ constexpr int KGROUPS = THREADS / 32;   // one warp a group, each KS / KGROUPS d
 constexpr int KG = KS / KGROUPS;
 constexpr int LDB = TS + 4;        // both slabs are [KS k][64], row stride 68 floats
 constexpr int SLAB_FLOATS = KS * LDB, STAGE_FLOATS = 2 * SLAB_FLOATS;
+constexpr int TMA_SLAB_FLOATS = KS * TS, TMA_STAGE_FLOATS = 2 * TMA_SLAB_FLOATS;     // dense boxes [KS k][64]
+constexpr unsigned TMA_STAGE_BYTES = TMA_STAGE_FLOATS * sizeof(float);
+constexpr int TMA_PREF = 2;        // slabs in flight ahead of the one being multiplied (one stage of slack for the slowest warp)
 constexpr int PMAT = TS * LDB;     // a group's partial tile, staged with the slabs' row stride
 constexpr int RPT = TS * TS / 4 / THREADS;   // float4 pieces of a tile per thread (rows (t >> 4) + (THREADS / 16) h)
 constexpr int LDT = TS + 16;       // in-tile matrices, row stride 80 floats = 16 banks mod 32: the two rows x four lanes of a quarter-warp
@@ -73,6 +82,8 @@ struct Params {
     double *max_abs_e;
     int *info;
     unsigned long long spin_limit;
+    int use_tma;                   // slabs by bulk tensor copies (tensor maps are separate kernel parameters)
+    int pad_;
 };
 
 __device__ __forceinline__ void cp_async16f(float *smem, const float *gmem, int src_bytes) {
@@ -124,19 +135,20 @@ struct Gemm {
         issue_one(As + SLAB_FLOATS, B, ldb, b_cols, kmax, k0);
     }
     // the thread's piece: rows 4 ty + (i & 3) + 16 (i >> 2), i < 16; columns 4 tx + (j & 3) + 32 (j >> 2), j < 8
-    __device__ __forceinline__ void multiply(float (&acc)[16][8], int stage) const {
-        const float *As = stages + stage * STAGE_FLOATS + gk * KG * LDB, *Bs = As + SLAB_FLOATS;
+    template <int LD, int SLAB>
+    __device__ __forceinline__ void multiply(float (&acc)[16][8], const float *stage) const {
+        const float *As = stage + gk * KG * LD, *Bs = As + SLAB;
 #pragma unroll
         for (int k = 0; k < KG; ++k) {
             float av[16], bv[8];
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
-                const float4 a = *reinterpret_cast<const float4 *>(As + k * LDB + 16 * h + 4 * ty);
+                const float4 a = *reinterpret_cast<const float4 *>(As + k * LD + 16 * h + 4 * ty);
                 av[4 * h + 0] = a.x; av[4 * h + 1] = a.y; av[4 * h + 2] = a.z; av[4 * h + 3] = a.w;
             }
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const float4 b = *reinterpret_cast<const float4 *>(Bs + k * LDB + 32 * h + 4 * tx);
+                const float4 b = *reinterpret_cast<const float4 *>(Bs + k * LD + 32 * h + 4 * tx);
                 bv[4 * h + 0] = b.x; bv[4 * h + 1] = b.y; bv[4 * h + 2] = b.z; bv[4 * h + 3] = b.w;
             }
 #pragma unroll
@@ -157,8 +169,12 @@ struct Gemm {
     }
 };
 
-__global__ void __launch_bounds__(THREADS, 1) round_tiled_f32_kernel(Params p) {
-    extern __shared__ __align__(16) float smem[];
+__global__ void __launch_bounds__(THREADS, 1)
+round_tiled_f32_kernel(Params p, const __grid_constant__ CUtensorMap mapL, const __grid_constant__ CUtensorMap mapE,
+                       const __grid_constant__ CUtensorMap mapC, const __grid_constant__ CUtensorMap mapU) {
+    extern __shared__ __align__(128) float smem[];
+    __shared__ __align__(8) unsigned long long s_full[NSTAGE], s_empty[NSTAGE];
+    __shared__ int s_fail, s_issued;
     __shared__ int s_task;
     __shared__ int s_ok, s_upto;
     __shared__ double s_red[THREADS / 32];
@@ -175,7 +191,15 @@ __global__ void __launch_bounds__(THREADS, 1) round_tiled_f32_kernel(Params p) {
     Gemm gm{stages, tid, tid >> 5, (tid & 31) >> 3, tid & 7};
     float *park_rt = smem + RING_FLOATS, *park_cd = park_rt + TS * TS;     // [64][64] each, behind the ring
     double max_abs_e = 0.0;
-    if (tid == 0) s_badkey = ~0ull;
+    if (tid == 0) {
+        s_badkey = ~0ull;
+        s_fail = 0;
+        if (p.use_tma) {
+            for (int i = 0; i < NSTAGE; ++i) { mbar_init(&s_full[i], 1u); mbar_init(&s_empty[i], (unsigned)KGROUPS); }
+            mbar_init_fence();
+        }
+    }
+    unsigned ring_it = 0;          // slabs that went through the TMA ring so far (the same in every thread)
 #ifdef TILED_STATS
     long long sw_sums = 0, sw_round = 0, sw_bar = 0;
     long long st_claim = 0, st_gemm = 0, st_form = 0, st_sweep = 0, st_store = 0, st_wait = 0, st_n = 0, st_t = clock64();
@@ -284,10 +308,105 @@ __global__ void __launch_bounds__(THREADS, 1) round_tiled_f32_kernel(Params p) {
                 if (g + NSTAGE - 1 < nslab) ok = issue_slab(g + NSTAGE - 1);
                 cp_async_commit();
                 if (!ok) break;
-                gm.multiply(acc, g % NSTAGE);
+                gm.multiply<LDB, SLAB_FLOATS>(acc, stages + (g % NSTAGE) * STAGE_FLOATS);
             }
             cp_async_wait<0>();
             __syncthreads();
+        };
+        // The same contraction with the slabs brought in by the copy engine: one bulk tensor copy per operand and
+        // source (a dense 64 x 64 box; what lies outside the matrix reads as zeros), completion counted by a "full"
+        // mbarrier per stage, the stage handed back through an "empty" mbarrier on which each warp arrives once.  No
+        // copy instruction, no address arithmetic and no CTA barrier sits in the multiply loop; the warps drift apart
+        // by up to a stage.  Warp 0 is also the producer: it checks the flags of the sources 32 at a time and its lane 0
+        // issues slab g + 2 before the warp multiplies slab g.  Every wait is bounded; one that runs out raises the abort
+        // word, and the pass then waits (bounded) for the copies still in flight before anyone leaves.
+        auto contract_tma = [&](int dir, int k0, int k1) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+            const int nslab = k1 - k0, lane = tid & 31;
+            const bool producer_warp = tid < 32;
+            const CUtensorMap *ma = dir == 0 ? &mapL : &mapC, *mb = dir == 0 ? &mapE : &mapU;
+            const int xa = row0, xb = col0;
+            int ready_upto = k0;
+            if (tid == 0) s_issued = 0;
+            bool good = true;
+            if (tid == 0) fence_proxy_async();           // the ring's memory was last touched by ordinary loads and stores
+            auto produce = [&](int q) {                  // warp 0, all lanes: slab q of this pass
+                const int k = k0 + q;
+                if (k >= ready_upto) {                   // flags of the next 32 sources in line, one per lane
+                    unsigned long long spins = 0;
+                    while (k >= ready_upto && good) {
+                        const int kk = ready_upto + lane;
+                        const unsigned *fl = dir == 0 ? p.flags + (long)kk * p.ntj + J : p.flags + (long)I * p.ntj + kk;
+                        const bool rdy = kk < k1 && ld_acquire_u32(fl) != 0u;
+                        const unsigned got = __ballot_sync(0xffffffffu, rdy);
+                        const int lead = got == 0xffffffffu ? 32 : __ffs(~got) - 1;
+                        ready_upto += lead;
+                        if (lead == 0) {
+                            if (++spins > p.spin_limit || ld_relaxed_u32(p.abort) != 0u) {
+                                if (lane == 0) {
+                                    report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -9, task, (int)blockIdx.x);
+                                    atomicExch(p.abort, 1u);
+                                }
+                                good = false;
+                            }
+                            __nanosleep(100);
+                        }
+                    }
+                    __syncwarp();                        // the lanes' acquires come before lane 0's copies
+                    if (lane == 0) fence_proxy_async();
+                }
+                if (!good) return;
+                if (lane == 0) {
+                    const unsigned it = ring_it + (unsigned)q;
+                    const int st = (int)(it % NSTAGE);
+                    if (it >= (unsigned)NSTAGE && !mbar_wait(&s_empty[st], ((it / NSTAGE) - 1u) & 1u, p.abort)) {
+                        report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -10, task, (int)blockIdx.x);
+                        atomicExch(p.abort, 1u);            // (the consumers' waits watch the abort word)
+                    } else {
+                        float *dst = stages + st * TMA_STAGE_FLOATS;
+                        mbar_arrive_expect_tx(&s_full[st], TMA_STAGE_BYTES);
+                        tma_load_2d(dst, ma, xa, k * TS, &s_full[st]);
+                        tma_load_2d(dst + TMA_SLAB_FLOATS, mb, xb, k * TS, &s_full[st]);
+                        s_issued = q + 1;
+                    }
+                }
+                __syncwarp();        // lane 0 rejoins the warp here, not somewhere inside the multiply that follows
+            };
+            if (producer_warp)
+                for (int q = 0; q < TMA_PREF && q < nslab && good; ++q) produce(q);
+            int g = 0;
+            for (; g < nslab && good; ++g) {
+                if (producer_warp && g + TMA_PREF < nslab) produce(g + TMA_PREF);
+                if (!good) break;
+                const unsigned it = ring_it + (unsigned)g;
+                const int st = (int)(it % NSTAGE);
+                if (!mbar_wait(&s_full[st], (it / NSTAGE) & 1u, p.abort)) {
+                    if (lane == 0) {
+                        report(p.info, GPTQ2D_ERR_DEVICE_TIMEOUT, -11, task, (int)blockIdx.x);
+                        atomicExch(p.abort, 1u);
+                    }
+                    good = false;
+                    break;
+                }
+                gm.multiply<TS, TMA_SLAB_FLOATS>(acc, stages + st * TMA_STAGE_FLOATS);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s_empty[st]);
+            }
+            if (!good) {
+                s_fail = 1;
+                // copies of this pass that may still be in flight: wait for them (bounded) before the memory is reused or left
+                if (tid == 0)
+                    for (int q = g; q < s_issued; ++q) {
+                        const unsigned it = ring_it + (unsigned)q;
+                        mbar_wait(&s_full[it % NSTAGE], (it / NSTAGE) & 1u, nullptr);
+                    }
+            }
+            ring_it += (unsigned)nslab;
+            __syncthreads();
+            if (s_fail) ok = false;
         };
         // Sum of the groups' partial tiles; thread t gets rows (t >> 4) + (THREADS / 16) h, columns 4 (t & 15) .. + 3.  The ring
         // is drained on entry and free again on return.
@@ -313,21 +432,21 @@ __global__ void __launch_bounds__(THREADS, 1) round_tiled_f32_kernel(Params p) {
         float4 v4[RPT];
         const bool far_rt = J > 1;
         if (far_rt) {
-            contract(1, 0, J - 1);
+            if (p.use_tma) contract_tma(1, 0, J - 1); else contract(1, 0, J - 1);
             if (!ok) break;
             reduce(v4);
 #pragma unroll
             for (int h = 0; h < RPT; ++h) *reinterpret_cast<float4 *>(park_rt + own + h * OWN_STEP) = v4[h];
         }
         if (I > 0) {
-            contract(0, 0, I);
+            if (p.use_tma) contract_tma(0, 0, I); else contract(0, 0, I);
             if (!ok) break;
             reduce(v4);
 #pragma unroll
             for (int h = 0; h < RPT; ++h) *reinterpret_cast<float4 *>(park_cd + own + h * OWN_STEP) = v4[h];
         }
         if (J > 0) {
-            contract(1, J - 1, J);
+            if (p.use_tma) contract_tma(1, J - 1, J); else contract(1, J - 1, J);
             if (!ok) break;
             reduce(v4);
         }
@@ -531,6 +650,7 @@ __global__ void __launch_bounds__(THREADS, 1) round_tiled_f32_kernel(Params p) {
     if (tid == 128 && (blockIdx.x % 61) == 0 && st_n > 0)
         printf("cta %3d row 32 per step: sums %lld rounding %lld barrier %lld\n", (int)blockIdx.x, sw_sums / (st_n * 128), sw_round / (st_n * 128),
                sw_bar / (st_n * 128));
+    if (tid == 0 && blockIdx.x == 0) printf("slabs by %s\n", p.use_tma ? "bulk tensor copies" : "cp.async");
     if (tid == 0 && (blockIdx.x % 61) == 0 && st_n > 0)
         printf("cta %3d tiles %lld | per tile: claim %lld gemm(+flag waits) %lld of which flag scans and waits %lld form %lld sweep %lld store %lld\n",
                (int)blockIdx.x, st_n, st_claim / st_n, st_gemm / st_n, st_wait / st_n, st_form / st_n, st_sweep / st_n, st_store / st_n);
@@ -598,6 +718,10 @@ static Layout layout(int m, int n) {
 
 size_t round_tiled_f32_workspace_bytes(int m, int n) { return f32::layout(m, n).total; }
 
+// 0: slabs by bulk tensor copies where the driver offers tensor maps; 1: always by cp.async (comparison, tests)
+static int g_f32_tma_mode = 0;
+void round_tiled_f32_set_tma_mode(int mode) { g_f32_tma_mode = mode; }
+
 int launch_round_tiled_f32(const TiledParams &in, void *ws, size_t ws_bytes, cudaStream_t stream) {
     using namespace f32;
     const Layout l = layout(in.m, in.n);
@@ -632,7 +756,15 @@ int launch_round_tiled_f32(const TiledParams &in, void *ws, size_t ws_bytes, cud
     if (per_sm > 1) per_sm = 1;
     int grid = sms * per_sm;
     if (grid > p.ntiles) grid = p.ntiles;
-    void *args[] = {&p};
+    // tensor maps of the four operand matrices (this GPU's own workspace; every CTA fetches its own boxes)
+    CUtensorMap mapL, mapE, mapC, mapU;
+    memset(&mapL, 0, sizeof(mapL)); memset(&mapE, 0, sizeof(mapE)); memset(&mapC, 0, sizeof(mapC)); memset(&mapU, 0, sizeof(mapU));
+    p.use_tma = g_f32_tma_mode == 0 &&
+                encode_f32_matrix_map(&mapL, L32, in.m, in.m, l.ldl, TS, KS) &&
+                encode_f32_matrix_map(&mapE, p.E32, l.mp, l.np, l.np, TS, KS) &&
+                encode_f32_matrix_map(&mapC, p.C32t, l.np, l.mp, l.mp, TS, KS) &&
+                encode_f32_matrix_map(&mapU, U32, in.n, in.n, l.ldu, TS, KS);
+    void *args[] = {&p, &mapL, &mapE, &mapC, &mapU};
     if (cudaLaunchCooperativeKernel((const void *)round_tiled_f32_kernel, dim3(grid), dim3(THREADS), args, SMEM_BYTES, stream) !=
         cudaSuccess)
         return GPTQ2D_ERR_CUDA;

@@ -1,4 +1,4 @@
-// Host side of the TMA path: tensor maps for fp64 operands (driver entry point looked up through the
+// Host side of the TMA path: tensor maps for fp64 and fp32 operands (driver entry point looked up through the
 // runtime, so the library has no link-time dependency on the driver library).
 #pragma once
 #include <cuda.h>
@@ -21,6 +21,12 @@ TensorMapEncodeTiledFn tensor_map_encoder();
 // Requirements (checked; false if not met): base 16-byte aligned, ld and batch_stride even.
 bool encode_f64_matrix_map(CUtensorMap *map, const double *base, long rows, long cols, long ld, long batch,
                            long batch_stride, int box_cols, int box_rows);
+
+// A row-major fp32 matrix (rows x cols, leading dimension ld) as a 2-D tensor {cols, rows} read in dense boxes of
+// box_cols x box_rows (no swizzle: the reader's lanes all sit in one row of the box at a time).  Out-of-range parts
+// of a box read as zeros.  Requirements (checked; false if not met): base 16-byte aligned, ld a multiple of 4,
+// box_cols a multiple of 4, both box extents at most 256.
+bool encode_f32_matrix_map(CUtensorMap *map, const float *base, long rows, long cols, long ld, int box_cols, int box_rows);
 
 inline bool tma_operand_ok(const double *base, long ld, long batch_stride) {
     return (reinterpret_cast<uintptr_t>(base) & 15) == 0 && (ld & 1) == 0 && (batch_stride & 1) == 0;

@@ -113,3 +113,38 @@ def test_fp32_ragged_multi_wave_repeatable_and_close_to_fp64(g):
     o64 = O.objective(X, Z64, A, B)
     assert abs(O.objective(X, Z1, A, B) - o64) <= 1e-3 * o64
     assert np.max(np.abs(E1)) <= 0.5 + 1e-5
+
+
+@pytest.mark.parametrize("m,n", [(200, 330), (515, 300), (129, 1100)])
+def test_fp32_poisoned_workspace(g, m, n):
+    """The fp32 copies of E and C^T in the workspace, and the padding of the transposed fp32 copy of L, are written
+    before they are read: a workspace filled with NaN patterns gives the Z, E and margin of a fresh one."""
+    X, A, B = W.headline_like(m, n, 23)
+    L, U, _, _ = O.feedback_factors(A, B)
+    dX, dL, dU = (torch.from_numpy(a).cuda() for a in (X, L, U))
+    nbytes = (g.gptq2d_round_workspace_bytes(m, n, g.FP32) + 7) // 8 * 8
+    fresh = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    Z0, E0, m0, i0 = g.gptq2d_round(dX, dL, dU, want_E=True, want_margin=True, precision=g.FP32, workspace=fresh)
+    poisoned = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    poisoned.view(torch.int32)[: nbytes // 4] = 0x7FC0BEEF             # a quiet NaN in every float
+    Z1, E1, m1, i1 = g.gptq2d_round(dX, dL, dU, want_E=True, want_margin=True, precision=g.FP32, workspace=poisoned)
+    torch.cuda.synchronize()
+    g.check_info(i0); g.check_info(i1)
+    assert torch.equal(Z0, Z1) and torch.equal(E0, E1) and float(m0[0]) == float(m1[0])
+
+
+@pytest.mark.parametrize("m,n", [(70, 100), (200, 330), (515, 300), (1000, 1300)])
+def test_fp32_slabs_by_tensor_copies_and_by_cp_async_agree(g, m, n):
+    """The contraction's operand slabs arrive by bulk tensor copies (the default; ragged edges are the copy engine's zero
+    fill) or by cp.async with clipping arithmetic (hook 6 = 1): same sums in the same order, so Z, E and the margin are
+    identical bit for bit, on shapes with ragged last tiles in both directions."""
+    X, A, B = W.headline_like(m, n, 31)
+    L, U, _, _ = O.feedback_factors(A, B)
+    try:
+        assert g._lib.gptq2d_internal_test_hook(6, 1) == 0
+        Zc, Ec, mc = run(g, X, L, U, g.FP32)
+        assert g._lib.gptq2d_internal_test_hook(6, 0) == 0
+        Zt, Et, mt = run(g, X, L, U, g.FP32)
+    finally:
+        g._lib.gptq2d_internal_test_hook(6, 0)
+    assert np.array_equal(Zc, Zt) and np.array_equal(Ec, Et) and mc == mt
