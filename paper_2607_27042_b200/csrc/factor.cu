@@ -398,10 +398,7 @@ int factor_one_side(int k, const double *M, long ldm, int side, double *out, lon
         CK(launch_gemm(t, s));
         return GPTQ2D_OK;
     };
-#ifndef FACTOR_OUTER
-#define FACTOR_OUTER 4
-#endif
-    constexpr int OUTER = FACTOR_OUTER;      // block rows per outer block (512 rows)
+    constexpr int OUTER = 4;                 // block rows per outer block (512 rows; 2, 6 and 8 measured slower at order 8192)
     if (look && nblk >= 4 * OUTER) {
         // Two-level right-looking factorisation.  The block rows are grouped four by four into outer blocks of 512
         // rows.  Inside an outer block S the 128-row steps run as before (diag, panel, update of the outer block's
