@@ -536,6 +536,10 @@ __device__ __forceinline__ void sweep_quadrant(int I, int J, int q, double *smem
     accC.zero();
     accR.zero();
     TS_RESET();
+    {   // X of the quadrant is read once, after the pulls, and comes from HBM: ask for it now (one 128-byte line per thread)
+        const int gr = row0 + (tid >> 2), gc = col0 + (tid & 3) * 16;
+        if (gr < p.m && gc < p.n) asm volatile("prefetch.global.L2 [%0];\n" ::"l"(p.X + (long)gr * p.ldx + gc));
+    }
     {
         const int r = 2 * I + qi, c = 2 * J + qj;
         const int fa = max(0, 2 * I - 4), fl = max(0, 2 * J - 4);
