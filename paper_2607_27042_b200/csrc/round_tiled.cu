@@ -691,7 +691,7 @@ __device__ __forceinline__ void load_acc(Acc &acc, const double *srcT, long np, 
 // ring from the sum over its matrices.
 constexpr unsigned QCAP = 4096;
 constexpr int FAR_RUN_CHUNKS = 64;      // a far part looks at the ready ring every this many K = 128 chunks
-constexpr unsigned IDLE_SLEEP_NS = 400; // pause of a CTA that found nothing to do
+constexpr unsigned IDLE_SLEEP_NS = 100; // pause of a CTA that found nothing to do (100 - 1600 ns and far runs of 8 - 64 chunks all time within 1 %)
 
 // multi-producer / multi-consumer ring in global memory; slot value 0 = empty.
 __device__ __forceinline__ void ready_push(const TiledKernelParams &p, unsigned entry) {
