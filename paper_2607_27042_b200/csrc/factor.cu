@@ -399,7 +399,9 @@ int factor_one_side(int k, const double *M, long ldm, int side, double *out, lon
         return GPTQ2D_OK;
     };
     constexpr int OUTER = 4;                 // block rows per outer block (512 rows; 2, 6 and 8 measured slower at order 8192)
-    if (look && nblk >= 4 * OUTER) {
+    // (orders below about 5 500 are faster with the one-level loop further down: 12.3 against 12.6 ms at 4096, 30.7
+    // against 30.0 at 6144, 67.9 against 61.8 at 8192)
+    if (look && nblk >= 44) {
         // Two-level right-looking factorisation.  The block rows are grouped four by four into outer blocks of 512
         // rows.  Inside an outer block S the 128-row steps run as before (diag, panel, update of the outer block's
         // own rows above the step), all on look->spine; the rows ABOVE the outer block receive the four panels in

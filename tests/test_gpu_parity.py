@@ -133,10 +133,10 @@ def test_factor_triangular_shortcut_needs_no_oracle(g):
 
 
 def test_factor_two_level_blocking_ragged(g):
-    """Orders of 16 block rows and more take the two-level route of the set-up (128-row steps inside outer blocks
-    of 512 rows, rank-512 updates above them); 2100 and 2300 give ragged last blocks at both levels and one side
+    """Orders of 44 block rows and more take the two-level route of the set-up (128-row steps inside outer blocks
+    of 512 rows, rank-512 updates above them); 5700 and 5889 give ragged last blocks at both levels and one side
     with a last outer block of a single block row."""
-    m, n = 2100, 2177
+    m, n = 5700, 5889
     X, A, B = W.general_bases(m, n, 5)
     A = A + np.sqrt(m) * np.eye(m)
     B = B + np.sqrt(n) * np.eye(n)
