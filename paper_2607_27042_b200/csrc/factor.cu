@@ -384,7 +384,7 @@ int factor_one_side(int k, const double *M, long ldm, int side, double *out, lon
         return GPTQ2D_OK;
     };
     // the same update with the panels of block rows [K0, K1) at once (contraction over all their rows): a rank-128
-    // update runs at 16 TFLOP/s, rank 256 at 22, rank 512 at 28 (measured, 8192^2 target, C read and rewritten)
+    // update runs at 23.5 TFLOP/s, rank 256 at 28, rank 512 at 31.5 (measured, 8192^2 target, C read and rewritten)
     auto trailing_multi = [&](int K0, int K1, long r0, long r1, cudaStream_t s) -> int {
         const long k0 = (long)K0 * FB;
         const long k1 = (long)K1 * FB < k ? (long)K1 * FB : k;
@@ -399,8 +399,8 @@ int factor_one_side(int k, const double *M, long ldm, int side, double *out, lon
         return GPTQ2D_OK;
     };
     constexpr int OUTER = 4;                 // block rows per outer block (512 rows; 2, 6 and 8 measured slower at order 8192)
-    // (orders below about 5 500 are faster with the one-level loop further down: 12.3 against 12.6 ms at 4096, 30.7
-    // against 30.0 at 6144, 67.9 against 61.8 at 8192)
+    // (orders below about 5 500 are faster with the one-level loop further down: 11.9 against 12.2 ms at 4096, 28.9
+    // against 29.2 at 6144, but 62.0 against 60.2 at 8192)
     if (look && nblk >= 44) {
         // Two-level right-looking factorisation.  The block rows are grouped four by four into outer blocks of 512
         // rows.  Inside an outer block S the 128-row steps run as before (diag, panel, update of the outer block's

@@ -67,6 +67,31 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(GemmArgs p) {
 
     double *Cb = p.C + (long)bz * p.strideC;
     const bool vec = ((((uintptr_t)Cb) & 15) == 0) && ((p.ldc & 1) == 0);
+    if (p.beta != 0.0 && vec && m0 + BM <= p.M && n0 + BN <= p.N) {
+        // Update of a full tile (the rank-k updates of the set-up): the old values are read in two batches of sixteen
+        // 16-byte loads per thread before anything is stored, so that the loads of a batch are in flight together
+        // (loads and stores to the same matrix one after the other run as a chain of dependent round trips).
+        double *c00 = Cb + (long)(m0 + wm * 64 + g) * p.ldc + n0 + wn * 32 + t * 2;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            double2 old[4][4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b)
+                    old[a][b] = *reinterpret_cast<const double2 *>(c00 + (long)((half * 4 + a) * 8) * p.ldc + b * 8);
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    double2 o;
+                    o.x = fma(p.beta, old[a][b].x, p.alpha * acc.v[half * 4 + a][b][0]);
+                    o.y = fma(p.beta, old[a][b].y, p.alpha * acc.v[half * 4 + a][b][1]);
+                    *reinterpret_cast<double2 *>(c00 + (long)((half * 4 + a) * 8) * p.ldc + b * 8) = o;
+                }
+        }
+        return;
+    }
 #pragma unroll
     for (int a = 0; a < 8; ++a) {
         int r = m0 + wm * 64 + a * 8 + g;
@@ -173,6 +198,36 @@ gemm_tma_kernel(GemmArgs p, const __grid_constant__ CUtensorMap mapA, const __gr
 
     double *Cb = p.C + (long)bz * p.strideC;
     const bool vec = ((((uintptr_t)Cb) & 15) == 0) && ((p.ldc & 1) == 0);
+    if (p.beta != 0.0 && vec && m0 + BM <= p.M && n0 + BN <= p.N) {
+        // update of a full tile: old values read in two batches of sixteen 16-byte loads before anything is stored (see the
+        // cp.async kernel above)
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            double2 old[4][4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    int col;
+                    double x0, x1;
+                    acc_pair<B_KCONTIG>(acc, half * 4 + a, q, wn, t, col, x0, x1);
+                    old[a][q] = *reinterpret_cast<const double2 *>(Cb + (long)(m0 + acc_row<A_KCONTIG>(wm, half * 4 + a, g)) * p.ldc + n0 + col);
+                }
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    int col;
+                    double x0, x1;
+                    acc_pair<B_KCONTIG>(acc, half * 4 + a, q, wn, t, col, x0, x1);
+                    double2 o;
+                    o.x = fma(p.beta, old[a][q].x, p.alpha * x0);
+                    o.y = fma(p.beta, old[a][q].y, p.alpha * x1);
+                    *reinterpret_cast<double2 *>(Cb + (long)(m0 + acc_row<A_KCONTIG>(wm, half * 4 + a, g)) * p.ldc + n0 + col) = o;
+                }
+        }
+        return;
+    }
 #pragma unroll
     for (int a = 0; a < 8; ++a) {
         const int r = m0 + acc_row<A_KCONTIG>(wm, a, g);
