@@ -11,7 +11,8 @@ constexpr int GEMM_NSTAGE = 3;
 template <bool A_KCONTIG, bool B_KCONTIG>
 __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(GemmArgs p) {
     extern __shared__ __align__(16) double smem[];
-    const int tn = blockIdx.x, tm = blockIdx.y, bz = blockIdx.z;
+    // (with a lower-triangular A the contraction of tile row tm is tm + 1 blocks long: the longest rows are started first)
+    const int tn = blockIdx.x, tm = p.a_lower ? (int)(gridDim.y - 1 - blockIdx.y) : (int)blockIdx.y, bz = blockIdx.z;
     if (p.lower_tiles_only && tn > tm) return;
     const int m0 = tm * BM, n0 = tn * BN;
     const double *Ab = p.A + (long)bz * p.strideA;
@@ -150,7 +151,8 @@ gemm_tma_kernel(GemmArgs p, const __grid_constant__ CUtensorMap mapA, const __gr
                 unsigned *abort) {
     extern __shared__ __align__(16) double smem_raw[];
     __shared__ __align__(8) unsigned long long bars[2 * GEMM_TMA_NSTAGE];
-    const int tn = blockIdx.x, tm = blockIdx.y, bz = blockIdx.z;
+    // (with a lower-triangular A the contraction of tile row tm is tm + 1 blocks long: the longest rows are started first)
+    const int tn = blockIdx.x, tm = p.a_lower ? (int)(gridDim.y - 1 - blockIdx.y) : (int)blockIdx.y, bz = blockIdx.z;
     if (p.lower_tiles_only && tn > tm) return;
     const int m0 = tm * BM, n0 = tn * BN;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
