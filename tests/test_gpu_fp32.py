@@ -148,3 +148,25 @@ def test_fp32_slabs_by_tensor_copies_and_by_cp_async_agree(g, m, n):
     finally:
         g._lib.gptq2d_internal_test_hook(6, 0)
     assert np.array_equal(Zc, Zt) and np.array_equal(Ec, Et) and mc == mt
+
+
+def test_fp32_random_shapes_both_slab_feeds_agree_and_stay_close_to_fp64(g):
+    """Twelve seeded random shapes up to 330 x 330 (one to six tiles a side, ragged edges of every width class): the two
+    slab feeds give identical Z and E, |E| stays within one half, and the rounding differs from the fp64 sweep's in at
+    most a few per cent of the entries."""
+    rng = np.random.default_rng(2024)
+    for case in range(12):
+        m, n = int(rng.integers(1, 331)), int(rng.integers(1, 331))
+        X, A, B = W.general_bases(m, n, 100 + case)
+        L, U, _, _ = O.feedback_factors(A, B)
+        try:
+            assert g._lib.gptq2d_internal_test_hook(6, 1) == 0
+            Zc, Ec, mc = run(g, X, L, U, g.FP32)
+            assert g._lib.gptq2d_internal_test_hook(6, 0) == 0
+            Zt, Et, mt = run(g, X, L, U, g.FP32)
+        finally:
+            g._lib.gptq2d_internal_test_hook(6, 0)
+        assert np.array_equal(Zc, Zt) and np.array_equal(Ec, Et) and mc == mt, (m, n)
+        assert np.max(np.abs(Et)) <= 0.5 + 1e-5, (m, n)
+        Z64, _, _ = run(g, X, L, U, g.FP64)
+        assert float(np.mean(Zt != Z64)) <= 0.05, (m, n)
