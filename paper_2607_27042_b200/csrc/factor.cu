@@ -25,8 +25,8 @@ constexpr int FB = 128;
 // One CTA.  S: bs x bs Schur complement (lower triangle read).  Writes P (lower, in place),
 // W = P^{-1} (full block, zeros above the diagonal) and diag(P).
 // The block is padded to 128 x 128 with the identity in shared memory.  Cholesky runs from the last
-// index to the first (one column scaling + one rank-one update of the leading part per step, 16 x 16
-// thread tiling); the inverse is built from 32 x 32 diagonal blocks by doubling,
+// index to the first, blocked sixteen rows at a time (row scaling + rank-one update of the block's own rows
+// per step, one rank-16 DMMA update of the rows above per block); the inverse is built from 32 x 32 diagonal blocks by doubling,
 // W21 = -W22 (P21 W11), both products as m8n8k4 DMMA fragments, with the temporary product kept in
 // the unused upper triangle of the P array.
 __device__ __forceinline__ int tri(int i, int j) { return i * (i + 1) / 2 + j; }   // packed lower triangle
@@ -37,57 +37,92 @@ __device__ __forceinline__ int tri(int i, int j) { return i * (i + 1) / 2 + j; }
 // Ends with a barrier.  err_c: what a non-positive pivot reports in info[3], beside its index and the side.
 __device__ __forceinline__ void chol_inverse_128(double *a, double *w, int bs, int *info, int side, int k0, int err_c) {
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-    // Two barriers per step: the scaled row k goes to `prow` (the packed W array is free until the inverse),
-    // so the update below never reads what the scaling writes in place.
-    double *prow = w;
-    for (int k = bs - 1; k >= 0; --k) {
-        double d = a[k * 129 + k];
-        if (!(d > 0.0) || !isfinite(d)) {
-            if (tid == 0) report(info, GPTQ2D_ERR_NOT_SPD, k0 + k, side, err_c);
-            d = 1.0;
-        }
-        double rk = rsqrt(d);
-        rk = rk * fma(-0.5 * d, rk * rk, 1.5);                 // one Newton step: 1 / sqrt(d) to the last bit or two
-        if (tid < k) {
-            const double val = a[k * 129 + tid] * rk;          // P[k][tid]
-            a[k * 129 + tid] = val;
-            prow[tid] = val;
-        }
-        __syncthreads();                                       // everyone has read d; prow is complete
-        if (tid == 0) a[k * 129 + k] = d * rk;
-        // Schur complement of the leading k x k part (lower triangle).  Each thread's entries of four rows
-        // are read into registers before anything is stored, so that the loads are in flight together
-        // (loads and stores of the same array cannot be reordered by the compiler).  Every index is < 128,
-        // so the loads are unconditional; only the stores are masked.
-        {
-            double pj[8];
+    // Blocked, sixteen rows R = [r_lo, r_hi) at a time from the last block to the first, three barriers a block:
+    //  (1) warp 0 factors the block's own 16 x 16 part in place (the unblocked steps -- scale row k, rank-one update of
+    //      the rows of R above k -- between warp barriers only) and leaves 1 / P[k][k] in s_rk;
+    //  (2) every column j < r_lo of the block's rows is a triangular solve of its own, one thread per column, sixteen
+    //      values in registers:  P[k][j] = (A[k][j] - sum_{k' in R, k' > k} P[k'][k] P[k'][j]) / P[k][k],  k descending;
+    //  (3) the rows above the block receive the block's sixteen rank-one updates at once, as 8 x 8 fragments of the
+    //      lower triangle on the fp64 tensor path (four m8n8k4 products each).
+    // (The unblocked loop rewrote up to 128 x 128 entries of shared memory per step behind two CTA barriers: 57 of the
+    // kernel's 102 us.)  Rows from bs on are identity padding: they factor to the identity and contribute nothing.
+    __shared__ double s_rk[16];
+    // warp 0's share of the 16 x 16 lower triangle in (1): entries e = lane + 32 u -> (ii, jj), jj <= ii, row by row
+    int tri_i[4], tri_j[4];
 #pragma unroll
-            for (int jj = 0; jj < 8; ++jj) pj[jj] = prow[tx + 16 * jj];
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                if (64 * half >= k) break;                     // rows 64 .. 127 are done once k <= 64
-                double pi[4], v[4][8];
-#pragma unroll
-                for (int ii = 0; ii < 4; ++ii) {
-                    const int R = 4 * half + ii, i = ty + 16 * R;
-                    pi[ii] = prow[i];
-                    // only the 16 x 16 tiles that meet the lower triangle of the leading k x k part
-                    // (the same for the whole warp): the loop is bound by shared-memory bandwidth
-#pragma unroll
-                    for (int jj = 0; jj < 8; ++jj) v[ii][jj] = (jj <= R && 16 * R < k) ? a[i * 129 + tx + 16 * jj] : 0.0;
+    for (int u = 0; u < 4; ++u) {
+        int ii = 0, r = (tid & 31) + 32 * u;
+        while (r > ii) { r -= ii + 1; ++ii; }
+        tri_i[u] = ii; tri_j[u] = r;
+    }
+    for (int kb = (bs - 1) >> 4; kb >= 0; --kb) {
+        const int r_lo = 16 * kb;
+        if (tid < 32) {
+            for (int kk = 15; kk >= 0; --kk) {
+                const int k = r_lo + kk;
+                double d = a[k * 129 + k];
+                if (!(d > 0.0) || !isfinite(d)) {
+                    if (tid == 0) report(info, GPTQ2D_ERR_NOT_SPD, k0 + k, side, err_c);
+                    d = 1.0;
                 }
+                double rk = rsqrt(d);
+                rk = rk * fma(-0.5 * d, rk * rk, 1.5);         // one Newton step: 1 / sqrt(d) to the last bit or two
+                // entries (i, j) of the rows of R above k, r_lo <= j <= i < k: at most 120, four per lane
+                double v[4], pi[4], pj[4];
+                int at[4];
 #pragma unroll
-                for (int ii = 0; ii < 4; ++ii) {
-                    const int i = ty + 16 * (4 * half + ii);
-#pragma unroll
-                    for (int jj = 0; jj < 8; ++jj) {
-                        const int j = tx + 16 * jj;
-                        if (i < k && j <= i) a[i * 129 + j] = fma(-pi[ii], pj[jj], v[ii][jj]);
-                    }
+                for (int u = 0; u < 4; ++u) {
+                    const bool on = tri_i[u] < kk;
+                    at[u] = on ? (r_lo + tri_i[u]) * 129 + r_lo + tri_j[u] : -1;
+                    v[u] = on ? a[at[u]] : 0.0;
+                    pi[u] = on ? a[k * 129 + r_lo + tri_i[u]] * rk : 0.0;
+                    pj[u] = on ? a[k * 129 + r_lo + tri_j[u]] * rk : 0.0;
                 }
+                __syncwarp();
+                if (tid < kk) a[k * 129 + r_lo + tid] *= rk;   // P[k][r_lo + tid]
+                if (tid == 0) { a[k * 129 + k] = d * rk; s_rk[kk] = rk; }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (at[u] >= 0) a[at[u]] = fma(-pi[u], pj[u], v[u]);
+                __syncwarp();
             }
         }
         __syncthreads();
+        if (kb > 0 && tid < r_lo) {
+            double x[16];
+#pragma unroll
+            for (int kk = 0; kk < 16; ++kk) x[kk] = a[(r_lo + kk) * 129 + tid];
+#pragma unroll
+            for (int kk = 15; kk >= 0; --kk) {
+                double sum = x[kk];
+#pragma unroll
+                for (int k2 = 15; k2 > kk; --k2) sum = fma(-a[(r_lo + k2) * 129 + r_lo + kk], x[k2], sum);
+                x[kk] = sum * s_rk[kk];
+            }
+#pragma unroll
+            for (int kk = 0; kk < 16; ++kk) a[(r_lo + kk) * 129 + tid] = x[kk];
+        }
+        __syncthreads();
+        if (kb > 0) {
+            // leading (16 kb) x (16 kb) lower triangle -= P[R, :]^T P[R, :]
+            const int warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+            const int nb = 2 * kb, nfrag = nb * (nb + 1) / 2;
+            for (int f = warp; f < nfrag; f += 8) {
+                int bi = 0, r = f;
+                while (r > bi) { r -= bi + 1; ++bi; }
+                const int bj = r;
+                double c0 = 0.0, c1 = 0.0;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const double *row = a + (r_lo + 4 * kk + t) * 129;
+                    dmma_m8n8k4(c0, c1, row[8 * bi + g], row[8 * bj + g]);
+                }
+                const int ri = 8 * bi + g, cj = 8 * bj + 2 * t;
+                if (cj <= ri) a[ri * 129 + cj] -= c0;
+                if (cj + 1 <= ri) a[ri * 129 + cj + 1] -= c1;
+            }
+            __syncthreads();
+        }
     }
     // ---- W = P^{-1}.  Level 0: the four 32 x 32 diagonal blocks, one column per thread.
     if (tid < 128) {
@@ -152,26 +187,29 @@ __global__ void __launch_bounds__(256) factor_diag_kernel(double *S, long lds, i
     double *a = sm;               // [128][129]: P in the lower triangle, scratch above it
     double *w = sm + 128 * 129;   // packed lower triangle of W
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-    // the block, padded with the identity: eight loads in flight per thread
-    for (int base = 0; base < 128 * 128; base += 8 * 256) {
-        double v[8];
+    // the block, padded with the identity: the kernel sits on the serial spine of the set-up, so a thread's 64 loads
+    // are issued in two batches of 32 (entry idx = 256 u + tid: a warp reads 32 consecutive columns of one row)
+    for (int base = 0; base < 128 * 128; base += 32 * 256) {
+        double v[32];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < 32; ++u) {
             const int idx = base + u * 256 + tid, i = idx >> 7, j = idx & 127;
             v[u] = (j <= i && i < bs) ? S[(long)i * lds + j] : (i == j ? 1.0 : 0.0);
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < 32; ++u) {
             const int idx = base + u * 256 + tid, i = idx >> 7, j = idx & 127;
             if (j <= i) a[i * 129 + j] = v[u];
         }
     }
     __syncthreads();
     chol_inverse_128(a, w, bs, info, side, k0, 0);
-    for (int idx = tid; idx < bs * bs; idx += blockDim.x) {
-        int i = idx / bs, j = idx - i * bs;
-        if (j <= i) S[(long)i * lds + j] = a[i * 129 + j];
-        W[(long)i * ldw + j] = (j <= i) ? w[tri(i, j)] : 0.0;
+    for (int idx = tid; idx < 128 * 128; idx += 256) {
+        const int i = idx >> 7, j = idx & 127;
+        if (i < bs && j < bs) {
+            if (j <= i) S[(long)i * lds + j] = a[i * 129 + j];
+            W[(long)i * ldw + j] = (j <= i) ? w[tri(i, j)] : 0.0;
+        }
     }
     for (int i = tid; i < bs; i += blockDim.x) pdiag[i] = a[i * 129 + i];
 }
