@@ -132,6 +132,21 @@ def test_factor_triangular_shortcut_needs_no_oracle(g):
     assert np.allclose(Ld.cpu().numpy(), np.linalg.inv(A) @ np.diag(np.diag(A)), atol=1e-11)
 
 
+@pytest.mark.parametrize("m,n", [(1, 1), (15, 17), (16, 33), (127, 129), (130, 257), (300, 515)])
+def test_factor_orders_around_the_block_sizes(g, m, n):
+    """Orders just below, at and above the 16-row blocks of the diagonal-block kernel and the 128-row blocks of the
+    factorisation, against the oracle's factors."""
+    rng = np.random.default_rng(1000 * m + n)
+    A = rng.standard_normal((m, m)) / np.sqrt(m) + 2 * np.eye(m)
+    B = rng.standard_normal((n, n)) / np.sqrt(n) + 2 * np.eye(n)
+    L, U, lamL, lamU = O.feedback_factors(A, B)
+    Ld, Ud, dL, dU, info = g.gptq2d_factor(dev(A), dev(B))
+    torch.cuda.synchronize()
+    g.check_info(info)
+    assert np.max(np.abs(Ld.cpu().numpy() - L)) < 1e-11 and np.max(np.abs(Ud.cpu().numpy() - U)) < 1e-11
+    assert np.allclose(dL.cpu().numpy(), 1 / lamL, rtol=1e-11) and np.allclose(dU.cpu().numpy(), 1 / lamU, rtol=1e-11)
+
+
 def test_factor_two_level_blocking_ragged(g):
     """Orders of 44 block rows and more take the two-level route of the set-up (128-row steps inside outer blocks
     of 512 rows, rank-512 updates above them); 5700 and 5889 give ragged last blocks at both levels and one side
